@@ -1,0 +1,283 @@
+"""CPU oracle for the elastic (masked) backward pass of a stack of dense layers.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain float64 statement of what
+the CUDA library computes.  It shares no code with the CUDA path and must never be
+imported by it; only tests, the smoke check and the benchmark's CPU-baseline leg
+use it.  numpy's matmul is the one library primitive used as a step.
+
+Conventions (the paper, Sections 2.2, 3.3 and 5): layers and tensors are indexed
+in forward execution order, 0 = nearest the input.  Tensor 2*l is the kernel of
+layer l, tensor 2*l+1 its bias.  Layer l computes
+
+    Z_l     = a_l @ W_l + b_l                       a_l : [M, K_l], W_l : [K_l, N_l]
+    H_l     = act_l(Z_l)
+    a_{l+1} = sum of `fold` equal column slices of H_l  (+ a_j if residual_src = j)
+
+Pins (tests/test_oracle_*.py): central finite differences of the loss for every
+tensor and every layer kind; the closed form of the importance sum when the update
+is a gradient step; the first-order Taylor identity of Eq. (6); masked == full
+backprop on the selected tensors and all-selected == full; the two worked examples
+the paper prints for the time model (Section 2.2) and for f(M) (Eq. 3); brute-force
+enumeration for the selector.  The paper prints no numeric gradients or importances,
+so beyond those pins the values are unpinned against the paper itself.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
+STRICT, INCLUSIVE = 0, 1
+
+_C0 = np.sqrt(2.0 / np.pi)
+_C1 = 0.044715
+
+
+# --------------------------------------------------------------------------- activations
+def act_forward(z: np.ndarray, act: int) -> np.ndarray:
+    if act == ACT_NONE:
+        return z
+    if act == ACT_RELU:
+        return np.where(z > 0.0, z, 0.0)
+    if act == ACT_GELU_TANH:
+        # tanh form of GELU: 0.5 z (1 + tanh( sqrt(2/pi) (z + 0.044715 z^3) ))
+        return 0.5 * z * (1.0 + np.tanh(_C0 * (z + _C1 * z ** 3)))
+    raise ValueError(act)
+
+
+def act_derivative(z: np.ndarray, act: int) -> np.ndarray:
+    if act == ACT_NONE:
+        return np.ones_like(z)
+    if act == ACT_RELU:
+        return np.where(z > 0.0, 1.0, 0.0)
+    if act == ACT_GELU_TANH:
+        u = _C0 * (z + _C1 * z ** 3)
+        t = np.tanh(u)
+        du = _C0 * (1.0 + 3.0 * _C1 * z ** 2)
+        return 0.5 * (1.0 + t) + 0.5 * z * (1.0 - t * t) * du
+    raise ValueError(act)
+
+
+# --------------------------------------------------------------------------- forward
+@dataclass
+class Saved:
+    a: List[np.ndarray]    # a[0] = input, a[l+1] = output of layer l
+    Z: List[np.ndarray]    # pre-activations
+
+
+def forward(layers, W: Sequence[np.ndarray], b: Sequence[np.ndarray], x: np.ndarray) -> Saved:
+    """Forward pass of every layer (the forward time is the same for any selection,
+    Eq. 3), keeping what the backward pass needs."""
+    a = [np.asarray(x, dtype=np.float64)]
+    Z = []
+    for l, ly in enumerate(layers):
+        z = a[l] @ np.asarray(W[l], dtype=np.float64) + np.asarray(b[l], dtype=np.float64)
+        h = act_forward(z, ly.act)
+        w = ly.out_features // ly.fold
+        out = np.zeros((h.shape[0], w))
+        for s in range(ly.fold):
+            out = out + h[:, s * w:(s + 1) * w]
+        if ly.residual_src >= 0:
+            out = out + a[ly.residual_src]
+        Z.append(z)
+        a.append(out)
+    return Saved(a=a, Z=Z)
+
+
+def mse_loss(y: np.ndarray, target: np.ndarray) -> float:
+    """Mean over all M*D elements of (y - target)^2."""
+    return float(np.mean((y - target) ** 2))
+
+
+def mse_loss_grad(y: np.ndarray, target: np.ndarray):
+    n = y.size
+    return mse_loss(y, target), 2.0 * (y - target) / n
+
+
+# --------------------------------------------------------------------------- which work runs
+@dataclass
+class Plan:
+    deepest: int               # smallest layer index owning a selected tensor; L if none
+    dgrad: np.ndarray          # bool[L]  error gradient passed through layer l (dX_l computed)
+    wgrad: np.ndarray          # bool[L]  kernel gradient computed
+    bgrad: np.ndarray          # bool[L]  bias gradient computed
+    updated: np.ndarray        # bool[2L] tensor written by the update
+
+
+def exec_plan(L: int, mask: Sequence[int]) -> Plan:
+    """Section 2.2: a selected layer pays its own weight-gradient time, and every
+    LATER layer pays its error-gradient time whether selected or not; nothing at or
+    before the deepest selected layer passes a gradient further down."""
+    mask = np.asarray(mask).astype(bool)
+    assert mask.shape == (2 * L,)
+    sel_layers = [l for l in range(L) if mask[2 * l] or mask[2 * l + 1]]
+    d = min(sel_layers) if sel_layers else L
+    return Plan(
+        deepest=d,
+        dgrad=np.array([l > d for l in range(L)]),
+        wgrad=np.array([bool(mask[2 * l]) for l in range(L)]),
+        bgrad=np.array([bool(mask[2 * l + 1]) for l in range(L)]),
+        updated=mask.copy(),
+    )
+
+
+def executed_flops(layers, M: int, plan: Plan) -> float:
+    """2*M*K*N per executed GEMM (dgrad and wgrad of one layer cost the same)."""
+    fl = 0.0
+    for l, ly in enumerate(layers):
+        g = 2.0 * M * ly.in_features * ly.out_features
+        fl += g * (int(plan.dgrad[l]) + int(plan.wgrad[l]))
+    return fl
+
+
+# --------------------------------------------------------------------------- backward
+def _backward_sweep(layers, W, saved: Saved, dY: np.ndarray, stop: int,
+                    want_w, want_b) -> Dict[int, np.ndarray]:
+    """Reverse sweep over layers L-1 ... stop.  G[i] accumulates dL/da_i."""
+    L = len(layers)
+    G: List[Optional[np.ndarray]] = [None] * (L + 1)
+    G[L] = np.asarray(dY, dtype=np.float64)
+    grads: Dict[int, np.ndarray] = {}
+    for l in range(L - 1, stop - 1, -1):
+        ly = layers[l]
+        g_out = G[l + 1]
+        if ly.residual_src >= 0:
+            j = ly.residual_src
+            G[j] = g_out.copy() if G[j] is None else G[j] + g_out
+        # gradient w.r.t. H_l: each of the `fold` slices receives g_out
+        dH = np.concatenate([g_out] * ly.fold, axis=1)
+        dZ = dH * act_derivative(saved.Z[l], ly.act)
+        if want_w[l]:
+            grads[2 * l] = saved.a[l].T @ dZ                    # dW = X^T dZ
+        if want_b[l]:
+            grads[2 * l + 1] = dZ.sum(axis=0)                   # db = column sums
+        if l > stop:
+            dX = dZ @ np.asarray(W[l], dtype=np.float64).T      # dX = dZ W^T
+            G[l] = dX if G[l] is None else G[l] + dX
+    return grads
+
+
+def backward_masked(layers, W, saved: Saved, dY: np.ndarray, mask):
+    """Elastic backward: the sweep stops at the deepest selected layer, kernel /
+    bias gradients are formed only for selected tensors."""
+    L = len(layers)
+    plan = exec_plan(L, mask)
+    if plan.deepest == L:
+        return {}, plan
+    grads = _backward_sweep(layers, W, saved, dY, plan.deepest, plan.wgrad, plan.bgrad)
+    return grads, plan
+
+
+def backward_full(layers, W, saved: Saved, dY: np.ndarray) -> Dict[int, np.ndarray]:
+    """Plain full backprop: every gradient of every tensor."""
+    L = len(layers)
+    return _backward_sweep(layers, W, saved, dY, 0, [True] * L, [True] * L)
+
+
+# --------------------------------------------------------------------------- importance, update
+def importance(grads: Dict[int, np.ndarray], delta: Sequence[np.ndarray], mask) -> np.ndarray:
+    """Eq. (2): S_k = sum_i (dL/dw_i^k) * (delta w_i^k), for every selected tensor k;
+    0 for the others."""
+    out = np.zeros(len(mask))
+    for k, m in enumerate(mask):
+        if m:
+            out[k] = float(np.sum(grads[k] * np.asarray(delta[k], dtype=np.float64)))
+    return out
+
+
+def sgd_masked(params: Sequence[np.ndarray], grads: Dict[int, np.ndarray], mask, lr: float):
+    """w <- w - lr * g for selected tensors; the others are returned untouched
+    (same object, so a caller can check they were not rewritten)."""
+    out = []
+    for k, p in enumerate(params):
+        out.append(p - lr * grads[k] if mask[k] else p)
+    return out
+
+
+def tensors_of(W, b):
+    """Interleave kernels and biases into tensor order [W_0, b_0, W_1, b_1, ...]."""
+    out = []
+    for w_, b_ in zip(W, b):
+        out += [w_, b_]
+    return out
+
+
+# --------------------------------------------------------------------------- time model, selector
+def f_mask(mask) -> np.ndarray:
+    """Eq. (3): f(M) marks every tensor whose error-gradient time is paid; for any
+    selected tensor all later ones are included (and, in the example the paper
+    prints, the selected one itself)."""
+    m = np.asarray(mask).astype(bool)
+    return np.logical_or.accumulate(m).astype(np.uint8)
+
+
+def t_selective(mask, t_dw, t_dy, variant: int = STRICT) -> float:
+    """Backward time of a selection.  STRICT follows the Section 2.2 example and
+    Eq. (7): only tensors AFTER the deepest selected one pay t_dy.  INCLUSIVE is the
+    f(M) of the Eq. (3) example, where the deepest selected tensor pays it too."""
+    m = np.asarray(mask).astype(bool)
+    t_dw = np.asarray(t_dw, dtype=np.float64)
+    t_dy = np.asarray(t_dy, dtype=np.float64)
+    if not m.any():
+        return 0.0
+    f = f_mask(m).astype(bool)
+    if variant == STRICT:
+        f = f.copy()
+        f[int(np.argmax(m))] = False
+    return float(t_dw[m].sum() + t_dy[f].sum())
+
+
+def quantise(t_dw, t_dy, t_fwd: float, rho: float, Tq: int):
+    """Eq. (8): t~ = floor(t * Z), Z = Tq / T with T the full backward time.  The
+    budget for the backward pass is rho * T_full - T_fwd, T_full = T_fwd + T,
+    floored the same way."""
+    t_dw = np.asarray(t_dw, dtype=np.float64)
+    t_dy = np.asarray(t_dy, dtype=np.float64)
+    T = float(t_dw.sum() + t_dy.sum())
+    Z = Tq / T
+    qw = np.floor(t_dw * Z).astype(np.int64)
+    qy = np.floor(t_dy * Z).astype(np.int64)
+    budget = int(np.floor((rho * (t_fwd + T) - t_fwd) * Z))
+    return qw, qy, budget
+
+
+def select_bruteforce(I, qw, qy, budget: int, variant: int = STRICT):
+    """Enumerate all 2^n masks of the integer-cost problem
+    max M.I  s.t.  M.t_dw + f(M).t_dy <= budget   (Eq. 3 without the constant T_fwd)."""
+    I = np.asarray(I, dtype=np.float64)
+    n = len(I)
+    best_val, best_mask = 0.0, np.zeros(n, dtype=np.uint8)
+    for code in range(1, 1 << n):
+        m = np.array([(code >> i) & 1 for i in range(n)], dtype=np.uint8)
+        if t_selective(m, qw, qy, variant) <= budget:
+            v = float(I[m.astype(bool)].sum())
+            if v > best_val:
+                best_val, best_mask = v, m
+    return best_mask, best_val
+
+
+def select_by_depth_knapsack(I, qw, qy, budget: int, variant: int = STRICT) -> float:
+    """Second, independent route to the optimum: fix the deepest selected tensor d
+    (it must be selected and fixes all t_dy charges), then the rest is a 0/1
+    knapsack on t_dw over the tensors after d."""
+    I = np.asarray(I, dtype=np.float64)
+    n = len(I)
+    best = 0.0
+    for d in range(n):
+        fixed = qw[d] + qy[d + 1:].sum() + (qy[d] if variant == INCLUSIVE else 0)
+        cap = budget - fixed
+        if cap < 0:
+            continue
+        knap = np.zeros(cap + 1)
+        for i in range(d + 1, n):
+            if I[i] <= 0:
+                continue
+            w = int(qw[i])
+            if w == 0:
+                knap = knap + I[i]
+            elif w <= cap:
+                knap[w:] = np.maximum(knap[w:], knap[:-w] + I[i])
+        best = max(best, I[d] + knap[cap])
+    return float(best)

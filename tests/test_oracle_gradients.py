@@ -1,0 +1,181 @@
+"""Pins of the oracle's floating-point parts against what mathematics fixes:
+central finite differences of the loss, hand-computed 2x2 case, masked-vs-full
+invariants, closed form of the importance sum, first-order Taylor identity."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from oracle import elastic_oracle as orc
+
+
+def _loss(layers, W, b, x, target):
+    return orc.mse_loss(orc.forward(layers, W, b, x).a[-1], target)
+
+
+def _all_kinds_stack():
+    # every activation, a 3-way fold, two kinds of residual wiring, ragged widths
+    return [
+        wl.Layer(6, 9, fold=3),                                  # 0: fold, out width 3
+        wl.Layer(3, 6, residual_src=0),                          # 1: residual from the stack input (width 6)
+        wl.Layer(6, 10, act=wl.ACT_GELU_TANH),                   # 2
+        wl.Layer(10, 6, residual_src=2),                         # 3: residual from a_2
+        wl.Layer(6, 5, act=wl.ACT_RELU),                         # 4
+        wl.Layer(5, 6, act=wl.ACT_GELU_TANH, residual_src=4),    # 5: activation AND residual
+        wl.Layer(6, 4),                                          # 6
+    ]
+
+
+def _fd_check(layers, M, seed, h=1e-6, tol=2e-6):
+    w = wl.small_stack(layers, M, wl.DT_F32, seed, w_std=0.4, bias_std=0.3)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    grads = orc.backward_full(w.layers, w.W, saved, dY)
+    rng = np.random.default_rng(seed + 100)
+    for l in range(len(layers)):
+        for t, arr_list in ((2 * l, w.W), (2 * l + 1, w.b)):
+            p = arr_list[l]
+            g = grads[t]
+            assert g.shape == p.shape
+            idxs = [tuple(rng.integers(0, s) for s in p.shape) for _ in range(12)]
+            for idx in idxs:
+                old = p[idx]
+                p[idx] = old + h
+                lp = _loss(w.layers, w.W, w.b, w.x, w.target)
+                p[idx] = old - h
+                lm = _loss(w.layers, w.W, w.b, w.x, w.target)
+                p[idx] = old
+                fd = (lp - lm) / (2 * h)
+                scale = max(abs(fd), np.abs(g).max() * 1e-3, 1e-12)
+                assert abs(fd - g[idx]) / scale < tol, (l, t, idx, fd, g[idx])
+
+
+def test_finite_differences_all_layer_kinds():
+    _fd_check(_all_kinds_stack(), M=7, seed=11)
+
+
+def test_finite_differences_vit_and_mlp_wiring():
+    _fd_check(wl.vit_blocks(2, 6, 10), M=5, seed=5)
+    _fd_check(wl.mlp_blocks(2, 4, 7, wl.ACT_RELU), M=6, seed=6)
+
+
+def test_single_layer_by_hand():
+    # L = 1, no activation: dW = X^T dY, db = column sums, checked entry by entry
+    layers = [wl.Layer(2, 2)]
+    X = np.array([[1.0, 2.0], [3.0, -1.0]])
+    W = [np.array([[0.5, -1.0], [2.0, 0.25]])]
+    b = [np.array([0.1, -0.2])]
+    saved = orc.forward(layers, W, b, X)
+    assert np.allclose(saved.a[1], [[1 * .5 + 2 * 2 + .1, -1 + .5 - .2], [1.5 - 2 + .1, -3 - .25 - .2]])
+    dY = np.array([[1.0, 0.0], [0.0, 2.0]])
+    g = orc.backward_full(layers, W, saved, dY)
+    assert np.array_equal(g[0], [[1.0, 6.0], [2.0, -2.0]])
+    assert np.array_equal(g[1], [1.0, 2.0])
+
+
+def test_dgrad_orientation_two_layers_by_hand():
+    # two linear layers: dW_0 = X^T (dY W_1^T); a transposed operand fails this
+    layers = [wl.Layer(2, 3), wl.Layer(3, 2)]
+    rng = np.random.default_rng(0)
+    X, W0, W1 = rng.normal(size=(4, 2)), rng.normal(size=(2, 3)), rng.normal(size=(3, 2))
+    dY = rng.normal(size=(4, 2))
+    saved = orc.forward(layers, [W0, W1], [np.zeros(3), np.zeros(2)], X)
+    g = orc.backward_full(layers, [W0, W1], saved, dY)
+    want = np.zeros((2, 3))
+    for i in range(2):
+        for j in range(3):
+            for m in range(4):
+                for n in range(2):
+                    want[i, j] += X[m, i] * dY[m, n] * W1[j, n]
+    assert np.allclose(g[0], want, rtol=1e-12, atol=1e-12)
+
+
+def test_gelu_tanh_known_values():
+    # tanh-GELU at 0 is 0 with slope 1/2; for large |z| it tends to z and 0
+    z = np.array([0.0, 10.0, -10.0, 1.0])
+    v = orc.act_forward(z, orc.ACT_GELU_TANH)
+    assert v[0] == 0.0 and abs(v[1] - 10.0) < 1e-12 and abs(v[2]) < 1e-12
+    assert abs(v[3] - 0.8411919906082768) < 1e-12   # 0.5*(1+tanh(sqrt(2/pi)*1.044715))
+    d = orc.act_derivative(z, orc.ACT_GELU_TANH)
+    assert d[0] == 0.5 and abs(d[1] - 1.0) < 1e-9 and abs(d[2]) < 1e-9
+
+
+def test_masked_is_subset_of_full_and_all_selected_is_full():
+    w = wl.small_stack(_all_kinds_stack(), 9, wl.DT_F32, 3, w_std=0.3, bias_std=0.2)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    full = orc.backward_full(w.layers, w.W, saved, dY)
+    rng = np.random.default_rng(0)
+    for _ in range(20):
+        mask = (rng.random(2 * w.L) < 0.3).astype(np.uint8)
+        grads, plan = orc.backward_masked(w.layers, w.W, saved, dY, mask)
+        assert sorted(grads) == [k for k in range(2 * w.L) if mask[k]]
+        for k in grads:
+            assert np.array_equal(grads[k], full[k])      # same arithmetic, bit-identical
+    ones = np.ones(2 * w.L, dtype=np.uint8)
+    grads, plan = orc.backward_masked(w.layers, w.W, saved, dY, ones)
+    assert plan.deepest == 0 and plan.dgrad.sum() == w.L - 1
+    for k in range(2 * w.L):
+        assert np.array_equal(grads[k], full[k])
+
+
+def test_importance_closed_form_for_gradient_step():
+    # Eq. (2) with delta = -lr * g  =>  S_k = -lr * ||g_k||^2
+    w = wl.small_stack(wl.vit_blocks(1, 6, 8), 5, wl.DT_F32, 8, w_std=0.3)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    full = orc.backward_full(w.layers, w.W, saved, dY)
+    lr = 0.05
+    delta = [-lr * full[k] for k in range(2 * w.L)]
+    mask = np.ones(2 * w.L, dtype=np.uint8)
+    S = orc.importance(full, delta, mask)
+    for k in range(2 * w.L):
+        assert abs(S[k] + lr * np.sum(full[k] ** 2)) <= 1e-14 * max(1.0, abs(S[k]))
+    # independent delta: brute-force double loop on one kernel
+    rng = np.random.default_rng(1)
+    dl = [rng.normal(size=full[k].shape) for k in range(2 * w.L)]
+    S = orc.importance(full, dl, mask)
+    acc = 0.0
+    for i in range(full[4].shape[0]):
+        for j in range(full[4].shape[1]):
+            acc += full[4][i, j] * dl[4][i, j]
+    assert abs(acc - S[4]) < 1e-12
+    # unselected tensors report 0
+    mask[3] = 0
+    assert orc.importance(full, dl, mask)[3] == 0.0
+
+
+def test_importance_is_first_order_loss_change():
+    # Eq. (6): L(w + dw) - L(w) = sum_k S_k + O(|dw|^2); the residual falls 4x when dw halves
+    w = wl.small_stack(wl.mlp_blocks(2, 5, 9, wl.ACT_GELU_TANH), 6, wl.DT_F32, 4, w_std=0.4, bias_std=0.1)
+    params = orc.tensors_of(w.W, w.b)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    L0, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    full = orc.backward_full(w.layers, w.W, saved, dY)
+    mask = np.ones(2 * w.L, dtype=np.uint8)
+    res = []
+    for lr in (0.004, 0.002, 0.001):
+        delta = [-lr * full[k] for k in range(2 * w.L)]
+        S = orc.importance(full, delta, mask).sum()
+        new = orc.sgd_masked(params, full, mask, lr)
+        L1 = _loss(w.layers, new[0::2], new[1::2], w.x, w.target)
+        assert L1 < L0 and S < 0
+        res.append((L1 - L0) - S)
+    assert 3.5 < res[0] / res[1] < 4.5 and 3.5 < res[1] / res[2] < 4.5
+    assert abs(res[2]) < 0.05 * abs(S)
+
+
+def test_sgd_masked_leaves_frozen_tensors_alone():
+    w = wl.small_stack(wl.mlp_blocks(1, 4, 6, wl.ACT_RELU), 3, wl.DT_F32, 2)
+    params = orc.tensors_of(w.W, w.b)
+    grads = {k: np.ones_like(p) for k, p in enumerate(params)}
+    mask = np.array([1, 0, 0, 1], dtype=np.uint8)
+    new = orc.sgd_masked(params, grads, mask, 0.5)
+    assert new[1] is params[1] and new[2] is params[2]
+    assert np.array_equal(new[0], params[0] - 0.5) and np.array_equal(new[3], params[3] - 0.5)
+
+
+def test_mse_gradient_normalisation():
+    y = np.array([[1.0, 2.0], [3.0, 5.0]])
+    t = np.zeros((2, 2))
+    loss, g = orc.mse_loss_grad(y, t)
+    assert loss == (1 + 4 + 9 + 25) / 4 and np.array_equal(g, y / 2)

@@ -1,0 +1,204 @@
+"""Seeded synthetic workloads shared by the CUDA path's tests/bench and by the CPU oracle.
+
+This module holds shapes, wiring and random draws only. It contains none of the
+method's arithmetic (no GEMM, no activation, no gradient, no importance, no
+selection): both sides receive the same arrays from here and compute on their own.
+
+Layer / tensor indexing is forward execution order, 0 = nearest the input
+(the paper lists trainable tensors in execution order, Section 5).  Tensor
+``2*l`` is the kernel of layer ``l`` and tensor ``2*l + 1`` its bias
+(Section 5.1: a dense layer carries a Kernel and a Bias tensor).
+
+The stacks stand in for the models the paper trains (ViT, ResNet50; Section 8)
+with every non-dense operator replaced by the identity, so that the whole
+backward pass is dense-layer work.  No dataset item is reproduced: inputs and
+targets are N(0,1) draws.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import numpy as np
+
+# activation / post-op codes (mirrored by include/et.h)
+ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
+DT_F32, DT_BF16 = 0, 1
+
+
+@dataclass(frozen=True)
+class Layer:
+    in_features: int
+    out_features: int          # width of Z = X W + b
+    act: int = ACT_NONE
+    fold: int = 1              # output = sum of `fold` equal column slices of act(Z)
+    residual_src: int = -1     # -1, or j: add activation a_j (a_0 = stack input,
+                               # a_{j+1} = output of layer j) to this layer's output
+
+    @property
+    def out_width(self) -> int:
+        return self.out_features // self.fold
+
+
+@dataclass
+class Workload:
+    name: str
+    layers: List[Layer]
+    M: int                     # tokens (rows)
+    dtype: int                 # storage type of weights / activations
+    lr: float
+    mask: np.ndarray           # uint8[2L], tensor order
+    W: List[np.ndarray] = field(default_factory=list)   # float64 values, exactly representable in `dtype`
+    b: List[np.ndarray] = field(default_factory=list)
+    x: Optional[np.ndarray] = None
+    target: Optional[np.ndarray] = None
+
+    @property
+    def L(self) -> int:
+        return len(self.layers)
+
+
+# --------------------------------------------------------------------------- rounding of inputs
+def round_to_bf16(a: np.ndarray) -> np.ndarray:
+    """Round float values to the nearest bfloat16 (ties to even); returns float64
+    holding exactly those bf16 values.  Used only so that both sides start from
+    identical input bits."""
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    lsb = (u >> 16) & 1
+    u = (u + 0x7FFF + lsb) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(a.shape)
+
+
+def round_to_f32(a: np.ndarray) -> np.ndarray:
+    return np.asarray(a, dtype=np.float32).astype(np.float64)
+
+
+def to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """uint16 bit patterns of values that are already exactly bf16-representable."""
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    return (f.view(np.uint32) >> 16).astype(np.uint16).reshape(a.shape)
+
+
+def from_bf16_bits(u: np.ndarray) -> np.ndarray:
+    return (u.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _store(a: np.ndarray, dtype: int) -> np.ndarray:
+    return round_to_bf16(a) if dtype == DT_BF16 else round_to_f32(a)
+
+
+# --------------------------------------------------------------------------- stack shapes
+def mlp_blocks(n_blocks: int, d: int, hidden: int, act: int) -> List[Layer]:
+    """[Linear d->hidden, act, Linear hidden->d, + block input] repeated."""
+    layers: List[Layer] = []
+    for blk in range(n_blocks):
+        base = 2 * blk
+        layers.append(Layer(d, hidden, act=act))
+        layers.append(Layer(hidden, d, residual_src=base))
+    return layers
+
+
+def vit_blocks(n_blocks: int, d: int, ffn: int) -> List[Layer]:
+    """Transformer block with the attention core replaced by identity:
+    QKV d->3d whose three slices are summed, out-proj d->d + block input,
+    fc1 d->ffn with tanh-GELU, fc2 ffn->d + fc1's input."""
+    layers: List[Layer] = []
+    for blk in range(n_blocks):
+        base = 4 * blk
+        layers.append(Layer(d, 3 * d, fold=3))
+        layers.append(Layer(d, d, residual_src=base))
+        layers.append(Layer(d, ffn, act=ACT_GELU_TANH))
+        layers.append(Layer(ffn, d, residual_src=base + 2))
+    return layers
+
+
+# --------------------------------------------------------------------------- draws
+def _draw_params(rng, layers, dtype, w_std=None, he_init=False):
+    W, b = [], []
+    for ly in layers:
+        std = np.sqrt(2.0 / ly.in_features) if he_init else w_std
+        W.append(_store(rng.normal(0.0, std, size=(ly.in_features, ly.out_features)), dtype))
+        b.append(np.zeros(ly.out_features, dtype=np.float64))
+    return W, b
+
+
+def bernoulli_weight_mask(rng, L: int, p: float) -> np.ndarray:
+    """One Bernoulli(p) draw per kernel tensor; each bias follows its kernel."""
+    bits = (rng.random(L) < p).astype(np.uint8)
+    return np.repeat(bits, 2)
+
+
+def _finish(name, layers, M, dtype, lr, mask, rng, w_std=None, he_init=False, params=True):
+    wl = Workload(name=name, layers=layers, M=M, dtype=dtype, lr=lr, mask=mask)
+    if params:
+        wl.W, wl.b = _draw_params(rng, layers, dtype, w_std=w_std, he_init=he_init)
+        wl.x = _store(rng.normal(size=(M, layers[0].in_features)), dtype)
+        wl.target = _store(rng.normal(size=(M, layers[-1].out_width)), dtype)
+    return wl
+
+
+def tiny_mlp(seed: int = 0, params: bool = True) -> Workload:
+    """fp32, 2 blocks of [128->512, tanh-GELU, 512->128, residual], 256 tokens;
+    only the first layer of block 2 (kernel + bias) is selected."""
+    rng = np.random.default_rng(seed)
+    layers = mlp_blocks(2, 128, 512, ACT_GELU_TANH)
+    mask = np.zeros(2 * len(layers), dtype=np.uint8)
+    mask[4] = mask[5] = 1
+    return _finish("tiny_mlp_fp32", layers, 256, DT_F32, 0.01, mask, rng, w_std=0.02, params=params)
+
+
+def vit_b(seed: int = 1, p_select: float = 0.3, n_blocks: int = 12, tokens: int = 64 * 197,
+          d: int = 768, ffn: int = 3072, params: bool = True, name: str = "vit_b_linear_bf16") -> Workload:
+    """bf16 ViT-B/16-shaped linear-only stack, Bernoulli(p_select) mask over kernels."""
+    rng = np.random.default_rng(seed)
+    layers = vit_blocks(n_blocks, d, ffn)
+    mask = bernoulli_weight_mask(rng, len(layers), p_select)
+    return _finish(name, layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
+
+
+def vit_l(seed: int = 3, params: bool = True, n_blocks: int = 24, tokens: int = 32 * 197,
+          d: int = 1024, ffn: int = 4096) -> Workload:
+    """bf16 ViT-L-shaped linear-only stack; the mask starts all-selected and is
+    replaced by the selector while training."""
+    rng = np.random.default_rng(seed)
+    layers = vit_blocks(n_blocks, d, ffn)
+    mask = np.ones(2 * len(layers), dtype=np.uint8)
+    return _finish("vit_l_linear_bf16", layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
+
+
+def resnet_1x1(seed: int = 2, p_select: float = 0.5, n_blocks: int = 6, tokens: int = 32 * 14 * 14,
+               params: bool = True) -> Workload:
+    """bf16 ResNet-50 conv4_x 1x1 bottleneck convs as NHWC GEMMs:
+    [1024->256, ReLU, 256->1024 (3x3 replaced by identity), + block input]."""
+    rng = np.random.default_rng(seed)
+    layers = mlp_blocks(n_blocks, 1024, 256, ACT_RELU)
+    mask = bernoulli_weight_mask(rng, len(layers), p_select)
+    return _finish("resnet50_conv4_1x1_bf16", layers, tokens, DT_BF16, 0.01, mask, rng,
+                   he_init=True, params=params)
+
+
+def small_stack(layers: List[Layer], M: int, dtype: int, seed: int, mask=None, w_std: float = 0.05,
+                bias_std: float = 0.0, lr: float = 0.01) -> Workload:
+    """Arbitrary small stack for parity and oracle tests (ragged sizes, every act/fold/residual kind)."""
+    rng = np.random.default_rng(seed)
+    if mask is None:
+        mask = (rng.random(2 * len(layers)) < 0.5).astype(np.uint8)
+    wl = _finish("small", layers, M, dtype, lr, np.asarray(mask, dtype=np.uint8), rng, w_std=w_std)
+    if bias_std > 0:
+        wl.b = [_store(rng.normal(0.0, bias_std, size=ly.out_features), dtype) for ly in layers]
+    return wl
+
+
+def selector_instance(rng, n: int, t_max: int = 20, integer: bool = True):
+    """Random importances and per-tensor costs for selector tests (biases get t_dy = 0
+    on odd indices, Section 5.1)."""
+    I = rng.random(n)
+    if integer:
+        t_dw = rng.integers(0, t_max, size=n).astype(np.float64)
+        t_dy = rng.integers(0, t_max, size=n).astype(np.float64)
+    else:
+        t_dw = rng.random(n) * t_max
+        t_dy = rng.random(n) * t_max
+    t_dy[1::2] = 0.0
+    return I, t_dw, t_dy
