@@ -1,0 +1,214 @@
+/*
+ * et.h -- C ABI of the elastic (masked) backward pass of a stack of dense layers.
+ *
+ * The operation is the one ElasticTrainer's tensor selection speeds up (arXiv
+ * 2312.14227): given a binary selection mask over the trainable tensors, listed in
+ * forward execution order (Section 5), the backward pass
+ *   - passes the error gradient  dX_l = dZ_l * W_l^T  only through layers AFTER the
+ *     deepest selected one (Section 2.2: an unselected layer still passes gradients,
+ *     nothing at or below the deepest selected layer does),
+ *   - forms the weight gradient  dW_l = X_l^T * dZ_l  and the bias gradient
+ *     db_l = column sums of dZ_l  only for selected tensors (Section 5.1: the three
+ *     backward operations of a dense layer),
+ *   - reduces the first-order tensor importance  S_k = sum_i g_i * dw_i  (Eq. 2),
+ *   - and updates the selected tensors only.
+ *
+ * Conventions
+ *   Layers l = 0..L-1 in forward order, 0 nearest the input.  Tensor 2l is the kernel
+ *   W_l [in_features x out_features], row-major (out_features contiguous); tensor
+ *   2l+1 is the bias b_l [out_features].  Activations are [M x features], row-major.
+ *       Z_l     = a_l * W_l + b_l
+ *       H_l     = act_l(Z_l)
+ *       a_{l+1} = sum of the `fold` equal column slices of H_l  (+ a_j if residual_src = j)
+ *   a_0 is the stack input; the width of a_{l+1} is out_features / fold.
+ *
+ *   Storage type (et_dtype) applies to weights, biases, activations, error gradients
+ *   and delta-W; accumulation is always fp32.  Exported gradients and importances are
+ *   fp32.  ET_BF16 stacks run on tcgen05 tensor cores and need every feature count to
+ *   be a multiple of 8, and out_features/fold a multiple of 256 when fold > 1.
+ *
+ * Memory and errors
+ *   Every "device" pointer is caller-owned CUDA device memory, 16-byte aligned, valid
+ *   until the work enqueued on `stream` has finished.  Arrays of pointers, masks and
+ *   reports are host memory, read before the call returns.  The library allocates no
+ *   device memory: one caller-provided workspace (et_stack_workspace_bytes) holds
+ *   saved activations, error gradients, split-K partials and a status word.
+ *   Arguments are validated on the host before anything is launched; a call that
+ *   returns an error has enqueued nothing.  Calls are asynchronous on `stream`
+ *   (a cudaStream_t passed as void*, NULL = default stream) unless stated otherwise.
+ *   Calls on one stack must not overlap on the GPU (they share the workspace).
+ */
+#ifndef ET_H_
+#define ET_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ET_OK = 0,
+  ET_ERR_INVALID_ARG = 1,   /* null pointer, bad enum, bad length */
+  ET_ERR_SHAPE = 2,         /* layer widths do not chain, residual width mismatch */
+  ET_ERR_DTYPE = 3,
+  ET_ERR_STATE = 4,         /* not bound, backward before forward */
+  ET_ERR_WORKSPACE = 5,     /* workspace too small or misaligned */
+  ET_ERR_UNSUPPORTED = 6,   /* shape outside what the kernels handle */
+  ET_ERR_CUDA = 7,          /* a CUDA runtime call failed; see et_last_cuda_error */
+  ET_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up */
+} et_status;
+
+typedef enum { ET_F32 = 0, ET_BF16 = 1 } et_dtype;
+typedef enum { ET_ACT_NONE = 0, ET_ACT_GELU_TANH = 1, ET_ACT_RELU = 2 } et_act;
+
+/* Cost-model reading for the selector (Section 2.2 / Eq. 7 versus the example after Eq. 3). */
+typedef enum {
+  ET_COST_STRICT = 0,      /* tensors after the deepest selected one pay t_dy */
+  ET_COST_INCLUSIVE = 1    /* the deepest selected tensor pays its own t_dy too */
+} et_cost_variant;
+
+enum {
+  ET_FLAG_FUSE_SGD = 1u    /* et_backward_elastic also applies w <- w - lr*g to selected tensors */
+};
+
+typedef struct {
+  int32_t in_features;
+  int32_t out_features;
+  int32_t act;            /* et_act; must be ET_ACT_NONE when fold > 1 */
+  int32_t fold;           /* >= 1, divides out_features */
+  int32_t residual_src;   /* -1, or j in [0, l]: add a_j to this layer's output */
+} et_layer_desc;
+
+/* What one et_backward_elastic call executed.  The four arrays are caller-owned host
+ * memory (any may be NULL): dgrad/wgrad/bgrad have L entries, updated has 2L. */
+typedef struct {
+  uint8_t* dgrad;
+  uint8_t* wgrad;
+  uint8_t* bgrad;
+  uint8_t* updated;
+  int32_t deepest;          /* smallest layer index owning a selected tensor; L if none */
+  int32_t launches;         /* kernels enqueued by the call */
+  double flops_executed;    /* 2*M*K*N per executed dgrad / wgrad GEMM */
+} et_exec_report;
+
+typedef struct et_stack et_stack;
+
+/* ---- stack object (host) ---------------------------------------------------------- */
+
+/* Validates the layer chain and builds the host-side plan.  M = rows (tokens). */
+et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_dtype dtype,
+                          et_stack** out);
+et_status et_stack_destroy(et_stack* s);
+
+/* Bytes of device workspace et_stack_bind needs (a multiple of 256). */
+et_status et_stack_workspace_bytes(const et_stack* s, size_t* bytes);
+
+/* Attaches parameters and workspace.  W, b: host arrays of L device pointers (storage
+ * dtype).  The workspace must be 256-byte aligned.  The library zeroes what it needs on
+ * `stream`.  May be called again to re-attach. */
+et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/* ---- forward and loss (precede the hot path; Eq. 3's T_forward) -------------------- */
+
+/* x: device [M x in_features(0)], y: device [M x width(a_L)], storage dtype.  Saves every
+ * a_l and the pre-activations of activated layers in the workspace.  x itself is
+ * referenced, not copied: it must stay valid and unchanged until the backward call that
+ * uses this forward pass has finished. */
+et_status et_forward_stack(et_stack* s, const void* x, void* y, void* stream);
+
+/* Mean-squared error over all M*D elements and its gradient dY = 2 (y - target) / (M*D).
+ * y, target, dY: device, storage dtype; loss_dev: device float (may be NULL). */
+et_status et_loss_mse_grad(et_stack* s, const void* y, const void* target, void* dY,
+                           float* loss_dev, void* stream);
+
+/* ---- the hot path ----------------------------------------------------------------- */
+
+/* Elastic backward (Section 2.2, Section 5.1, Eq. 2).
+ *   dY         device [M x width(a_L)], storage dtype: dL/da_L.
+ *   mask       host uint8[n_tensors], n_tensors must equal 2L; non-zero = selected.
+ *   grads      host array of 2L device float* (or NULL array): where selected gradients
+ *              are written, dW_l as [in x out] row-major, db_l as [out].  An entry may be
+ *              NULL when the gradient itself is not wanted.  Entries of unselected
+ *              tensors are ignored and their buffers never touched.
+ *   delta      host array of 2L device pointers, storage dtype, same shapes as the
+ *              tensors (or NULL array): the recent update dw of Eq. 2.  If given,
+ *              importance_dev must be given too, and every selected tensor needs an entry.
+ *   importance_dev  device float[2L]: S_k for selected tensors, 0 for the others.
+ *   flags, lr  ET_FLAG_FUSE_SGD applies w <- w - lr*g (Section 2.2's weight update) to
+ *              selected tensors inside the same call, after every read of the old weight.
+ *              Unselected tensors are never written.
+ *   report     host, optional.
+ * Nothing is launched for layers below the deepest selected one; with an empty mask
+ * nothing is launched at all except zeroing importance_dev.  Needs a preceding
+ * et_forward_stack on the same stack. */
+et_status et_backward_elastic(et_stack* s, const void* dY, const uint8_t* mask, int32_t n_tensors,
+                              float* const* grads, const void* const* delta,
+                              float* importance_dev, uint32_t flags, float lr,
+                              et_exec_report* report, void* stream);
+
+/* Same call for host-resident buffers: copies dY (host, storage dtype) to the device,
+ * runs et_backward_elastic, copies the 2L importances back to importance_host (if delta
+ * is given) and synchronises `stream` before returning.  dY_host / importance_host should
+ * be pinned for full copy bandwidth.  grads / delta stay device pointers as above. */
+et_status et_backward_elastic_host(et_stack* s, const void* dY_host, const uint8_t* mask,
+                                   int32_t n_tensors, float* const* grads,
+                                   const void* const* delta, float* importance_host,
+                                   uint32_t flags, float lr, et_exec_report* report, void* stream);
+
+/* Stand-alone Eq. 2 on already materialised gradients: importance_dev[k] =
+ * sum(grads[k] * delta[k]) for selected k, 0 otherwise. */
+et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads,
+                        const void* const* delta, float* importance_dev, void* stream);
+
+/* Stand-alone masked SGD: w_k <- w_k - lr * grads[k] for selected k (fp32 arithmetic,
+ * rounded once to the storage dtype).  Unselected tensors are never written. */
+et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads,
+                        float lr, void* stream);
+
+/* ---- selection support (host) ------------------------------------------------------ */
+
+/* Times each layer's dgrad and wgrad(+bias) launches with CUDA events (median of `iters`)
+ * and fills per-TENSOR cost vectors of length 2L following Section 5.1: kernel tensor:
+ * t_dw = weight-gradient time, t_dy = error-gradient time (with the fused backward of the
+ * non-trainable work below it, Section 5.3); bias tensor: t_dw = bias-gradient time,
+ * t_dy = 0.  t_fwd receives the forward time.  Milliseconds.  Synchronous.  Runs a forward
+ * pass from x (writing y) and a full backward from dY first; weights are not changed. */
+et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, int32_t iters,
+                           double* t_dw, double* t_dy, double* t_fwd, void* stream);
+
+/* Backward time of a selection under the model of Section 2.2 / Eq. 3 (host arithmetic). */
+et_status et_time_selective(const uint8_t* mask, const double* t_dw, const double* t_dy,
+                            int32_t n, int32_t variant, double* t_out);
+
+/* Tensor selector (Section 6): maximise sum of importance[k] over selected k subject to
+ * t_fwd + selected t_dw + charged t_dy <= rho * (t_fwd + sum t_dw + sum t_dy), by dynamic
+ * programming over (depth from the output, quantised time), times quantised with
+ * Eq. 8 at resolution Tq.  Host only, synchronous.  mask_out: uint8[n]; value_out: the
+ * optimum of the quantised problem; est_time_out: unquantised backward time of the mask. */
+et_status et_select_dp(const double* importance, const double* t_dw, const double* t_dy, int32_t n,
+                       double t_fwd, double rho, int32_t Tq, int32_t variant,
+                       uint8_t* mask_out, double* value_out, double* est_time_out);
+
+/* Same problem with integer costs given directly (no quantisation step). */
+et_status et_select_dp_int(const double* importance, const int64_t* t_dw, const int64_t* t_dy,
+                           int32_t n, int64_t budget, int32_t variant,
+                           uint8_t* mask_out, double* value_out);
+
+/* ---- status ------------------------------------------------------------------------ */
+
+/* Synchronises `stream` and reports ET_ERR_TIMEOUT if a kernel's bounded wait gave up,
+ * ET_ERR_CUDA if the stream is in error, else ET_OK. */
+et_status et_device_status(et_stack* s, void* stream);
+const char* et_status_string(et_status st);
+/* cudaError_t of the last failing CUDA call seen by this thread (0 if none). */
+int32_t et_last_cuda_error(void);
+/* Number of kernels this library has launched in this process. */
+int64_t et_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ET_H_ */

@@ -1,0 +1,208 @@
+// Memory-bound kernels: split-K reduction with the fused importance / SGD epilogue, bias
+// gradient (column sums), stand-alone importance and SGD, activation backward for the top
+// layer, MSE loss gradient.  16-byte accesses, fixed-order reductions (results do not
+// depend on scheduling).
+#pragma once
+
+#include "common.cuh"
+
+namespace et {
+
+constexpr int kEltThreads = 256;
+constexpr int kVec = 8;                         // elements per thread per step
+constexpr int kColsumRows = 128;                // rows per column-sum chunk
+
+// ---- weight gradient: sum the K-split partials, then everything that consumes g ----------
+//   g = sum_s partial[s]                       (fixed order s = 0, 1, ...)
+//   grad        <- g                           if grad != nullptr
+//   imp_part[b] <- sum over this block of g * delta     if delta != nullptr   (Eq. 2)
+//   W           <- W - lr * g                  if do_sgd   (fp32 arithmetic, one rounding)
+template <typename T>
+__global__ void __launch_bounds__(kEltThreads)
+wgrad_reduce_kernel(const float* __restrict__ partial, int splits, size_t split_stride, size_t count,
+                    float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
+                    T* __restrict__ W, float lr, int do_sgd) {
+  const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
+  float dot = 0.0f;
+  if (i0 < count) {
+    const int n = (int)min((size_t)kVec, count - i0);
+    float g[kVec], t[kVec];
+    load_seg<kVec>(partial + i0, n, g);
+    for (int s = 1; s < splits; ++s) {
+      load_seg<kVec>(partial + (size_t)s * split_stride + i0, n, t);
+#pragma unroll
+      for (int i = 0; i < kVec; ++i) g[i] += t[i];
+    }
+    if (grad != nullptr) store_seg<kVec>(grad + i0, n, g);
+    if (delta != nullptr) {
+      load_seg<kVec>(delta + i0, n, t);
+#pragma unroll
+      for (int i = 0; i < kVec; ++i) dot = fmaf(g[i], t[i], dot);
+    }
+    if (do_sgd) {
+      load_seg<kVec>(W + i0, n, t);
+#pragma unroll
+      for (int i = 0; i < kVec; ++i) t[i] = fmaf(-lr, g[i], t[i]);
+      store_seg<kVec>(W + i0, n, t);
+    }
+  }
+  if (delta != nullptr) {
+    dot = block_sum(dot);
+    if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
+  }
+}
+
+// ---- bias gradient, stage 1: column sums of one chunk of rows ------------------------------
+// grid (ceil(width / 256), ceil(M / kColsumRows)); block (32, 8): x -> 8 columns, y -> row phase.
+template <typename T>
+__global__ void __launch_bounds__(256)
+colsum_partial_kernel(const T* __restrict__ dZ, int M, int width, float* __restrict__ part) {
+  __shared__ float sm[8][256 + 8];
+  const int col0 = blockIdx.x * 256 + threadIdx.x * kVec;
+  const int r0 = blockIdx.y * kColsumRows;
+  const int r1 = min(M, r0 + kColsumRows);
+  float acc[kVec];
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) acc[i] = 0.0f;
+  const int n = width - col0;
+  if (n > 0) {
+    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
+      float v[kVec];
+      load_seg<kVec>(dZ + (size_t)r * width + col0, n, v);
+#pragma unroll
+      for (int i = 0; i < kVec; ++i) acc[i] += v[i];
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) sm[threadIdx.y][threadIdx.x * kVec + i] = acc[i];
+  __syncthreads();
+  const int tid = threadIdx.y * 32 + threadIdx.x;      // 256 threads, one column each
+  const int col = blockIdx.x * 256 + tid;
+  if (col < width) {
+    float s = 0.0f;
+#pragma unroll
+    for (int y = 0; y < 8; ++y) s += sm[y][tid];
+    part[(size_t)blockIdx.y * width + col] = s;
+  }
+}
+
+// ---- bias gradient, stage 2: sum the chunks, then grad / importance / SGD -----------------
+// One thread per bias element j in [0, fold*width); column = j mod width (a folded layer's
+// dZ is the same gradient repeated for each slice).
+template <typename T>
+__global__ void __launch_bounds__(kEltThreads)
+bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
+                   float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
+                   T* __restrict__ b, float lr, int do_sgd) {
+  const int j = blockIdx.x * kEltThreads + threadIdx.x;
+  float dot = 0.0f;
+  if (j < count) {
+    const int col = j % width;
+    float g = 0.0f;
+    for (int c = 0; c < chunks; ++c) g += part[(size_t)c * width + col];
+    if (grad != nullptr) grad[j] = g;
+    if (delta != nullptr) dot = g * to_f32(delta[j]);
+    if (do_sgd) b[j] = from_f32<T>(fmaf(-lr, g, to_f32(b[j])));
+  }
+  if (delta != nullptr) {
+    dot = block_sum(dot);
+    if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
+  }
+}
+
+// ---- importance, last stage: per tensor, sum its block partials in a fixed order ----------
+struct MaskBits { uint32_t w[64]; };            // up to 2048 tensors
+__global__ void __launch_bounds__(128)
+importance_finalize_kernel(const float* __restrict__ parts, const int* __restrict__ offs,
+                           const int* __restrict__ counts, const MaskBits active, float* __restrict__ out) {
+  const int t = blockIdx.x;
+  float s = 0.0f;
+  if ((active.w[t >> 5] >> (t & 31)) & 1u) {
+    const int o = offs[t], c = counts[t];
+    for (int i = threadIdx.x; i < c; i += blockDim.x) s += parts[o + i];
+  }
+  s = block_sum(s);
+  if (threadIdx.x == 0) out[t] = s;
+}
+
+// ---- stand-alone Eq. 2 on a materialised gradient (V elements per thread) ------------------
+template <typename T, int V>
+__global__ void __launch_bounds__(kEltThreads)
+importance_kernel(const float* __restrict__ grad, const T* __restrict__ delta, size_t count,
+                  float* __restrict__ imp_part) {
+  const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * V;
+  float dot = 0.0f;
+  if (i0 < count) {
+    const int n = (int)min((size_t)V, count - i0);
+    float g[V], t[V];
+    load_seg<V>(grad + i0, n, g);
+    load_seg<V>(delta + i0, n, t);
+#pragma unroll
+    for (int i = 0; i < V; ++i) dot = fmaf(g[i], t[i], dot);
+  }
+  dot = block_sum(dot);
+  if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
+}
+
+// ---- stand-alone masked SGD on one selected tensor -----------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kEltThreads)
+sgd_kernel(T* __restrict__ w, const float* __restrict__ grad, size_t count, float lr) {
+  const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
+  if (i0 >= count) return;
+  const int n = (int)min((size_t)kVec, count - i0);
+  float g[kVec], t[kVec];
+  load_seg<kVec>(grad + i0, n, g);
+  load_seg<kVec>(w + i0, n, t);
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) t[i] = fmaf(-lr, g[i], t[i]);
+  store_seg<kVec>(w + i0, n, t);
+}
+
+// ---- dZ = dY * act'(Z) for a top layer that has an activation -------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kEltThreads)
+act_backward_kernel(const T* __restrict__ dY, const T* __restrict__ Z, T* __restrict__ dZ, size_t count, int act) {
+  const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
+  if (i0 >= count) return;
+  const int n = (int)min((size_t)kVec, count - i0);
+  float g[kVec], z[kVec];
+  load_seg<kVec>(dY + i0, n, g);
+  load_seg<kVec>(Z + i0, n, z);
+#pragma unroll
+  for (int i = 0; i < kVec; ++i) g[i] *= act_grad(z[i], act);
+  store_seg<kVec>(dZ + i0, n, g);
+}
+
+// ---- MSE: dY = 2 (y - t) / count, block partials of (y - t)^2 ---------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kEltThreads)
+mse_grad_kernel(const T* __restrict__ y, const T* __restrict__ target, T* __restrict__ dY, size_t count,
+                float scale, float* __restrict__ loss_part) {
+  const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
+  float sq = 0.0f;
+  if (i0 < count) {
+    const int n = (int)min((size_t)kVec, count - i0);
+    float a[kVec], t[kVec];
+    load_seg<kVec>(y + i0, n, a);
+    load_seg<kVec>(target + i0, n, t);
+#pragma unroll
+    for (int i = 0; i < kVec; ++i) {
+      const float d = a[i] - t[i];
+      sq = fmaf(d, d, sq);
+      a[i] = d * scale;
+    }
+    store_seg<kVec>(dY + i0, n, a);
+  }
+  sq = block_sum(sq);
+  if (threadIdx.x == 0) loss_part[blockIdx.x] = sq;
+}
+__global__ void __launch_bounds__(256)
+loss_finalize_kernel(const float* __restrict__ parts, int n, float inv_count, float* __restrict__ loss) {
+  float s = 0.0f;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) s += parts[i];
+  s = block_sum(s);
+  if (threadIdx.x == 0) *loss = s * inv_count;
+}
+
+}  // namespace et
