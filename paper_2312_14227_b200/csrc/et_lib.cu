@@ -1,0 +1,739 @@
+// Host side of the C ABI declared in et.h: stack object, workspace layout, execution plan
+// from the selection mask, kernel launches.  No device memory is allocated here.
+#include <algorithm>
+#include <atomic>
+#include <cstring>
+#include <new>
+#include <type_traits>
+#include <vector>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "et.h"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+
+namespace {
+
+thread_local int g_last_cuda = 0;
+std::atomic<long long> g_launches{0};
+
+#define CU_TRY(expr)                                   \
+  do {                                                 \
+    cudaError_t e__ = (expr);                          \
+    if (e__ != cudaSuccess) {                          \
+      g_last_cuda = (int)e__;                          \
+      return ET_ERR_CUDA;                              \
+    }                                                  \
+  } while (0)
+#define ET_TRY(expr)                                   \
+  do {                                                 \
+    et_status s__ = (expr);                            \
+    if (s__ != ET_OK) return s__;                      \
+  } while (0)
+
+inline et_status after_launch() {
+  CU_TRY(cudaGetLastError());
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return ET_OK;
+}
+inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
+inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// ---- TMA descriptors ---------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+// Row-major bf16 matrix [outer x inner], box 64 x 64, 128-byte swizzle, zero fill outside.
+et_status make_map(CUtensorMap* m, const void* ptr, int inner, long long outer) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return ET_ERR_CUDA;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)inner * 2};
+  cuuint32_t box[2] = {64, 64};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda = (int)cudaErrorInvalidValue;
+    return ET_ERR_CUDA;
+  }
+  return ET_OK;
+}
+
+struct LayerRT {
+  int K = 0, N = 0, Nw = 0, fold = 1, act = 0, residual_src = -1;
+  int consumer = -1;        // layer whose residual reads a_l (its output gradient joins G_l), or -1
+  void* W = nullptr;
+  void* b = nullptr;
+  size_t off_a_out = 0;     // a_{l+1}           (unused for the last layer: that is the caller's y)
+  size_t off_Z = 0;         // Z_l               (act != none)
+  size_t off_G_out = 0;     // G_{l+1}           (unused for the last layer: that is the caller's dY)
+  size_t off_dZ = 0;        // dZ_l              (act != none)
+  int split = 1;            // wgrad contraction splits
+  int imp_count_w = 0, imp_count_b = 0;
+  CUtensorMap map_a, map_W, map_dz;   // bf16 stacks; map_a of layer 0 and map_dz of an
+                                      // activation-free last layer are built per call
+};
+
+}  // namespace
+
+struct et_stack {
+  int L = 0;
+  long long M = 0;
+  et_dtype dtype = ET_F32;
+  size_t elt = 4;
+  int sms = 148;
+  std::vector<LayerRT> ly;
+  std::vector<int> imp_offs, imp_counts;
+  size_t ws_bytes = 0;
+  size_t off_status = 0, off_partial = 0, off_biaspart = 0, off_imp_parts = 0, off_imp_offs = 0,
+         off_imp_counts = 0, off_loss_parts = 0, off_dy_stage = 0, off_imp_stage = 0;
+  int imp_total = 0;
+  char* ws = nullptr;
+  bool bound = false, forwarded = false;
+  const void* x = nullptr;
+  CUtensorMap map_x, map_dy;
+  const void* map_dy_ptr = nullptr;
+
+  char* at(size_t off) const { return ws + off; }
+  int width_in(int l) const { return ly[l].K; }
+  int out_width() const { return ly[L - 1].Nw; }
+};
+
+namespace {
+
+using et::bf16;
+
+int choose_split(int tiles, int kb_total, int sms) {
+  int best = 1;
+  long long best_cost = -1;
+  for (int s = 1; s <= 16 && s <= kb_total; ++s) {
+    const int kbs = ceil_div(kb_total, s);
+    if ((long long)(s - 1) * kbs >= kb_total) continue;        // an empty split
+    const long long waves = ceil_div((long long)tiles * s, sms);
+    const long long cost = waves * (kbs + 6);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+  }
+  return best;
+}
+
+template <typename T> struct is_bf16 : std::false_type {};
+template <> struct is_bf16<bf16> : std::true_type {};
+
+// ---- pointer helpers -----------------------------------------------------------------------
+template <typename T> const T* act_in(const et_stack* s, int l) {       // a_l
+  return l == 0 ? (const T*)s->x : (const T*)s->at(s->ly[l - 1].off_a_out);
+}
+template <typename T> T* grad_act(const et_stack* s, int i, const void* dY) {   // G_i = dL/da_i, i >= 1
+  return i == s->L ? (T*)const_cast<void*>(dY) : (T*)s->at(s->ly[i - 1].off_G_out);
+}
+template <typename T> const T* dz_src(const et_stack* s, int l, const void* dY) {   // dZ_l (width Nw)
+  const LayerRT& y = s->ly[l];
+  return y.act != ET_ACT_NONE ? (const T*)s->at(y.off_dZ) : grad_act<T>(s, l + 1, dY);
+}
+const CUtensorMap& dz_map(const et_stack* s, int l) {
+  return (l == s->L - 1 && s->ly[l].act == ET_ACT_NONE) ? s->map_dy : s->ly[l].map_dz;
+}
+const CUtensorMap& a_map(const et_stack* s, int l) { return l == 0 ? s->map_x : s->ly[l].map_a; }
+
+// ---- GEMM launches ---------------------------------------------------------------------------
+template <bool A_MN, bool B_MN, class Epi>
+et_status launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::Params& p, const Epi& epi, int sms,
+                    cudaStream_t st) {
+  auto kern = et::tc::gemm_tc_kernel<A_MN, B_MN, Epi>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)et::tc::SMEM_BYTES));
+    attr_done = true;
+  }
+  const int units = p.tiles_m * p.tiles_n * p.split;
+  const int grid = std::min(units, sms);
+  kern<<<grid, et::tc::THREADS, et::tc::SMEM_BYTES, st>>>(ma, mb, p, epi);
+  return after_launch();
+}
+template <typename T, class Epi>
+et_status launch_simt(const T* A, const T* B, const et::simt::Params& p, const Epi& epi, cudaStream_t st) {
+  dim3 grid(ceil_div(p.cols, et::simt::TN), ceil_div(p.rows, et::simt::TM));
+  et::simt::gemm_simt_kernel<T, Epi><<<grid, et::simt::THREADS, 0, st>>>(A, B, p, epi);
+  return after_launch();
+}
+
+et::tc::Params tc_params(const et_stack* s, int rows, int cols, int contraction, int fold, int split) {
+  et::tc::Params p;
+  p.rows = rows; p.cols = cols;
+  p.tiles_m = ceil_div(rows, et::tc::BM);
+  p.tiles_n = ceil_div(cols, et::tc::BN);
+  p.split = split;
+  p.kb_per_seg = ceil_div(contraction, et::tc::BK);
+  p.kb_total = p.kb_per_seg * fold;
+  p.kb_per_split = ceil_div(p.kb_total, split);
+  p.b_k_seg_stride = 0; p.b_mn_seg_stride = 0; p.b_mn_wrap = 0;
+  p.status = (uint32_t*)s->at(s->off_status);
+  return p;
+}
+
+// Z_l = a_l W_l + b_l, activation, fold, residual -> a_{l+1}
+template <typename T>
+et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
+  const LayerRT& L = s->ly[l];
+  et::FwdEpi<T> epi;
+  epi.bias = (const T*)L.b;
+  epi.fold = L.fold;
+  epi.Z = L.act != ET_ACT_NONE ? (T*)s->at(L.off_Z) : nullptr;
+  epi.act = L.act;
+  epi.resid = L.residual_src >= 0 ? act_in<T>(s, L.residual_src) : nullptr;
+  epi.out = l == s->L - 1 ? (T*)y : (T*)s->at(L.off_a_out);
+  epi.ld = L.Nw;
+  if constexpr (is_bf16<T>::value) {
+    et::tc::Params p = tc_params(s, (int)s->M, L.Nw, L.K, L.fold, 1);
+    p.b_mn_seg_stride = L.Nw;
+    return launch_tc<false, true>(a_map(s, l), L.map_W, p, epi, s->sms, st);
+  } else {
+    et::simt::Params p;
+    p.rows = (int)s->M; p.cols = L.Nw; p.kc = L.K; p.segs = L.fold;
+    p.sa_i = L.K; p.sa_k = 1;
+    p.sb_k = L.N; p.sb_seg = L.Nw; p.sb_j = 1; p.b_wrap = 0;
+    return launch_simt<T>(act_in<T>(s, l), (const T*)L.W, p, epi, st);
+  }
+}
+
+// G_l = dZ_l W_l^T (+ skip gradient), dZ_{l-1} = G_l * act'(Z_{l-1});  l >= 1
+template <typename T>
+et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st) {
+  const LayerRT& L = s->ly[l];
+  const LayerRT& P = s->ly[l - 1];
+  et::DgradEpi<T> epi;
+  epi.skip = L.consumer >= 0 ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
+  epi.act_prev = P.act;
+  epi.ld = L.K;
+  if (P.act == ET_ACT_NONE) {
+    epi.Zprev = nullptr;
+    epi.outG = (T*)s->at(P.off_G_out);
+    epi.outdZ = nullptr;
+  } else {
+    epi.Zprev = (const T*)s->at(P.off_Z);
+    epi.outdZ = (T*)s->at(P.off_dZ);
+    epi.outG = P.residual_src >= 0 ? (T*)s->at(P.off_G_out) : nullptr;
+  }
+  if constexpr (is_bf16<T>::value) {
+    et::tc::Params p = tc_params(s, (int)s->M, L.K, L.Nw, L.fold, 1);
+    p.b_k_seg_stride = L.Nw;
+    return launch_tc<false, false>(dz_map(s, l), L.map_W, p, epi, s->sms, st);
+  } else {
+    et::simt::Params p;
+    p.rows = (int)s->M; p.cols = L.K; p.kc = L.Nw; p.segs = L.fold;
+    p.sa_i = L.Nw; p.sa_k = 1;
+    p.sb_k = 1; p.sb_seg = L.Nw; p.sb_j = L.N; p.b_wrap = 0;
+    return launch_simt<T>(dz_src<T>(s, l, dY), (const T*)L.W, p, epi, st);
+  }
+}
+
+// dW_l = a_l^T dZ_l as split partials, then the reducer with grad / importance / SGD.
+template <typename T>
+et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
+                          int* launches, cudaStream_t st) {
+  const LayerRT& L = s->ly[l];
+  float* partial = (float*)s->at(s->off_partial);
+  const size_t count = (size_t)L.K * L.N;
+  et::PartialEpi epi;
+  epi.base = partial; epi.split_stride = count; epi.ld = L.N; epi.split = 0;
+  int split = 1;
+  if constexpr (is_bf16<T>::value) {
+    split = L.split;
+    et::tc::Params p = tc_params(s, L.K, L.N, (int)s->M, 1, split);
+    p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
+    ET_TRY((launch_tc<true, true>(a_map(s, l), dz_map(s, l), p, epi, s->sms, st)));
+  } else {
+    et::simt::Params p;
+    p.rows = L.K; p.cols = L.N; p.kc = (int)s->M; p.segs = 1;
+    p.sa_i = 1; p.sa_k = L.K;
+    p.sb_k = L.Nw; p.sb_seg = 0; p.sb_j = 1; p.b_wrap = L.fold > 1 ? L.Nw : 0;
+    ET_TRY(launch_simt<T>(act_in<T>(s, l), dz_src<T>(s, l, dY), p, epi, st));
+  }
+  ++*launches;
+  if (grad == nullptr && delta == nullptr && !sgd) return ET_OK;     // nothing consumes g
+  float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
+  et::wgrad_reduce_kernel<T><<<L.imp_count_w, et::kEltThreads, 0, st>>>(partial, split, count, count, grad, delta, imp,
+                                                                        (T*)L.W, lr, sgd ? 1 : 0);
+  ++*launches;
+  return after_launch();
+}
+
+template <typename T>
+et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
+                          int* launches, cudaStream_t st) {
+  const LayerRT& L = s->ly[l];
+  float* part = (float*)s->at(s->off_biaspart);
+  const int chunks = ceil_div(s->M, et::kColsumRows);
+  dim3 grid(ceil_div(L.Nw, 256), chunks), block(32, 8);
+  et::colsum_partial_kernel<T><<<grid, block, 0, st>>>(dz_src<T>(s, l, dY), (int)s->M, L.Nw, part);
+  ET_TRY(after_launch());
+  ++*launches;
+  float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l + 1];
+  et::bias_finish_kernel<T><<<L.imp_count_b, et::kEltThreads, 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
+                                                                       (T*)L.b, lr, sgd ? 1 : 0);
+  ++*launches;
+  return after_launch();
+}
+
+et::MaskBits mask_bits(const uint8_t* mask, int n) {
+  et::MaskBits b;
+  std::memset(&b, 0, sizeof(b));
+  for (int t = 0; t < n; ++t)
+    if (mask[t]) b.w[t >> 5] |= 1u << (t & 31);
+  return b;
+}
+
+et_status check_ready(const et_stack* s, const uint8_t* mask, int n_tensors) {
+  if (s == nullptr || mask == nullptr) return ET_ERR_INVALID_ARG;
+  if (n_tensors != 2 * s->L) return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  return ET_OK;
+}
+
+template <typename T>
+et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float* const* grads,
+                        const void* const* delta, float* importance_dev, uint32_t flags, float lr,
+                        et_exec_report* report, cudaStream_t st) {
+  const int L = s->L;
+  int d = L;
+  for (int l = 0; l < L; ++l)
+    if (mask[2 * l] || mask[2 * l + 1]) { d = l; break; }
+  const bool sgd = (flags & ET_FLAG_FUSE_SGD) != 0;
+  int launches = 0;
+  double flops = 0.0;
+
+  if (report != nullptr) {
+    for (int l = 0; l < L; ++l) {
+      if (report->dgrad) report->dgrad[l] = l > d;
+      if (report->wgrad) report->wgrad[l] = mask[2 * l] != 0;
+      if (report->bgrad) report->bgrad[l] = mask[2 * l + 1] != 0;
+      if (report->updated) {
+        report->updated[2 * l] = sgd && mask[2 * l];
+        report->updated[2 * l + 1] = sgd && mask[2 * l + 1];
+      }
+    }
+    report->deepest = d;
+  }
+
+  if (d == L) {
+    if (delta != nullptr) CU_TRY(cudaMemsetAsync(importance_dev, 0, sizeof(float) * 2 * L, st));
+  } else {
+    if constexpr (is_bf16<T>::value) {
+      if (s->ly[L - 1].act == ET_ACT_NONE && s->map_dy_ptr != dY) {
+        ET_TRY(make_map(&s->map_dy, dY, s->out_width(), s->M));
+        s->map_dy_ptr = dY;
+      }
+    }
+    const LayerRT& top = s->ly[L - 1];
+    if (top.act != ET_ACT_NONE) {
+      const size_t count = (size_t)s->M * top.N;
+      et::act_backward_kernel<T><<<ceil_div(count, et::kEltThreads * et::kVec), et::kEltThreads, 0, st>>>(
+          (const T*)dY, (const T*)s->at(top.off_Z), (T*)s->at(top.off_dZ), count, top.act);
+      ET_TRY(after_launch());
+      ++launches;
+    }
+    for (int l = L - 1; l >= d; --l) {
+      const LayerRT& Y = s->ly[l];
+      const double gemm = 2.0 * (double)s->M * Y.K * Y.N;
+      if (l > d) {                        // reads the old W_l: must precede this layer's update
+        ET_TRY(run_dgrad_layer<T>(s, l, dY, st));
+        ++launches;
+        flops += gemm;
+      }
+      if (mask[2 * l]) {
+        ET_TRY(run_wgrad_layer<T>(s, l, dY, grads ? grads[2 * l] : nullptr,
+                                  delta ? (const T*)delta[2 * l] : nullptr, sgd, lr, &launches, st));
+        flops += gemm;
+      }
+      if (mask[2 * l + 1]) {
+        ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
+                                  delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, st));
+      }
+    }
+    if (delta != nullptr) {
+      et::importance_finalize_kernel<<<2 * L, 128, 0, st>>>((const float*)s->at(s->off_imp_parts),
+                                                            (const int*)s->at(s->off_imp_offs),
+                                                            (const int*)s->at(s->off_imp_counts), mask_bits(mask, 2 * L),
+                                                            importance_dev);
+      ET_TRY(after_launch());
+      ++launches;
+    }
+  }
+  if (report != nullptr) {
+    report->launches = launches;
+    report->flops_executed = flops;
+  }
+  return ET_OK;
+}
+
+et_status validate_backward_args(const et_stack* s, const void* dY, const uint8_t* mask, int32_t n_tensors,
+                                 const void* const* delta, const void* importance) {
+  ET_TRY(check_ready(s, mask, n_tensors));
+  if (dY == nullptr) return ET_ERR_INVALID_ARG;
+  if (!s->forwarded) return ET_ERR_STATE;
+  if (delta != nullptr) {
+    if (importance == nullptr) return ET_ERR_INVALID_ARG;
+    for (int t = 0; t < n_tensors; ++t)
+      if (mask[t] && delta[t] == nullptr) return ET_ERR_INVALID_ARG;
+  }
+  return ET_OK;
+}
+
+template <typename T>
+et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
+  if constexpr (is_bf16<T>::value) {
+    if (s->x != x || !s->forwarded) ET_TRY(make_map(&s->map_x, x, s->ly[0].K, s->M));
+  }
+  s->x = x;
+  for (int l = 0; l < s->L; ++l) ET_TRY(run_forward_layer<T>(s, l, y, st));
+  s->forwarded = true;
+  return ET_OK;
+}
+
+double median(std::vector<float>& v) {
+  std::sort(v.begin(), v.end());
+  return v.empty() ? 0.0 : (double)v[v.size() / 2];
+}
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_dtype dtype, et_stack** out) {
+  if (layers == nullptr || out == nullptr || L < 1 || L > 1024 || M < 1 || M > (1ll << 30)) return ET_ERR_INVALID_ARG;
+  if (dtype != ET_F32 && dtype != ET_BF16) return ET_ERR_DTYPE;
+  et_stack* s = new (std::nothrow) et_stack();
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  s->L = L; s->M = M; s->dtype = dtype; s->elt = dtype == ET_BF16 ? 2 : 4;
+  s->ly.resize(L);
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      s->sms = sms;
+    else
+      (void)cudaGetLastError();
+  }
+  et_status err = ET_OK;
+  std::vector<int> width(L + 1);
+  width[0] = layers[0].in_features;
+  for (int l = 0; l < L && err == ET_OK; ++l) {
+    const et_layer_desc& d = layers[l];
+    LayerRT& y = s->ly[l];
+    if (d.in_features < 1 || d.out_features < 1 || d.fold < 1 || d.act < 0 || d.act > 2) { err = ET_ERR_INVALID_ARG; break; }
+    if (d.out_features % d.fold != 0) { err = ET_ERR_SHAPE; break; }
+    if (d.fold > 1 && d.act != ET_ACT_NONE) { err = ET_ERR_UNSUPPORTED; break; }
+    y.K = d.in_features; y.N = d.out_features; y.fold = d.fold; y.Nw = d.out_features / d.fold;
+    y.act = d.act; y.residual_src = d.residual_src;
+    if (y.K != width[l]) { err = ET_ERR_SHAPE; break; }
+    width[l + 1] = y.Nw;
+    if (d.residual_src < -1 || d.residual_src > l) { err = ET_ERR_INVALID_ARG; break; }
+    if (d.residual_src >= 0) {
+      if (width[d.residual_src] != y.Nw) { err = ET_ERR_SHAPE; break; }
+      if (d.residual_src >= 1) {          // a_0's gradient is never formed, no bookkeeping needed
+        LayerRT& src = s->ly[d.residual_src];
+        if (src.consumer >= 0) { err = ET_ERR_UNSUPPORTED; break; }   // one skip consumer per activation
+        src.consumer = l;
+      }
+    }
+    if (dtype == ET_BF16) {
+      if (y.K % 8 || y.N % 8 || y.Nw % 8) { err = ET_ERR_UNSUPPORTED; break; }
+      if (y.fold > 1 && y.Nw % et::tc::BN) { err = ET_ERR_UNSUPPORTED; break; }
+    }
+  }
+  if (err != ET_OK) { delete s; return err; }
+
+  // ---- workspace layout
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
+  s->off_status = take(256);
+  size_t max_partial = 0, max_biaspart = 0;
+  const int chunks = ceil_div(M, et::kColsumRows);
+  s->imp_offs.resize(2 * L); s->imp_counts.resize(2 * L);
+  int imp_total = 0;
+  for (int l = 0; l < L; ++l) {
+    LayerRT& y = s->ly[l];
+    const size_t act_bytes = (size_t)M * y.Nw * s->elt;
+    if (l < L - 1) { y.off_a_out = take(act_bytes); y.off_G_out = take(act_bytes); }
+    if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
+    if (dtype == ET_BF16) {
+      const int tiles = ceil_div(y.K, et::tc::BM) * ceil_div(y.N, et::tc::BN);
+      y.split = choose_split(tiles, ceil_div(M, et::tc::BK), s->sms);
+    }
+    max_partial = std::max(max_partial, (size_t)y.split * y.K * y.N * sizeof(float));
+    max_biaspart = std::max(max_biaspart, (size_t)chunks * y.Nw * sizeof(float));
+    y.imp_count_w = ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
+    y.imp_count_b = ceil_div(y.N, et::kEltThreads);
+    s->imp_offs[2 * l] = imp_total; s->imp_counts[2 * l] = y.imp_count_w; imp_total += y.imp_count_w;
+    s->imp_offs[2 * l + 1] = imp_total; s->imp_counts[2 * l + 1] = y.imp_count_b; imp_total += y.imp_count_b;
+  }
+  s->imp_total = imp_total;
+  s->off_partial = take(max_partial);
+  s->off_biaspart = take(max_biaspart);
+  s->off_imp_parts = take((size_t)imp_total * sizeof(float));
+  s->off_imp_offs = take((size_t)2 * L * sizeof(int));
+  s->off_imp_counts = take((size_t)2 * L * sizeof(int));
+  const size_t out_count = (size_t)M * s->out_width();
+  s->off_loss_parts = take((size_t)ceil_div(out_count, et::kEltThreads * et::kVec) * sizeof(float));
+  s->off_dy_stage = take(out_count * s->elt);
+  s->off_imp_stage = take((size_t)2 * L * sizeof(float));
+  s->ws_bytes = off;
+  *out = s;
+  return ET_OK;
+}
+
+et_status et_stack_destroy(et_stack* s) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  delete s;
+  return ET_OK;
+}
+
+et_status et_stack_workspace_bytes(const et_stack* s, size_t* bytes) {
+  if (s == nullptr || bytes == nullptr) return ET_ERR_INVALID_ARG;
+  *bytes = s->ws_bytes;
+  return ET_OK;
+}
+
+et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+  if (s == nullptr || W == nullptr || b == nullptr || workspace == nullptr) return ET_ERR_INVALID_ARG;
+  if (workspace_bytes < s->ws_bytes || ((uintptr_t)workspace & 255) != 0) return ET_ERR_WORKSPACE;
+  for (int l = 0; l < s->L; ++l)
+    if (W[l] == nullptr || b[l] == nullptr || ((uintptr_t)W[l] & 15) || ((uintptr_t)b[l] & 15)) return ET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  s->bound = false;
+  s->ws = (char*)workspace;
+  for (int l = 0; l < s->L; ++l) { s->ly[l].W = W[l]; s->ly[l].b = b[l]; }
+  if (s->dtype == ET_BF16) {
+    for (int l = 0; l < s->L; ++l) {
+      LayerRT& y = s->ly[l];
+      ET_TRY(make_map(&y.map_W, y.W, y.N, y.K));
+      if (l >= 1) ET_TRY(make_map(&y.map_a, s->at(s->ly[l - 1].off_a_out), y.K, s->M));
+      if (y.act != ET_ACT_NONE) ET_TRY(make_map(&y.map_dz, s->at(y.off_dZ), y.Nw, s->M));
+      else if (l < s->L - 1) ET_TRY(make_map(&y.map_dz, s->at(y.off_G_out), y.Nw, s->M));
+    }
+  }
+  CU_TRY(cudaMemsetAsync(s->at(s->off_status), 0, 256, st));
+  CU_TRY(cudaMemcpyAsync(s->at(s->off_imp_offs), s->imp_offs.data(), sizeof(int) * 2 * s->L, cudaMemcpyHostToDevice, st));
+  CU_TRY(cudaMemcpyAsync(s->at(s->off_imp_counts), s->imp_counts.data(), sizeof(int) * 2 * s->L, cudaMemcpyHostToDevice, st));
+  CU_TRY(cudaStreamSynchronize(st));     // the host vectors may be freed / changed afterwards
+  s->bound = true;
+  s->forwarded = false;
+  s->map_dy_ptr = nullptr;
+  s->x = nullptr;
+  return ET_OK;
+}
+
+et_status et_forward_stack(et_stack* s, const void* x, void* y, void* stream) {
+  if (s == nullptr || x == nullptr || y == nullptr) return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  if (((uintptr_t)x & 15) || ((uintptr_t)y & 15)) return ET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  return s->dtype == ET_BF16 ? forward_impl<bf16>(s, x, y, st) : forward_impl<float>(s, x, y, st);
+}
+
+et_status et_loss_mse_grad(et_stack* s, const void* y, const void* target, void* dY, float* loss_dev, void* stream) {
+  if (s == nullptr || y == nullptr || target == nullptr || dY == nullptr) return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t count = (size_t)s->M * s->out_width();
+  const int blocks = ceil_div(count, et::kEltThreads * et::kVec);
+  float* parts = (float*)s->at(s->off_loss_parts);
+  const float scale = (float)(2.0 / (double)count);
+  if (s->dtype == ET_BF16)
+    et::mse_grad_kernel<bf16><<<blocks, et::kEltThreads, 0, st>>>((const bf16*)y, (const bf16*)target, (bf16*)dY, count, scale, parts);
+  else
+    et::mse_grad_kernel<float><<<blocks, et::kEltThreads, 0, st>>>((const float*)y, (const float*)target, (float*)dY, count, scale, parts);
+  ET_TRY(after_launch());
+  if (loss_dev != nullptr) {
+    et::loss_finalize_kernel<<<1, 256, 0, st>>>(parts, blocks, (float)(1.0 / (double)count), loss_dev);
+    ET_TRY(after_launch());
+  }
+  return ET_OK;
+}
+
+et_status et_backward_elastic(et_stack* s, const void* dY, const uint8_t* mask, int32_t n_tensors,
+                              float* const* grads, const void* const* delta, float* importance_dev,
+                              uint32_t flags, float lr, et_exec_report* report, void* stream) {
+  ET_TRY(validate_backward_args(s, dY, mask, n_tensors, delta, importance_dev));
+  if ((uintptr_t)dY & 15) return ET_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)ET_FLAG_FUSE_SGD) return ET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  return s->dtype == ET_BF16
+             ? backward_impl<bf16>(s, dY, mask, grads, delta, importance_dev, flags, lr, report, st)
+             : backward_impl<float>(s, dY, mask, grads, delta, importance_dev, flags, lr, report, st);
+}
+
+et_status et_backward_elastic_host(et_stack* s, const void* dY_host, const uint8_t* mask, int32_t n_tensors,
+                                   float* const* grads, const void* const* delta, float* importance_host,
+                                   uint32_t flags, float lr, et_exec_report* report, void* stream) {
+  ET_TRY(validate_backward_args(s, dY_host, mask, n_tensors, delta, importance_host));
+  if (flags & ~(uint32_t)ET_FLAG_FUSE_SGD) return ET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  void* dY = s->at(s->off_dy_stage);
+  float* imp = (float*)s->at(s->off_imp_stage);
+  CU_TRY(cudaMemcpyAsync(dY, dY_host, (size_t)s->M * s->out_width() * s->elt, cudaMemcpyHostToDevice, st));
+  et_status r = s->dtype == ET_BF16
+                    ? backward_impl<bf16>(s, dY, mask, grads, delta, imp, flags, lr, report, st)
+                    : backward_impl<float>(s, dY, mask, grads, delta, imp, flags, lr, report, st);
+  if (r != ET_OK) return r;
+  if (delta != nullptr)
+    CU_TRY(cudaMemcpyAsync(importance_host, imp, sizeof(float) * 2 * s->L, cudaMemcpyDeviceToHost, st));
+  CU_TRY(cudaStreamSynchronize(st));
+  return ET_OK;
+}
+
+et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads,
+                        const void* const* delta, float* importance_dev, void* stream) {
+  ET_TRY(check_ready(s, mask, n_tensors));
+  if (grads == nullptr || delta == nullptr || importance_dev == nullptr) return ET_ERR_INVALID_ARG;
+  for (int t = 0; t < n_tensors; ++t)
+    if (mask[t] && (grads[t] == nullptr || delta[t] == nullptr)) return ET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* parts = (float*)s->at(s->off_imp_parts);
+  for (int t = 0; t < n_tensors; ++t) {
+    if (!mask[t]) continue;
+    const LayerRT& y = s->ly[t / 2];
+    const bool is_w = (t & 1) == 0;
+    const size_t count = is_w ? (size_t)y.K * y.N : (size_t)y.N;
+    const int blocks = s->imp_counts[t];
+    float* out = parts + s->imp_offs[t];
+    if (s->dtype == ET_BF16) {
+      if (is_w) et::importance_kernel<bf16, 8><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const bf16*)delta[t], count, out);
+      else      et::importance_kernel<bf16, 1><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const bf16*)delta[t], count, out);
+    } else {
+      if (is_w) et::importance_kernel<float, 8><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const float*)delta[t], count, out);
+      else      et::importance_kernel<float, 1><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const float*)delta[t], count, out);
+    }
+    ET_TRY(after_launch());
+  }
+  et::importance_finalize_kernel<<<n_tensors, 128, 0, st>>>(parts, (const int*)s->at(s->off_imp_offs),
+                                                            (const int*)s->at(s->off_imp_counts),
+                                                            mask_bits(mask, n_tensors), importance_dev);
+  return after_launch();
+}
+
+et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads, float lr,
+                        void* stream) {
+  ET_TRY(check_ready(s, mask, n_tensors));
+  if (grads == nullptr) return ET_ERR_INVALID_ARG;
+  for (int t = 0; t < n_tensors; ++t)
+    if (mask[t] && grads[t] == nullptr) return ET_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int t = 0; t < n_tensors; ++t) {
+    if (!mask[t]) continue;
+    const LayerRT& y = s->ly[t / 2];
+    const bool is_w = (t & 1) == 0;
+    const size_t count = is_w ? (size_t)y.K * y.N : (size_t)y.N;
+    void* w = is_w ? y.W : y.b;
+    const int blocks = ceil_div(count, et::kEltThreads * et::kVec);
+    if (s->dtype == ET_BF16) et::sgd_kernel<bf16><<<blocks, et::kEltThreads, 0, st>>>((bf16*)w, grads[t], count, lr);
+    else                     et::sgd_kernel<float><<<blocks, et::kEltThreads, 0, st>>>((float*)w, grads[t], count, lr);
+    ET_TRY(after_launch());
+  }
+  return ET_OK;
+}
+
+et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, int32_t iters, double* t_dw,
+                           double* t_dy, double* t_fwd, void* stream) {
+  if (s == nullptr || x == nullptr || y == nullptr || dY == nullptr || t_dw == nullptr || t_dy == nullptr ||
+      iters < 1 || iters > 10000)
+    return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int L = s->L;
+  cudaEvent_t e0, e1;
+  CU_TRY(cudaEventCreate(&e0));
+  CU_TRY(cudaEventCreate(&e1));
+  et_status rc = ET_OK;
+  std::vector<float> ts;
+  auto timed = [&](auto&& fn, double* out) -> et_status {
+    ts.clear();
+    for (int it = 0; it < iters + 1; ++it) {          // first run is a warm-up
+      CU_TRY(cudaEventRecord(e0, st));
+      ET_TRY(fn());
+      CU_TRY(cudaEventRecord(e1, st));
+      CU_TRY(cudaEventSynchronize(e1));
+      float ms = 0.f;
+      CU_TRY(cudaEventElapsedTime(&ms, e0, e1));
+      if (it > 0) ts.push_back(ms);
+    }
+    *out = median(ts);
+    return ET_OK;
+  };
+  auto body = [&]() -> et_status {
+    double fwd = 0.0;
+    ET_TRY(timed([&]() { return et_forward_stack(s, x, y, stream); }, &fwd));
+    if (t_fwd != nullptr) *t_fwd = fwd;
+    std::vector<uint8_t> ones(2 * L, 1);
+    ET_TRY(et_backward_elastic(s, dY, ones.data(), 2 * L, nullptr, nullptr, nullptr, 0, 0.f, nullptr, stream));
+    float* scratch_grad = (float*)s->at(s->off_partial);      // in-place: each element is read before it is written
+    for (int l = L - 1; l >= 0; --l) {
+      int dummy = 0;
+      t_dy[2 * l] = 0.0; t_dy[2 * l + 1] = 0.0;
+      if (s->dtype == ET_BF16) {
+        if (l >= 1) ET_TRY(timed([&]() { return run_dgrad_layer<bf16>(s, l, dY, st); }, &t_dy[2 * l]));
+        ET_TRY(timed([&]() { return run_wgrad_layer<bf16>(s, l, dY, scratch_grad, nullptr, false, 0.f, &dummy, st); }, &t_dw[2 * l]));
+        ET_TRY(timed([&]() { return run_bgrad_layer<bf16>(s, l, dY, nullptr, nullptr, false, 0.f, &dummy, st); }, &t_dw[2 * l + 1]));
+      } else {
+        if (l >= 1) ET_TRY(timed([&]() { return run_dgrad_layer<float>(s, l, dY, st); }, &t_dy[2 * l]));
+        ET_TRY(timed([&]() { return run_wgrad_layer<float>(s, l, dY, scratch_grad, nullptr, false, 0.f, &dummy, st); }, &t_dw[2 * l]));
+        ET_TRY(timed([&]() { return run_bgrad_layer<float>(s, l, dY, nullptr, nullptr, false, 0.f, &dummy, st); }, &t_dw[2 * l + 1]));
+      }
+    }
+    return ET_OK;
+  };
+  rc = body();
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  return rc;
+}
+
+et_status et_device_status(et_stack* s, void* stream) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint32_t word = 0;
+  CU_TRY(cudaMemcpyAsync(&word, s->at(s->off_status), sizeof(word), cudaMemcpyDeviceToHost, st));
+  CU_TRY(cudaStreamSynchronize(st));
+  return word == 0 ? ET_OK : ET_ERR_TIMEOUT;
+}
+
+const char* et_status_string(et_status st) {
+  switch (st) {
+    case ET_OK: return "ok";
+    case ET_ERR_INVALID_ARG: return "invalid argument";
+    case ET_ERR_SHAPE: return "layer shapes do not chain";
+    case ET_ERR_DTYPE: return "unknown dtype";
+    case ET_ERR_STATE: return "call out of order (bind / forward first)";
+    case ET_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case ET_ERR_UNSUPPORTED: return "shape not supported by the kernels";
+    case ET_ERR_CUDA: return "CUDA call failed";
+    case ET_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int32_t et_last_cuda_error(void) { return g_last_cuda; }
+int64_t et_launch_count(void) { return (int64_t)g_launches.load(); }
+
+}  // extern "C"

@@ -19,8 +19,8 @@ constexpr int kColsumRows = 128;                // rows per column-sum chunk
 //   W           <- W - lr * g                  if do_sgd   (fp32 arithmetic, one rounding)
 template <typename T>
 __global__ void __launch_bounds__(kEltThreads)
-wgrad_reduce_kernel(const float* __restrict__ partial, int splits, size_t split_stride, size_t count,
-                    float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
+wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_t count,
+                    float* grad /* may alias partial: each thread reads its elements before writing them */, const T* __restrict__ delta, float* __restrict__ imp_part,
                     T* __restrict__ W, float lr, int do_sgd) {
   const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
   float dot = 0.0f;
