@@ -8,6 +8,20 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def _ensure_library():
+    """Build libet.so in-tree if it is missing or stale (run as a script: importing the
+    package itself needs the library)."""
+    import subprocess
+    script = os.path.join(ROOT, "paper_2312_14227_b200", "build.py")
+    lib = os.path.join(ROOT, "paper_2312_14227_b200", "libet.so")
+    if os.path.exists(lib):
+        return
+    subprocess.run([sys.executable, script], check=True, capture_output=True)
+
+
+_ensure_library()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 

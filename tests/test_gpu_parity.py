@@ -1,0 +1,170 @@
+"""Parity of the CUDA path against the float64 oracle, through the C ABI.
+Bars: executed-work sets and frozen weights exact; gradients / importances within 1e-4
+(fp32 stacks) or 2e-2 (bf16 stacks) max-norm relative error; updated weights within 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2312_14227_b200 as et
+import workloads as wl
+from oracle import elastic_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+
+
+def _h():
+    import gpu_harness
+    return gpu_harness
+
+
+def test_tiny_mlp_fp32_config():
+    h = _h()
+    w = wl.tiny_mlp()
+    rep = h.check_step(w, w.mask, TOL_F32)
+    assert rep.deepest == 2 and rep.dgrad.tolist() == [0, 0, 0, 1]
+    assert rep.wgrad.tolist() == [0, 0, 1, 0] and rep.bgrad.tolist() == [0, 0, 1, 0]
+
+
+def test_tiny_mlp_fp32_all_selected_is_full_backprop():
+    h = _h()
+    w = wl.tiny_mlp()
+    h.check_step(w, np.ones(2 * w.L, dtype=np.uint8), TOL_F32)
+
+
+def _all_kinds_layers(scale=1):
+    s = scale
+    return [
+        wl.Layer(6 * s, 9 * s, fold=3),
+        wl.Layer(3 * s, 6 * s, residual_src=0),
+        wl.Layer(6 * s, 10 * s, act=wl.ACT_GELU_TANH),
+        wl.Layer(10 * s, 6 * s, residual_src=2),
+        wl.Layer(6 * s, 5 * s, act=wl.ACT_RELU),
+        wl.Layer(5 * s, 6 * s, act=wl.ACT_GELU_TANH, residual_src=4),
+        wl.Layer(6 * s, 4 * s),
+    ]
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_fp32_ragged_all_layer_kinds(seed):
+    h = _h()
+    rng = np.random.default_rng(seed)
+    layers = _all_kinds_layers(scale=[1, 11, 23][seed])          # widths not multiples of any tile
+    M = [7, 131, 77][seed]
+    for trial in range(3):
+        mask = (rng.random(2 * len(layers)) < 0.4).astype(np.uint8)
+        w = wl.small_stack(layers, M, wl.DT_F32, seed * 10 + trial, mask=mask, w_std=0.2, bias_std=0.1)
+        h.check_step(w, mask, TOL_F32)
+
+
+def test_empty_mask_launches_nothing():
+    h = _h()
+    w = wl.tiny_mlp()
+    run = h.GpuRun(w)
+    run.forward_loss()
+    before = [p.clone() for p in run.params()]
+    delta = [h.to_dev(d, w.dtype) for d in wl.draw_delta(w, 1)]
+    n0 = et.et_launch_count()
+    rep = run.backward(np.zeros(2 * w.L, dtype=np.uint8), None, delta, flags=et.ET_FLAG_FUSE_SGD, lr=0.1)
+    assert et.et_launch_count() == n0 and rep.launches == 0 and rep.deepest == w.L
+    assert rep.flops_executed == 0.0 and not rep.dgrad.any()
+    assert torch.all(run.importance == 0)
+    for p, q in zip(run.params(), before):
+        assert torch.equal(p, q)
+
+
+def test_backward_before_forward_is_refused():
+    h = _h()
+    w = wl.tiny_mlp()
+    run = h.GpuRun(w)
+    with pytest.raises(et.EtError) as e:
+        et.et_backward_elastic(run.stack, run.dY, w.mask)
+    assert e.value.status == et.ET_ERR_STATE
+
+
+def test_standalone_importance_and_sgd_match_fused_path():
+    h = _h()
+    w = wl.tiny_mlp()
+    mask = np.ones(2 * w.L, dtype=np.uint8); mask[2] = 0; mask[7] = 0
+    delta_np = wl.draw_delta(w, 3)
+    ref = h.oracle_step(w, mask, delta_np)
+    run = h.GpuRun(w)
+    run.forward_loss()
+    before = [p.clone() for p in run.params()]
+    grads = run.alloc_grads(mask)
+    run.backward(mask, grads, None)                       # gradients only
+    delta = [h.to_dev(d, w.dtype) for d in delta_np]
+    imp = torch.full((2 * w.L,), float("nan"), dtype=torch.float32, device=h.DEV)
+    et.et_importance(run.stack, mask, grads, delta, imp)
+    et.et_sgd_masked(run.stack, mask, grads, w.lr)
+    imp = h.to_np(imp)
+    for t in range(2 * w.L):
+        if mask[t]:
+            assert h.importance_err(imp[t], ref["grads"][t], delta_np[t]) <= TOL_F32
+            assert np.abs(h.to_np(run.params()[t]) - ref["new"][t]).max() <= 1e-3
+        else:
+            assert imp[t] == 0.0 and torch.equal(run.params()[t], before[t])
+
+
+# ------------------------------------------------------------------ bf16 / tensor-core path
+def test_bf16_small_vit_block_ragged_rows():
+    h = _h()
+    # one transformer-shaped block, widths = one to three tiles, rows not a multiple of 128 or 64
+    w = wl.vit_b(seed=11, p_select=0.6, n_blocks=2, tokens=300, d=256, ffn=512, name="vit_small")
+    w.mask[:] = 1
+    h.check_step(w, w.mask, TOL_BF16)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_bf16_random_masks_small_vit(seed):
+    h = _h()
+    w = wl.vit_b(seed=20 + seed, p_select=0.3, n_blocks=3, tokens=[197, 520, 1000, 333][seed], d=256, ffn=768)
+    if not w.mask.any():
+        w.mask[-2:] = 1
+    h.check_step(w, w.mask, TOL_BF16)
+
+
+def test_bf16_ragged_widths_and_bias_only_selection():
+    h = _h()
+    layers = [wl.Layer(72, 200, act=wl.ACT_RELU), wl.Layer(200, 72, residual_src=0),
+              wl.Layer(72, 328, act=wl.ACT_GELU_TANH), wl.Layer(328, 136)]
+    mask = np.array([0, 1, 0, 0, 1, 0, 0, 1], dtype=np.uint8)
+    w = wl.small_stack(layers, 450, wl.DT_BF16, 5, mask=mask, w_std=0.1, bias_std=0.05)
+    h.check_step(w, mask, TOL_BF16)
+    w = wl.small_stack(layers, 129, wl.DT_BF16, 6, mask=np.ones(8, dtype=np.uint8), w_std=0.1, bias_std=0.05)
+    h.check_step(w, w.mask, TOL_BF16)
+
+
+def test_bf16_resnet_1x1_config():
+    h = _h()
+    w = wl.resnet_1x1()
+    h.check_step(w, w.mask, TOL_BF16)
+
+
+def test_bf16_deterministic():
+    h = _h()
+    w = wl.vit_b(seed=31, p_select=0.5, n_blocks=2, tokens=700, d=256, ffn=512)
+    w.mask[:] = 1
+    outs = []
+    for _ in range(2):
+        run = h.GpuRun(w)
+        run.forward_loss()
+        grads = run.alloc_grads(w.mask)
+        delta = [h.to_dev(d, w.dtype) for d in wl.draw_delta(w, 4)]
+        run.backward(w.mask, grads, delta)
+        outs.append(([g.clone() for g in grads], run.importance.clone()))
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert torch.equal(a, b)
+    assert torch.equal(outs[0][1], outs[1][1])
+
+
+def test_bf16_vit_b_full_size_config():
+    """The benchmark configuration itself (12 blocks, 12608 tokens, Bernoulli(0.3) mask),
+    launched exactly as bench.py launches it, against the full oracle."""
+    h = _h()
+    w = wl.vit_b()
+    stats = {}
+    h.check_step(w, w.mask, TOL_BF16, stats=stats)
+    print("vit_b worst gradient error", stats)

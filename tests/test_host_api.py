@@ -1,0 +1,156 @@
+"""Host-side checks that need no GPU: the library loads and exports every symbol the
+header declares, argument validation, and the selector DP against the oracle's brute force."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2312_14227_b200 as et
+import workloads as wl
+from oracle import elastic_oracle as orc
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    with open(os.path.join(ROOT, "include", "et.h")) as f:
+        header = f.read()
+    declared = set(re.findall(r"\b(et_[a-z_0-9]+)\s*\(", header))
+    assert len(declared) >= 18
+    lib = ctypes.CDLL(et.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} declared in et.h but not exported"
+    assert declared == set(et.EXPORTED_SYMBOLS)
+
+
+def test_status_strings():
+    assert et.et_status_string(0) == "ok"
+    assert "timed out" in et.et_status_string(et.ET_ERR_TIMEOUT)
+
+
+def _err(layers, M=16, dtype=et.ET_F32):
+    with pytest.raises(et.EtError) as e:
+        et.et_stack_create(layers, M, dtype)
+    return e.value.status
+
+
+def test_create_validates_the_layer_chain():
+    ok = et.et_stack_create([(8, 16, 1, 1, -1), (16, 8, 0, 1, 0)], 4, et.ET_F32)
+    assert et.et_stack_workspace_bytes(ok) % 256 == 0
+    assert _err([(8, 16, 0, 1, -1), (12, 8, 0, 1, -1)]) == et.ET_ERR_SHAPE          # widths do not chain
+    assert _err([(8, 16, 0, 1, -1), (16, 4, 0, 1, 0)]) == et.ET_ERR_SHAPE           # residual width mismatch
+    assert _err([(8, 15, 0, 2, -1)]) == et.ET_ERR_SHAPE                             # fold does not divide
+    assert _err([(8, 16, 1, 2, -1)]) == et.ET_ERR_UNSUPPORTED                       # activation under a fold
+    assert _err([(8, 16, 7, 1, -1)]) == et.ET_ERR_INVALID_ARG                       # unknown activation
+    assert _err([(8, 16, 0, 1, 1)]) == et.ET_ERR_INVALID_ARG                        # residual from the future
+    assert _err([(8, 16, 0, 1, -1)], M=0) == et.ET_ERR_INVALID_ARG
+    assert _err([(8, 16, 0, 1, -1)], dtype=5) == et.ET_ERR_DTYPE
+    assert _err([(8, 12, 0, 1, -1)], dtype=et.ET_BF16) == et.ET_ERR_UNSUPPORTED     # bf16 needs multiples of 8
+    assert _err([(8, 384, 0, 3, -1)], dtype=et.ET_BF16) == et.ET_ERR_UNSUPPORTED    # folded width not a tile multiple
+
+
+def test_calls_before_bind_are_refused():
+    s = et.et_stack_create([(8, 16, 0, 1, -1)], 4, et.ET_F32)
+    x = np.zeros(1, dtype=np.float32)     # any non-null address: nothing may be launched
+    with pytest.raises(et.EtError) as e:
+        et.et_forward_stack(s, x, x)
+    assert e.value.status == et.ET_ERR_STATE
+    with pytest.raises(et.EtError) as e:
+        et.et_backward_elastic(s, x, np.zeros(2, dtype=np.uint8))
+    assert e.value.status == et.ET_ERR_STATE
+    with pytest.raises(et.EtError) as e:
+        et.et_backward_elastic(s, x, np.zeros(3, dtype=np.uint8))                   # wrong mask length
+    assert e.value.status == et.ET_ERR_INVALID_ARG
+
+
+def test_workspace_is_sized_for_the_paper_shaped_stacks():
+    w = wl.vit_b(params=False)
+    s = et.et_stack_create(w.layers, w.M, et.ET_BF16)
+    gb = et.et_stack_workspace_bytes(s) / 1e9
+    assert 2.0 < gb < 20.0
+    w = wl.vit_l(params=False)
+    s = et.et_stack_create(w.layers, w.M, et.ET_BF16)
+    assert et.et_stack_workspace_bytes(s) / 1e9 < 40.0
+
+
+@pytest.mark.parametrize("variant", [et.ET_COST_STRICT, et.ET_COST_INCLUSIVE])
+def test_time_selective_matches_oracle(variant):
+    rng = np.random.default_rng(variant)
+    for _ in range(100):
+        n = int(rng.integers(1, 12))
+        _, t_dw, t_dy = wl.selector_instance(rng, n, integer=False)
+        mask = (rng.random(n) < 0.4).astype(np.uint8)
+        assert et.et_time_selective(mask, t_dw, t_dy, variant) == pytest.approx(
+            orc.t_selective(mask, t_dw, t_dy, variant), rel=1e-12, abs=1e-12)
+
+
+@pytest.mark.parametrize("variant", [et.ET_COST_STRICT, et.ET_COST_INCLUSIVE])
+def test_dp_matches_bruteforce(variant):
+    rng = np.random.default_rng(100 + variant)
+    for trial in range(120):
+        n = int(rng.integers(1, 13))
+        I, qw, qy = wl.selector_instance(rng, n, t_max=15)
+        if trial % 4 == 0:
+            I[rng.integers(0, n)] = -0.5
+        if trial % 7 == 0:
+            qw[rng.integers(0, n)] = 0
+        qw, qy = qw.astype(np.int64), qy.astype(np.int64)
+        budget = int(rng.integers(0, int(qw.sum() + qy.sum()) + 3))
+        mask, val = et.et_select_dp_int(I, qw, qy, budget, variant)
+        _, want = orc.select_bruteforce(I, qw, qy, budget, variant)
+        assert abs(val - want) < 1e-12, (trial, n, budget)
+        assert orc.t_selective(mask, qw, qy, variant) <= budget                     # returned mask is feasible
+        assert abs(I[mask.astype(bool)].sum() - val) < 1e-12                        # and attains the value
+
+
+def test_dp_larger_instance_against_depth_knapsack():
+    rng = np.random.default_rng(5)
+    I, qw, qy = wl.selector_instance(rng, 96, t_max=40)
+    qw, qy = qw.astype(np.int64), qy.astype(np.int64)
+    for frac in (0.1, 0.4, 0.8):
+        budget = int(frac * (qw.sum() + qy.sum()))
+        for variant in (et.ET_COST_STRICT, et.ET_COST_INCLUSIVE):
+            mask, val = et.et_select_dp_int(I, qw, qy, budget, variant)
+            assert abs(val - orc.select_by_depth_knapsack(I, qw, qy, budget, variant)) < 1e-9
+            assert orc.t_selective(mask, qw, qy, variant) <= budget
+
+
+def test_dp_edge_cases():
+    I = np.array([0.5, 0.2, 0.9])
+    w = np.array([3, 1, 2]); y = np.array([4, 0, 5])
+    mask, val = et.et_select_dp_int(I, w, y, -1)
+    assert not mask.any() and val == 0.0
+    mask, val = et.et_select_dp_int(I, w, y, 0)
+    assert not mask.any()
+    mask, val = et.et_select_dp_int(I, w, y, 1000)
+    assert mask.all() and abs(val - I.sum()) < 1e-12
+    mask, val = et.et_select_dp_int(np.array([-1.0, -2.0]), np.array([1, 1]), np.array([1, 1]), 100)
+    assert not mask.any() and val == 0.0                                             # empty selection is allowed
+    mask, val = et.et_select_dp_int(np.zeros(0), np.zeros(0, dtype=np.int64), np.zeros(0, dtype=np.int64), 5)
+    assert len(mask) == 0 and val == 0.0
+    with pytest.raises(et.EtError):
+        et.et_select_dp_int(I, np.array([-1, 0, 0]), y, 5)
+
+
+def test_select_dp_quantised():
+    rng = np.random.default_rng(9)
+    for _ in range(30):
+        n = int(rng.integers(2, 12))
+        I, t_dw, t_dy = wl.selector_instance(rng, n, integer=False)
+        rho = float(rng.uniform(0.2, 1.0))
+        t_fwd = float(rng.uniform(0, 5))
+        Tq = 200
+        mask, val, est = et.et_select_dp(I, t_dw, t_dy, t_fwd, rho, Tq, et.ET_COST_STRICT)
+        qw, qy, budget = orc.quantise(t_dw, t_dy, t_fwd, rho, Tq)
+        _, want = orc.select_bruteforce(I, qw, qy, budget, orc.STRICT)
+        assert abs(val - want) < 1e-9
+        assert est == pytest.approx(orc.t_selective(mask, t_dw, t_dy, orc.STRICT), rel=1e-12, abs=1e-12)
+        # flooring under-estimates each time by < 1 quantum: the true time overshoots the budget by < n quanta
+        T = t_dw.sum() + t_dy.sum()
+        assert est <= rho * (t_fwd + T) - t_fwd + 2 * n * T / Tq + 1e-9
+    # rho = 1: everything is selected
+    I, t_dw, t_dy = wl.selector_instance(rng, 40, integer=False)
+    mask, val, est = et.et_select_dp(I + 0.01, t_dw, t_dy, 3.0, 1.0, 1000, et.ET_COST_INCLUSIVE)
+    assert mask.all()

@@ -202,3 +202,14 @@ def selector_instance(rng, n: int, t_max: int = 20, integer: bool = True):
         t_dy = rng.random(n) * t_max
     t_dy[1::2] = 0.0
     return I, t_dw, t_dy
+
+
+def draw_delta(w: Workload, seed: int, std: float = 1e-3):
+    """A recent weight update dw for every tensor (the second factor of the importance
+    sum), in tensor order [dW_0, db_0, ...], representable in the workload's dtype."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for ly in w.layers:
+        out.append(_store(rng.normal(0.0, std, size=(ly.in_features, ly.out_features)), w.dtype))
+        out.append(_store(rng.normal(0.0, std, size=ly.out_features), w.dtype))
+    return out
