@@ -88,16 +88,37 @@ def rel_max(a: np.ndarray, o: np.ndarray) -> float:
 
 
 def importance_err(s_gpu: float, g: np.ndarray, d: np.ndarray) -> float:
+    """Error of an importance sum relative to max(|S|, ||g||_inf * ||dw||_2).  The second
+    term is the size of the error that gradient entries which are each off by
+    tol * ||g||_inf, independently, put into the sum; it only matters when the terms of
+    the sum cancel (a dw unrelated to g)."""
     s_o = float(np.sum(g * d))
-    floor = 1e-6 * float(np.sum(np.abs(g * d)))
+    floor = float(np.abs(g).max()) * float(np.sqrt(np.sum(d * d)))
     return abs(s_gpu - s_o) / max(abs(s_o), floor, 1e-300)
 
 
-def check_step(w: wl.Workload, mask, tol: float, delta_seed: int = 77, w_tol: float = 1e-3, stats=None):
+def gradient_step_delta(w: wl.Workload, mask):
+    """dw = -c * g with the oracle's own gradient (the update a gradient step makes), scaled
+    to about 1e-3 and rounded to the storage type: the terms of the importance sum then all
+    have one sign, so its plain relative error is meaningful."""
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    grads, _ = orc.backward_masked(w.layers, w.W, saved, dY, mask)
+    rnd = wl.round_to_bf16 if w.dtype == wl.DT_BF16 else wl.round_to_f32
+    out = wl.draw_delta(w, 0)
+    for t, g in grads.items():
+        m = float(np.abs(g).max())
+        out[t] = rnd(-(1e-3 / m) * g) if m > 0 else np.zeros_like(g)
+    return out
+
+
+def check_step(w: wl.Workload, mask, tol: float, delta_seed: int = 77, w_tol: float = 1e-3, stats=None,
+               aligned_delta: bool = False):
     """Full parity check of one training step: forward, loss, elastic backward with fused
-    importance and SGD.  Returns the report."""
+    importance and SGD.  Returns the report.  With aligned_delta the importance is checked
+    by its plain relative error."""
     mask = np.asarray(mask, dtype=np.uint8)
-    delta_np = wl.draw_delta(w, delta_seed)
+    delta_np = gradient_step_delta(w, mask) if aligned_delta else wl.draw_delta(w, delta_seed)
     ref = oracle_step(w, mask, delta_np)
     run = GpuRun(w)
     before = [p.clone() for p in run.params()]
@@ -128,6 +149,8 @@ def check_step(w: wl.Workload, mask, tol: float, delta_seed: int = 77, w_tol: fl
             assert e <= tol, (t, e)
             ie = importance_err(imp[t], ref["grads"][t], delta_np[t])
             assert ie <= tol, (t, ie, imp[t])
+            if aligned_delta and ref["importance"][t] != 0.0:
+                assert abs(imp[t] - ref["importance"][t]) <= tol * abs(ref["importance"][t]), t
             new = to_np(run.params()[t])
             assert float(np.abs(new - ref["new"][t]).max()) <= w_tol, t
         else:

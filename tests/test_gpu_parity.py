@@ -34,6 +34,16 @@ def test_tiny_mlp_fp32_all_selected_is_full_backprop():
     h.check_step(w, np.ones(2 * w.L, dtype=np.uint8), TOL_F32)
 
 
+def test_importance_of_a_gradient_step_fp32_and_bf16():
+    # dw proportional to -g (Eq. 2 with the update a gradient step makes): plain relative error
+    h = _h()
+    w = wl.tiny_mlp()
+    h.check_step(w, np.ones(2 * w.L, dtype=np.uint8), TOL_F32, aligned_delta=True)
+    w = wl.vit_b(seed=12, p_select=0.5, n_blocks=2, tokens=520, d=256, ffn=768)
+    w.mask[:] = 1
+    h.check_step(w, w.mask, TOL_BF16, aligned_delta=True)
+
+
 def _all_kinds_layers(scale=1):
     s = scale
     return [
