@@ -113,10 +113,13 @@ def gradient_step_delta(w: wl.Workload, mask):
 
 
 def check_step(w: wl.Workload, mask, tol: float, delta_seed: int = 77, w_tol: float = 1e-3, stats=None,
-               aligned_delta: bool = False):
+               aligned_delta: bool = False, derived_w_tol: bool = False):
     """Full parity check of one training step: forward, loss, elastic backward with fused
     importance and SGD.  Returns the report.  With aligned_delta the importance is checked
-    by its plain relative error."""
+    by its plain relative error.  Updated weights must be within w_tol (1e-3) of the oracle's;
+    with derived_w_tol the bound also admits what the arithmetic cannot avoid when weights or
+    gradients are large: the bf16 store's half ulp (2^-9 |w|) and lr * tol * ||g||_inf from the
+    gradient's own tolerance."""
     mask = np.asarray(mask, dtype=np.uint8)
     delta_np = gradient_step_delta(w, mask) if aligned_delta else wl.draw_delta(w, delta_seed)
     ref = oracle_step(w, mask, delta_np)
@@ -152,7 +155,11 @@ def check_step(w: wl.Workload, mask, tol: float, delta_seed: int = 77, w_tol: fl
             if aligned_delta and ref["importance"][t] != 0.0:
                 assert abs(imp[t] - ref["importance"][t]) <= tol * abs(ref["importance"][t]), t
             new = to_np(run.params()[t])
-            assert float(np.abs(new - ref["new"][t]).max()) <= w_tol, t
+            bound = w_tol
+            if derived_w_tol:
+                half_ulp = 2.0 ** -9 * np.abs(ref["new"][t]) if w.dtype == wl.DT_BF16 else 0.0
+                bound = w_tol + half_ulp + w.lr * tol * float(np.abs(ref["grads"][t]).max())
+            assert np.all(np.abs(new - ref["new"][t]) <= bound), t
         else:
             assert imp[t] == 0.0
             assert torch.equal(run.params()[t], before[t]), f"frozen tensor {t} was written"

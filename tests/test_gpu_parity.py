@@ -150,7 +150,9 @@ def test_bf16_ragged_widths_and_bias_only_selection():
 def test_bf16_resnet_1x1_config():
     h = _h()
     w = wl.resnet_1x1()
-    h.check_step(w, w.mask, TOL_BF16)
+    # He-initialised weights reach 0.5 and gradients reach 35 here: a bf16 store alone is
+    # off by up to 2^-9 |w| ~ 1e-3, so the weight bound is the derived one
+    h.check_step(w, w.mask, TOL_BF16, derived_w_tol=True)
 
 
 def test_bf16_deterministic():
