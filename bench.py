@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the elastic backward step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one pass of the hot path over one batch: the execution plan from the mask, the
+error-gradient GEMMs above the deepest selected layer, the weight-gradient GEMMs, bias
+gradients, importance reduction and masked SGD of the selected tensors.  The forward pass and
+the loss gradient run once before the timed region (they precede the hot path).
+
+Workload: the ViT-B/16-shaped linear-only stack (12 blocks, 64 x 197 tokens, bf16 storage with
+fp32 accumulation, seeded Bernoulli(0.3) selection mask), synthetic N(0,1) inputs.
+Metric: executed TFLOP/s of the elastic backward step (2*M*K*N per executed GEMM; work the
+mask removes is not counted), with the step time beside it and the full-backprop step time
+for comparison.
+
+With --gpus N > 1 every rank runs an independent replica (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "elastic_backward_executed_tflops"
+UNIT = "TFLOP/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], tf_burst=p["bf16_tflops"], tf_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------ reference arm
+def oracle_sample(w_full: wl.Workload, n_blocks: int):
+    """Bounded sample of the workload for the CPU oracle: the top n_blocks transformer blocks of
+    the same stack (same widths, same token count, the mask bits of those layers)."""
+    from oracle import elastic_oracle as orc
+    layers = wl.vit_blocks(n_blocks, 768, 3072)
+    L = len(layers)
+    mask = w_full.mask[-2 * L:].copy()
+    if not mask.any():
+        mask[-2:] = 1
+    w = wl.small_stack(layers, w_full.M, wl.DT_BF16, 123, mask=mask, w_std=0.02)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    delta = wl.draw_delta(w, 5)
+    params = orc.tensors_of(w.W, w.b)
+
+    def step():
+        t0 = time.perf_counter()
+        grads, plan = orc.backward_masked(w.layers, w.W, saved, dY, mask)
+        orc.importance(grads, delta, mask)
+        orc.sgd_masked(params, grads, mask, w.lr)
+        dt = time.perf_counter() - t0
+        return dt, orc.executed_flops(w.layers, w.M, plan)
+
+    return step, f"oracle masked backward + importance + SGD on the top {n_blocks} of 12 blocks, all {w.M} tokens, float64"
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.vit_b(params=False)
+    step, sample = oracle_sample(w, 1)          # one block per step keeps K steps within minutes
+    for _ in range(min(args.warmup, 1)):
+        step()
+    times, flops = [], 0.0
+    for _ in range(args.steps):
+        dt, flops = step()
+        times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    val = flops / (ms * 1e-3) / 1e12
+    cores = blas_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "vit_b_linear_bf16 (oracle sample)", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ own arm
+def run_own(args):
+    import torch
+    import paper_2312_14227_b200 as et
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = wl.vit_b()
+    tdt = torch.bfloat16
+
+    def to_dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
+
+    stack = et.et_stack_create(w.layers, w.M, w.dtype)
+    W = [to_dev(a) for a in w.W]
+    b = [to_dev(a) for a in w.b]
+    ws = torch.empty(et.et_stack_workspace_bytes(stack), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    et.et_stack_bind(stack, W, b, ws, stream=stream)
+    x, target = to_dev(w.x), to_dev(w.target)
+    y = torch.empty((w.M, w.layers[-1].out_width), dtype=tdt, device=dev)
+    dY = torch.empty_like(y)
+    delta = [to_dev(d) for d in wl.draw_delta(w, 5)]
+    imp = torch.zeros(2 * w.L, dtype=torch.float32, device=dev)
+    et.et_forward_stack(stack, x, y, stream=stream)
+    et.et_loss_mse_grad(stack, y, target, dY, None, stream=stream)
+    torch.cuda.synchronize()
+    dY_host = dY.cpu().pin_memory()
+    imp_host = torch.zeros(2 * w.L, dtype=torch.float32).pin_memory()
+    ones = np.ones(2 * w.L, dtype=np.uint8)
+    rep = et.Report(w.L)
+    flags = et.ET_FLAG_FUSE_SGD
+
+    def step(mask):
+        et.et_backward_elastic(stack, dY, mask, None, delta, imp, flags, w.lr, rep, stream=stream)
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = et.et_launch_count()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, et.et_launch_count() - n0
+
+    # forward (context) and full backprop (comparison)
+    fwd_ms, _ = timed(lambda: et.et_forward_stack(stack, x, y, stream=stream), max(2, args.steps // 4), 2)
+    full_ms, _ = timed(lambda: step(ones), args.steps, args.warmup)
+    full_flops = rep.flops_executed
+
+    # the headline: elastic step, device-resident inputs
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, launches = timed(lambda: step(w.mask), args.steps, args.warmup)
+    clocks = sampler.stop()
+    flops = rep.flops_executed
+    st = et.et_device_status(stack, stream=stream)
+    assert st == et.ET_OK, et.et_status_string(st)
+    value = world * flops / (ms * 1e-3) / 1e12
+
+    # end to end through the host-buffer entry point: dY comes from pinned host memory and the
+    # importances go back to it, inside the timed region
+    def step_host():
+        et.et_backward_elastic_host(stack, dY_host, w.mask, None, delta, imp_host, flags, w.lr, rep, stream=stream)
+
+    e2e_ms, _ = timed(step_host, args.steps, args.warmup)
+    e2e_value = world * flops / (e2e_ms * 1e-3) / 1e12
+
+    # per-kernel-class device time over the same steps (event pair around every launch)
+    et.et_timing_enable(stack, True)
+    inst_ms, _ = timed(lambda: step(w.mask), args.steps, 1)
+    classes = et.et_timing_read(stack)
+    # the first (warm-up) step is included in the record: normalise by launches
+    et.et_timing_enable(stack, False)
+
+    peaks = _peaks()
+    # algorithmic work per class for the elastic mask
+    M = w.M
+    first = next(l for l in range(w.L) if w.mask[2 * l] or w.mask[2 * l + 1])
+    dgrad_flops = sum(2.0 * M * ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if l > first)
+    wgrad_flops = sum(2.0 * M * ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if w.mask[2 * l])
+    n_steps_rec = args.steps + 1
+
+    def per_step(cls):
+        t, n = classes[cls]
+        return t / n_steps_rec, n / n_steps_rec
+
+    dg_ms, dg_n = per_step("dgrad")
+    wg_ms, wg_n = per_step("wgrad")
+    rd_ms, rd_n = per_step("wgrad_reduce")
+    bg_ms, bg_n = per_step("bgrad")
+    ot_ms, ot_n = per_step("other")
+    # bytes the reducer must move per selected kernel tensor of P parameters: S*4P partial reads
+    # are its own scratch traffic; the algorithmic part is 4P (gradient) + 2P (dW) + 2P + 2P (W in/out)
+    sel_params = sum(ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if w.mask[2 * l])
+    reduce_bytes = 10.0 * sel_params
+    bgrad_bytes = sum(2.0 * M * ly.out_width for l, ly in enumerate(w.layers) if w.mask[2 * l + 1])
+    dg_tf = dgrad_flops / (dg_ms * 1e-3) / 1e12 if dg_ms > 0 else 0.0
+    kernels = {
+        "dgrad_gemm": {"launches_per_step": dg_n, "ms_per_step": dg_ms, "achieved": dg_tf, "unit": "TFLOP/s",
+                       "frac_of_sustained_peak": dg_tf / peaks["tf_sustained"]},
+        "wgrad_gemm": {"launches_per_step": wg_n, "ms_per_step": wg_ms,
+                       "achieved": wgrad_flops / (wg_ms * 1e-3) / 1e12 if wg_ms > 0 else 0.0, "unit": "TFLOP/s"},
+        "wgrad_reduce_importance_sgd": {"launches_per_step": rd_n, "ms_per_step": rd_ms,
+                                        "achieved": reduce_bytes / (rd_ms * 1e-3) / 1e9 if rd_ms > 0 else 0.0,
+                                        "unit": "GB/s"},
+        "bias_grad": {"launches_per_step": bg_n, "ms_per_step": bg_ms,
+                      "achieved": bgrad_bytes / (bg_ms * 1e-3) / 1e9 if bg_ms > 0 else 0.0, "unit": "GB/s"},
+        "other": {"launches_per_step": ot_n, "ms_per_step": ot_ms},
+        "instrumented_step_ms": inst_ms,
+    }
+    kernels["wgrad_gemm"]["frac_of_sustained_peak"] = kernels["wgrad_gemm"]["achieved"] / peaks["tf_sustained"]
+    kernels["wgrad_reduce_importance_sgd"]["frac_of_hbm_peak"] = \
+        kernels["wgrad_reduce_importance_sgd"]["achieved"] / peaks["hbm_gbs"]
+    kernels["bias_grad"]["frac_of_hbm_peak"] = kernels["bias_grad"]["achieved"] / peaks["hbm_gbs"]
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": w.name, "blocks": 12, "tokens": w.M, "d": 768, "ffn": 3072,
+                   "mask": "Bernoulli(0.3) per kernel tensor, seed 1, bias follows kernel",
+                   "selected_tensors": int(w.mask.sum()), "deepest_selected_layer": first,
+                   "step": "et_backward_elastic with fused importance and SGD",
+                   "l2": "inputs larger than L2 (a step streams > 1 GB of activations and gradients)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "executed_flops_per_step": flops,
+        "pct_of_measured_bf16_peak": {"sustained": value / world / peaks["tf_sustained"],
+                                      "burst": value / world / peaks["tf_burst"], "source": peaks["source"]},
+        "full_backprop": {"ms_per_step": full_ms, "tflops": full_flops / (full_ms * 1e-3) / 1e12,
+                          "executed_flops_per_step": full_flops, "elastic_speedup": full_ms / ms},
+        "forward_ms": fwd_ms,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": dY_host.numel() * dY_host.element_size(),
+                "d2h_bytes_per_step": imp_host.numel() * 4},
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "gemm_tc_kernel<dgrad>", "bound": "tensor", "achieved": dg_tf,
+                     "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": dg_tf / peaks["tf_sustained"],
+                     "peak_source": peaks["source"] + " (sustained cuBLAS bf16)", "traffic": None},
+        "kernels": kernels,
+    }
+    if world == 1:
+        cpu_step, sample = oracle_sample(w, 2)
+        dt, fl = cpu_step()
+        line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": sample, "seconds": dt}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_own(args)
+
+
+if __name__ == "__main__":
+    main()

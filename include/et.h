@@ -197,6 +197,27 @@ et_status et_select_dp_int(const double* importance, const int64_t* t_dw, const 
                            int32_t n, int64_t budget, int32_t variant,
                            uint8_t* mask_out, double* value_out);
 
+/* ---- per-kernel timing (measurement support) ---------------------------------------- */
+
+/* Kernel classes for et_timing_read. */
+typedef enum {
+  ET_K_FORWARD = 0,        /* forward GEMM (+bias, activation, fold, residual)          */
+  ET_K_DGRAD = 1,          /* error-gradient GEMM with its fused epilogue (Section 5.1 T1, 5.3) */
+  ET_K_WGRAD = 2,          /* weight-gradient GEMM writing split partials (T3)          */
+  ET_K_WGRAD_REDUCE = 3,   /* split reduction + gradient export + importance + SGD      */
+  ET_K_BGRAD = 4,          /* bias gradient: column sums + finish (T2)                  */
+  ET_K_OTHER = 5,          /* loss gradient, top-layer activation backward, importance finalise */
+  ET_K_CLASSES = 6
+} et_kernel_class;
+
+/* on != 0: every kernel this stack launches from now on is bracketed by a pair of CUDA
+ * events on its stream (host objects; no device memory).  on == 0: stop and drop them. */
+et_status et_timing_enable(et_stack* s, int32_t on);
+/* Waits for the recorded events, adds up device time (milliseconds) and launch counts per
+ * class into ms[ET_K_CLASSES] / launches[ET_K_CLASSES] (either may be NULL), and clears the
+ * record. */
+et_status et_timing_read(et_stack* s, double* ms, int64_t* launches);
+
 /* ---- status ------------------------------------------------------------------------ */
 
 /* Synchronises `stream` and reports ET_ERR_TIMEOUT if a kernel's bounded wait gave up,

@@ -52,6 +52,8 @@ _SIGS = {
     "et_select_dp": [_vp, _vp, _vp, _i32, _f64, _f64, _i32, _i32, _vp, _vp, _vp],
     "et_select_dp_int": [_vp, _vp, _vp, _i32, _i64, _i32, _vp, _vp],
     "et_device_status": [_vp, _vp],
+    "et_timing_enable": [_vp, _i32],
+    "et_timing_read": [_vp, _vp, _vp],
 }
 for _name, _args in _SIGS.items():
     _fn = getattr(_lib, _name)
@@ -268,9 +270,24 @@ def et_profile_costs(s: Stack, x, y, dY, iters: int = 20, stream=None):
     return t_dw, t_dy, t_fwd.value
 
 
+KERNEL_CLASSES = ("forward", "dgrad", "wgrad", "wgrad_reduce", "bgrad", "other")
+
+
+def et_timing_enable(s: Stack, on: bool):
+    _check(_lib.et_timing_enable(s.handle, 1 if on else 0), "et_timing_enable")
+
+
+def et_timing_read(s: Stack):
+    """{class name: (milliseconds, launches)} since the last read."""
+    ms = np.zeros(len(KERNEL_CLASSES), dtype=np.float64)
+    n = np.zeros(len(KERNEL_CLASSES), dtype=np.int64)
+    _check(_lib.et_timing_read(s.handle, _ptr(ms), _ptr(n)), "et_timing_read")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_CLASSES)}
+
+
 def et_device_status(s: Stack, stream=None) -> int:
     return int(_lib.et_device_status(s.handle, _stream_ptr(stream)))
 
 
 __all__ = [n for n in dir() if n.startswith(("et_", "ET_"))] + ["Stack", "Report", "EtError", "LIB_PATH",
-                                                                 "EXPORTED_SYMBOLS"]
+                                                                 "EXPORTED_SYMBOLS", "KERNEL_CLASSES"]

@@ -111,6 +111,11 @@ struct et_stack {
   const void* x = nullptr;
   CUtensorMap map_x, map_dy;
   const void* map_dy_ptr = nullptr;
+  // optional per-kernel timing
+  bool timing = false;
+  struct Timed { int cls; cudaEvent_t e0, e1; };
+  std::vector<Timed> timed;            // recorded this period
+  std::vector<cudaEvent_t> event_pool; // spare events
 
   char* at(size_t off) const { return ws + off; }
   int width_in(int l) const { return ly[l].K; }
@@ -133,6 +138,27 @@ int choose_split(int tiles, int kb_total, int sms) {
   }
   return best;
 }
+
+// ---- per-kernel timing: an event pair around one launch ---------------------------------------
+cudaEvent_t take_event(et_stack* s) {
+  cudaEvent_t e = nullptr;
+  if (!s->event_pool.empty()) { e = s->event_pool.back(); s->event_pool.pop_back(); return e; }
+  if (cudaEventCreate(&e) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+  return e;
+}
+struct TimedLaunch {
+  et_stack* s; cudaStream_t st; cudaEvent_t e0 = nullptr, e1 = nullptr; int cls;
+  TimedLaunch(et_stack* s_, int cls_, cudaStream_t st_) : s(s_), st(st_), cls(cls_) {
+    if (!s->timing) return;
+    e0 = take_event(s); e1 = take_event(s);
+    if (e0 != nullptr) cudaEventRecord(e0, st);
+  }
+  ~TimedLaunch() {
+    if (e0 == nullptr || e1 == nullptr) return;
+    cudaEventRecord(e1, st);
+    s->timed.push_back({cls, e0, e1});
+  }
+};
 
 template <typename T> struct is_bf16 : std::false_type {};
 template <> struct is_bf16<bf16> : std::true_type {};
@@ -192,6 +218,7 @@ et::tc::Params tc_params(const et_stack* s, int rows, int cols, int contraction,
 // Z_l = a_l W_l + b_l, activation, fold, residual -> a_{l+1}
 template <typename T>
 et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_FORWARD, st);
   const LayerRT& L = s->ly[l];
   et::FwdEpi<T> epi;
   epi.bias = (const T*)L.b;
@@ -217,6 +244,7 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
 // G_l = dZ_l W_l^T (+ skip gradient), dZ_{l-1} = G_l * act'(Z_{l-1});  l >= 1
 template <typename T>
 et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_DGRAD, st);
   const LayerRT& L = s->ly[l];
   const LayerRT& P = s->ly[l - 1];
   et::DgradEpi<T> epi;
@@ -255,20 +283,24 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   et::PartialEpi epi;
   epi.base = partial; epi.split_stride = count; epi.ld = L.N; epi.split = 0;
   int split = 1;
-  if constexpr (is_bf16<T>::value) {
-    split = L.split;
-    et::tc::Params p = tc_params(s, L.K, L.N, (int)s->M, 1, split);
-    p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
-    ET_TRY((launch_tc<true, true>(a_map(s, l), dz_map(s, l), p, epi, s->sms, st)));
-  } else {
-    et::simt::Params p;
-    p.rows = L.K; p.cols = L.N; p.kc = (int)s->M; p.segs = 1;
-    p.sa_i = 1; p.sa_k = L.K;
-    p.sb_k = L.Nw; p.sb_seg = 0; p.sb_j = 1; p.b_wrap = L.fold > 1 ? L.Nw : 0;
-    ET_TRY(launch_simt<T>(act_in<T>(s, l), dz_src<T>(s, l, dY), p, epi, st));
+  {
+    TimedLaunch tl(s, ET_K_WGRAD, st);
+    if constexpr (is_bf16<T>::value) {
+      split = L.split;
+      et::tc::Params p = tc_params(s, L.K, L.N, (int)s->M, 1, split);
+      p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
+      ET_TRY((launch_tc<true, true>(a_map(s, l), dz_map(s, l), p, epi, s->sms, st)));
+    } else {
+      et::simt::Params p;
+      p.rows = L.K; p.cols = L.N; p.kc = (int)s->M; p.segs = 1;
+      p.sa_i = 1; p.sa_k = L.K;
+      p.sb_k = L.Nw; p.sb_seg = 0; p.sb_j = 1; p.b_wrap = L.fold > 1 ? L.Nw : 0;
+      ET_TRY(launch_simt<T>(act_in<T>(s, l), dz_src<T>(s, l, dY), p, epi, st));
+    }
   }
   ++*launches;
   if (grad == nullptr && delta == nullptr && !sgd) return ET_OK;     // nothing consumes g
+  TimedLaunch tl(s, ET_K_WGRAD_REDUCE, st);
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
   et::wgrad_reduce_kernel<T><<<L.imp_count_w, et::kEltThreads, 0, st>>>(partial, split, count, count, grad, delta, imp,
                                                                         (T*)L.W, lr, sgd ? 1 : 0);
@@ -279,6 +311,7 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
 template <typename T>
 et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
                           int* launches, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_BGRAD, st);
   const LayerRT& L = s->ly[l];
   float* part = (float*)s->at(s->off_biaspart);
   const int chunks = ceil_div(s->M, et::kColsumRows);
@@ -344,6 +377,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
     }
     const LayerRT& top = s->ly[L - 1];
     if (top.act != ET_ACT_NONE) {
+      TimedLaunch tl(s, ET_K_OTHER, st);
       const size_t count = (size_t)s->M * top.N;
       et::act_backward_kernel<T><<<ceil_div(count, et::kEltThreads * et::kVec), et::kEltThreads, 0, st>>>(
           (const T*)dY, (const T*)s->at(top.off_Z), (T*)s->at(top.off_dZ), count, top.act);
@@ -369,6 +403,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
       }
     }
     if (delta != nullptr) {
+      TimedLaunch tl(s, ET_K_OTHER, st);
       et::importance_finalize_kernel<<<2 * L, 128, 0, st>>>((const float*)s->at(s->off_imp_parts),
                                                             (const int*)s->at(s->off_imp_offs),
                                                             (const int*)s->at(s->off_imp_counts), mask_bits(mask, 2 * L),
@@ -503,6 +538,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
 
 et_status et_stack_destroy(et_stack* s) {
   if (s == nullptr) return ET_ERR_INVALID_ARG;
+  et_timing_enable(s, 0);
   delete s;
   return ET_OK;
 }
@@ -705,6 +741,41 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
   rc = body();
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
+  return rc;
+}
+
+et_status et_timing_enable(et_stack* s, int32_t on) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  s->timing = on != 0;
+  if (!s->timing) {
+    for (auto& t : s->timed) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
+    for (auto e : s->event_pool) cudaEventDestroy(e);
+    s->timed.clear();
+    s->event_pool.clear();
+  }
+  return ET_OK;
+}
+
+et_status et_timing_read(et_stack* s, double* ms, int64_t* launches) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  for (int c = 0; c < ET_K_CLASSES; ++c) {
+    if (ms) ms[c] = 0.0;
+    if (launches) launches[c] = 0;
+  }
+  et_status rc = ET_OK;
+  for (auto& t : s->timed) {
+    float v = 0.f;
+    if (cudaEventSynchronize(t.e1) != cudaSuccess || cudaEventElapsedTime(&v, t.e0, t.e1) != cudaSuccess) {
+      g_last_cuda = (int)cudaGetLastError();
+      rc = ET_ERR_CUDA;
+    } else {
+      if (ms) ms[t.cls] += v;
+      if (launches) launches[t.cls] += 1;
+    }
+    s->event_pool.push_back(t.e0);
+    s->event_pool.push_back(t.e1);
+  }
+  s->timed.clear();
   return rc;
 }
 
