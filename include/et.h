@@ -57,7 +57,8 @@ typedef enum {
   ET_ERR_WORKSPACE = 5,     /* workspace too small or misaligned */
   ET_ERR_UNSUPPORTED = 6,   /* shape outside what the kernels handle */
   ET_ERR_CUDA = 7,          /* a CUDA runtime call failed; see et_last_cuda_error */
-  ET_ERR_TIMEOUT = 8        /* a bounded device-side wait gave up */
+  ET_ERR_TIMEOUT = 8,       /* a bounded device-side wait gave up */
+  ET_ERR_TOO_LARGE = 9      /* problem exceeds the fixed built-in scratch of a *_noalloc call */
 } et_status;
 
 typedef enum { ET_F32 = 0, ET_BF16 = 1 } et_dtype;
@@ -167,6 +168,35 @@ et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
  * rounded once to the storage dtype).  Unselected tensors are never written. */
 et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads,
                         float lr, void* stream);
+
+/* Bias gradient without any allocation.  (The paper has no counterpart for this call; it
+ * exists for how this library gets embedded.)
+ *
+ * Who needs it: code that must not, or cannot, call cudaMalloc or hand the library a
+ * workspace at the point where it needs a bias gradient -- for instance a plug-in running
+ * inside a host application that owns all device memory and gives none out, a callback on a
+ * latency-critical path where an allocation (which may synchronise the device) is forbidden,
+ * or a process whose memory budget is fixed at start-up.  Such a caller still passes its own
+ * input and output buffers; only the intermediate storage comes from the library.
+ *
+ * Computes db[j] = sum over the M rows of dZ[:, j] (Section 5.1's bias update, the same
+ * two-stage fixed-order column reduction et_backward_elastic uses for selected biases).
+ *   dZ     device [M x width], row-major, storage dtype `dtype`, 16-byte aligned
+ *   db     device float[width]
+ * The stage-1 partial sums live in a fixed array compiled into the library:
+ * ET_NOALLOC_SCRATCH_FLOATS floats (4 MiB) on every GPU that loads the library, kept until
+ * the process ends.  A problem needs ceil(M / 128) * width floats of it; a larger one is
+ * refused with ET_ERR_TOO_LARGE and nothing is launched.  The call itself performs no
+ * cudaMalloc / cudaFree and calls no allocating routine.
+ * The first call on each device looks up the device address of that array (with that
+ * device current); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps whatever the last call left in
+ * it.  No clearing is needed (each call overwrites every entry it later reads), but two
+ * calls that run concurrently on the same GPU -- different streams, or different host
+ * threads -- race on it: serialise them.  Asynchronous on `stream`. */
+#define ET_NOALLOC_SCRATCH_FLOATS (1 << 20)
+et_status et_bias_grad_noalloc(const void* dZ, int64_t M, int32_t width, et_dtype dtype, float* db,
+                               void* stream);
 
 /* ---- selection support (host) ------------------------------------------------------ */
 

@@ -23,6 +23,8 @@ ET_COST_STRICT, ET_COST_INCLUSIVE = 0, 1
 ET_FLAG_FUSE_SGD = 1
 ET_ERR_INVALID_ARG, ET_ERR_SHAPE, ET_ERR_DTYPE, ET_ERR_STATE = 1, 2, 3, 4
 ET_ERR_WORKSPACE, ET_ERR_UNSUPPORTED, ET_ERR_CUDA, ET_ERR_TIMEOUT = 5, 6, 7, 8
+ET_ERR_TOO_LARGE = 9
+ET_NOALLOC_SCRATCH_FLOATS = 1 << 20
 
 
 class et_layer_desc(C.Structure):
@@ -52,6 +54,7 @@ _SIGS = {
     "et_select_dp": [_vp, _vp, _vp, _i32, _f64, _f64, _i32, _i32, _vp, _vp, _vp],
     "et_select_dp_int": [_vp, _vp, _vp, _i32, _i64, _i32, _vp, _vp],
     "et_device_status": [_vp, _vp],
+    "et_bias_grad_noalloc": [_vp, _i64, _i32, _i32, _vp, _vp],
     "et_timing_enable": [_vp, _i32],
     "et_timing_read": [_vp, _vp, _vp],
 }
@@ -283,6 +286,14 @@ def et_timing_read(s: Stack):
     n = np.zeros(len(KERNEL_CLASSES), dtype=np.int64)
     _check(_lib.et_timing_read(s.handle, _ptr(ms), _ptr(n)), "et_timing_read")
     return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_CLASSES)}
+
+
+def et_bias_grad_noalloc(dZ, M: int, width: int, dtype: int, db, stream=None):
+    """Column sums of dZ [M x width] into db (float32[width]) using the library's built-in
+    scratch instead of a workspace: for callers that are not allowed to allocate device
+    memory.  Problems over ET_NOALLOC_SCRATCH_FLOATS raise EtError(ET_ERR_TOO_LARGE)."""
+    _check(_lib.et_bias_grad_noalloc(_ptr(dZ), int(M), int(width), dtype, _ptr(db), _stream_ptr(stream)),
+           "et_bias_grad_noalloc")
 
 
 def et_device_status(s: Stack, stream=None) -> int:

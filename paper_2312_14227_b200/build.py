@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libet.so")
-SOURCES = ["et_lib.cu", "select.cpp"]
+SOURCES = ["et_lib.cu", "et_noalloc.cu", "select.cpp"]
 
 
 def _newest_source_mtime() -> float:

@@ -800,6 +800,7 @@ const char* et_status_string(et_status st) {
     case ET_ERR_UNSUPPORTED: return "shape not supported by the kernels";
     case ET_ERR_CUDA: return "CUDA call failed";
     case ET_ERR_TIMEOUT: return "device-side wait timed out";
+    case ET_ERR_TOO_LARGE: return "problem exceeds the built-in scratch capacity of the no-allocation call";
   }
   return "unknown status";
 }

@@ -112,7 +112,7 @@ bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int co
 
 // ---- importance, last stage: per tensor, sum its block partials in a fixed order ----------
 struct MaskBits { uint32_t w[64]; };            // up to 2048 tensors
-__global__ void __launch_bounds__(128)
+static __global__ void __launch_bounds__(128)
 importance_finalize_kernel(const float* __restrict__ parts, const int* __restrict__ offs,
                            const int* __restrict__ counts, const MaskBits active, float* __restrict__ out) {
   const int t = blockIdx.x;
@@ -197,7 +197,7 @@ mse_grad_kernel(const T* __restrict__ y, const T* __restrict__ target, T* __rest
   sq = block_sum(sq);
   if (threadIdx.x == 0) loss_part[blockIdx.x] = sq;
 }
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 loss_finalize_kernel(const float* __restrict__ parts, int n, float inv_count, float* __restrict__ loss) {
   float s = 0.0f;
   for (int i = threadIdx.x; i < n; i += blockDim.x) s += parts[i];
