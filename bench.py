@@ -184,7 +184,9 @@ def run_own(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = wl.vit_b()
+    w = wl.vit_b() if args.blocks == 12 else wl.vit_b(n_blocks=args.blocks, name=f"vit_b_linear_bf16_{args.blocks}blocks")
+    if args.profile:
+        w.mask[:] = 1
     tdt = torch.bfloat16
 
     def to_dev(a):
@@ -212,6 +214,15 @@ def run_own(args):
 
     def step(mask):
         et.et_backward_elastic(stack, dY, mask, None, delta, imp, flags, w.lr, rep, stream=stream)
+
+    if args.profile:
+        # short run for a profiler: forward above, then two full-backprop steps of a reduced stack
+        step(w.mask)
+        step(w.mask)
+        torch.cuda.synchronize()
+        assert et.et_device_status(stack, stream=stream) == et.ET_OK
+        print(json.dumps({"profile_run": w.name, "launches": et.et_launch_count()}))
+        return
 
     def timed(fn, steps, warmup):
         for _ in range(warmup):
@@ -348,6 +359,9 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--blocks", type=int, default=12, help="transformer blocks of the stack (12 = the benchmark workload)")
+    ap.add_argument("--profile", action="store_true",
+                    help="short run for ncu: one forward and two all-selected backward steps, no timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup
     if args.impl == "reference":
