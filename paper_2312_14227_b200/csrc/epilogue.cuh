@@ -72,8 +72,73 @@ struct DgradEpi {
   }
 };
 
+// ---- staged variants for the tensor-core kernel ---------------------------------------------
+// The kernel moves bf16 operand / result chunks through shared memory; combine() sees 32
+// consecutive columns of one row: the accumulator, and per slot the input values (on entry)
+// which it replaces by the output values (on exit).  has_in / has_out tell the kernel which
+// slots to load and store.
+
+// Forward.  slot 0: in = residual a_j (optional), out = a_{l+1}.  slot 1 (SLOTS == 2): out = Z.
+template <int SLOTS>
+struct FwdEpiS {
+  static constexpr int kSlots = SLOTS;
+  bool has_in[2], has_out[2];
+  const bf16* bias;  // [fold * ld]
+  int fold, ld, act;
+
+  __device__ __forceinline__ void combine(int col0, int nv, float (&v)[32], float (&s0)[32], float (&s1)[32]) const {
+    float t[32];
+    for (int s = 0; s < fold; ++s) {
+      load_seg<32>(bias + (size_t)s * ld + col0, nv, t);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] += t[i];
+    }
+    if constexpr (SLOTS == 2) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) s1[i] = v[i];
+    }
+    const bool res = has_in[0];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) s0[i] = act_apply(v[i], act) + (res ? s0[i] : 0.0f);
+  }
+};
+
+// Error-gradient pass.  SLOTS == 2: slot 0: in = skip gradient (optional), out = G_l (optional);
+// slot 1: in = Z_{l-1}, out = dZ_{l-1} = G_l * act'(Z_{l-1}).
+// SLOTS == 1, mul_act == false: in = skip (optional), out = G_l = acc + skip.
+// SLOTS == 1, mul_act == true : in = Z_{l-1}, out = dZ_{l-1} = acc * act'(Z_{l-1}).
+template <int SLOTS>
+struct DgradEpiS {
+  static constexpr int kSlots = SLOTS;
+  bool has_in[2], has_out[2];
+  bool mul_act;
+  int act_prev;
+
+  __device__ __forceinline__ void combine(int, int, float (&v)[32], float (&s0)[32], float (&s1)[32]) const {
+    if constexpr (SLOTS == 1) {
+      if (mul_act) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) s0[i] = v[i] * act_grad(s0[i], act_prev);
+      } else {
+        const bool skip = has_in[0];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) s0[i] = v[i] + (skip ? s0[i] : 0.0f);
+      }
+    } else {
+      const bool skip = has_in[0];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float g = v[i] + (skip ? s0[i] : 0.0f);
+        s0[i] = g;
+        s1[i] = g * act_grad(s1[i], act_prev);
+      }
+    }
+  }
+};
+
 // Weight-gradient partial of one K split: plain fp32 store.
 struct PartialEpi {
+  static constexpr int kSlots = 0;
   float* base;           // [split][rows x ld]
   size_t split_stride;   // rows * ld
   int ld;

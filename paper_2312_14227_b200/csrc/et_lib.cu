@@ -87,9 +87,10 @@ struct LayerRT {
   size_t off_G_out = 0;     // G_{l+1}           (unused for the last layer: that is the caller's dY)
   size_t off_dZ = 0;        // dZ_l              (act != none)
   int split = 1;            // wgrad contraction splits
+  int bn_fwd = 256, bn_dgrad = 256, bn_wgrad = 256;   // tile widths chosen per GEMM
   int imp_count_w = 0, imp_count_b = 0;
-  CUtensorMap map_a, map_W, map_dz;   // bf16 stacks; map_a of layer 0 and map_dz of an
-                                      // activation-free last layer are built per call
+  // bf16 stacks: one TMA descriptor per tensor (the caller's x, y and dY get theirs per call)
+  CUtensorMap map_W, map_aout, map_Gout, map_Z, map_dZ;
 };
 
 }  // namespace
@@ -109,8 +110,9 @@ struct et_stack {
   char* ws = nullptr;
   bool bound = false, forwarded = false;
   const void* x = nullptr;
-  CUtensorMap map_x, map_dy;
+  CUtensorMap map_x, map_y, map_dy;
   const void* map_dy_ptr = nullptr;
+  const void* map_y_ptr = nullptr;
   // optional per-kernel timing
   bool timing = false;
   struct Timed { int cls; cudaEvent_t e0, e1; };
@@ -126,15 +128,23 @@ namespace {
 
 using et::bf16;
 
-int choose_split(int tiles, int kb_total, int sms) {
-  int best = 1;
-  long long best_cost = -1;
-  for (int s = 1; s <= 16 && s <= kb_total; ++s) {
-    const int kbs = ceil_div(kb_total, s);
-    if ((long long)(s - 1) * kbs >= kb_total) continue;        // an empty split
-    const long long waves = ceil_div((long long)tiles * s, sms);
-    const long long cost = waves * (kbs + 6);
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+// Tile width and contraction split of one GEMM: minimise (waves of work units over the SMs) x
+// (k-blocks per unit + fixed per-unit cost) x (tile width), i.e. the time of the slowest SM.
+struct TilePlan { int bn; int split; };
+TilePlan choose_tiles(int rows, int cols, int kb_total, int sms, bool allow_split) {
+  TilePlan best{256, 1};
+  double best_cost = -1.0;
+  const int bns[3] = {256, 192, 128};
+  for (int bn : bns) {
+    const long long tiles = (long long)ceil_div(rows, et::tc::BM) * ceil_div(cols, bn);
+    const int smax = allow_split ? std::min(16, kb_total) : 1;
+    for (int s = 1; s <= smax; ++s) {
+      const int kbs = ceil_div(kb_total, s);
+      if ((long long)(s - 1) * kbs >= kb_total) continue;      // an empty split
+      const long long waves = ceil_div(tiles * s, sms);
+      const double cost = (double)waves * (kbs + 6) * (bn + 32);
+      if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = {bn, s}; }
+    }
   }
   return best;
 }
@@ -174,25 +184,37 @@ template <typename T> const T* dz_src(const et_stack* s, int l, const void* dY) 
   const LayerRT& y = s->ly[l];
   return y.act != ET_ACT_NONE ? (const T*)s->at(y.off_dZ) : grad_act<T>(s, l + 1, dY);
 }
-const CUtensorMap& dz_map(const et_stack* s, int l) {
-  return (l == s->L - 1 && s->ly[l].act == ET_ACT_NONE) ? s->map_dy : s->ly[l].map_dz;
+const CUtensorMap& a_map(const et_stack* s, int l) { return l == 0 ? s->map_x : s->ly[l - 1].map_aout; }   // a_l
+const CUtensorMap& g_map(const et_stack* s, int i) { return i == s->L ? s->map_dy : s->ly[i - 1].map_Gout; }  // G_i
+const CUtensorMap& dz_map(const et_stack* s, int l) {                                                         // dZ_l
+  return s->ly[l].act != ET_ACT_NONE ? s->ly[l].map_dZ : g_map(s, l + 1);
 }
-const CUtensorMap& a_map(const et_stack* s, int l) { return l == 0 ? s->map_x : s->ly[l].map_a; }
 
 // ---- GEMM launches ---------------------------------------------------------------------------
-template <bool A_MN, bool B_MN, class Epi>
-et_status launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::Params& p, const Epi& epi, int sms,
-                    cudaStream_t st) {
-  auto kern = et::tc::gemm_tc_kernel<A_MN, B_MN, Epi>;
+template <int BN, bool A_MN, bool B_MN, class Epi>
+et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em, et::tc::Params p,
+                       const Epi& epi, int sms, cudaStream_t st) {
+  auto kern = et::tc::gemm_tc_kernel<BN, A_MN, B_MN, Epi>;
+  using C = et::tc::Cfg<BN, Epi::kSlots>;
   static bool attr_done = false;
   if (!attr_done) {
-    CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)et::tc::SMEM_BYTES));
+    CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
     attr_done = true;
   }
+  p.tiles_n = ceil_div(p.cols, BN);
   const int units = p.tiles_m * p.tiles_n * p.split;
   const int grid = std::min(units, sms);
-  kern<<<grid, et::tc::THREADS, et::tc::SMEM_BYTES, st>>>(ma, mb, p, epi);
+  kern<<<grid, et::tc::THREADS, C::SMEM_BYTES, st>>>(ma, mb, em, p, epi);
   return after_launch();
+}
+template <bool A_MN, bool B_MN, class Epi>
+et_status launch_tc(int bn, const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em,
+                    const et::tc::Params& p, const Epi& epi, int sms, cudaStream_t st) {
+  if (bn == 128) return launch_tc_bn<128, A_MN, B_MN>(ma, mb, em, p, epi, sms, st);
+  // two staged slots leave too little shared memory for a 256-wide operand ring
+  if (bn == 192 || Epi::kSlots == 2) return launch_tc_bn<192, A_MN, B_MN>(ma, mb, em, p, epi, sms, st);
+  if constexpr (Epi::kSlots < 2) return launch_tc_bn<256, A_MN, B_MN>(ma, mb, em, p, epi, sms, st);
+  return ET_ERR_UNSUPPORTED;
 }
 template <typename T, class Epi>
 et_status launch_simt(const T* A, const T* B, const et::simt::Params& p, const Epi& epi, cudaStream_t st) {
@@ -205,7 +227,7 @@ et::tc::Params tc_params(const et_stack* s, int rows, int cols, int contraction,
   et::tc::Params p;
   p.rows = rows; p.cols = cols;
   p.tiles_m = ceil_div(rows, et::tc::BM);
-  p.tiles_n = ceil_div(cols, et::tc::BN);
+  p.tiles_n = 0;                       // set at launch from the tile width
   p.split = split;
   p.kb_per_seg = ceil_div(contraction, et::tc::BK);
   p.kb_total = p.kb_per_seg * fold;
@@ -220,19 +242,35 @@ template <typename T>
 et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
   TimedLaunch tl(s, ET_K_FORWARD, st);
   const LayerRT& L = s->ly[l];
-  et::FwdEpi<T> epi;
-  epi.bias = (const T*)L.b;
-  epi.fold = L.fold;
-  epi.Z = L.act != ET_ACT_NONE ? (T*)s->at(L.off_Z) : nullptr;
-  epi.act = L.act;
-  epi.resid = L.residual_src >= 0 ? act_in<T>(s, L.residual_src) : nullptr;
-  epi.out = l == s->L - 1 ? (T*)y : (T*)s->at(L.off_a_out);
-  epi.ld = L.Nw;
   if constexpr (is_bf16<T>::value) {
     et::tc::Params p = tc_params(s, (int)s->M, L.Nw, L.K, L.fold, 1);
     p.b_mn_seg_stride = L.Nw;
-    return launch_tc<false, true>(a_map(s, l), L.map_W, p, epi, s->sms, st);
+    et::tc::EpiMaps em;
+    const CUtensorMap& out = l == s->L - 1 ? s->map_y : L.map_aout;
+    em.in[0] = L.residual_src >= 0 ? a_map(s, L.residual_src) : out;
+    em.out[0] = out;
+    em.in[1] = out;
+    em.out[1] = L.act != ET_ACT_NONE ? L.map_Z : out;
+    auto fill = [&](auto& epi) {
+      epi.has_in[0] = L.residual_src >= 0; epi.has_in[1] = false;
+      epi.has_out[0] = true; epi.has_out[1] = L.act != ET_ACT_NONE;
+      epi.bias = (const bf16*)L.b; epi.fold = L.fold; epi.ld = L.Nw; epi.act = L.act;
+    };
+    if (L.act != ET_ACT_NONE) {
+      et::FwdEpiS<2> epi; fill(epi);
+      return launch_tc<false, true>(L.bn_fwd, a_map(s, l), L.map_W, em, p, epi, s->sms, st);
+    }
+    et::FwdEpiS<1> epi; fill(epi);
+    return launch_tc<false, true>(L.bn_fwd, a_map(s, l), L.map_W, em, p, epi, s->sms, st);
   } else {
+    et::FwdEpi<T> epi;
+    epi.bias = (const T*)L.b;
+    epi.fold = L.fold;
+    epi.Z = L.act != ET_ACT_NONE ? (T*)s->at(L.off_Z) : nullptr;
+    epi.act = L.act;
+    epi.resid = L.residual_src >= 0 ? act_in<T>(s, L.residual_src) : nullptr;
+    epi.out = l == s->L - 1 ? (T*)y : (T*)s->at(L.off_a_out);
+    epi.ld = L.Nw;
     et::simt::Params p;
     p.rows = (int)s->M; p.cols = L.Nw; p.kc = L.K; p.segs = L.fold;
     p.sa_i = L.K; p.sa_k = 1;
@@ -247,24 +285,48 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st) {
   TimedLaunch tl(s, ET_K_DGRAD, st);
   const LayerRT& L = s->ly[l];
   const LayerRT& P = s->ly[l - 1];
-  et::DgradEpi<T> epi;
-  epi.skip = L.consumer >= 0 ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
-  epi.act_prev = P.act;
-  epi.ld = L.K;
-  if (P.act == ET_ACT_NONE) {
-    epi.Zprev = nullptr;
-    epi.outG = (T*)s->at(P.off_G_out);
-    epi.outdZ = nullptr;
-  } else {
-    epi.Zprev = (const T*)s->at(P.off_Z);
-    epi.outdZ = (T*)s->at(P.off_dZ);
-    epi.outG = P.residual_src >= 0 ? (T*)s->at(P.off_G_out) : nullptr;
-  }
+  const bool need_skip = L.consumer >= 0;
+  const bool need_act = P.act != ET_ACT_NONE;
+  const bool need_G = !need_act || P.residual_src >= 0;     // G_l itself is read later
   if constexpr (is_bf16<T>::value) {
     et::tc::Params p = tc_params(s, (int)s->M, L.K, L.Nw, L.fold, 1);
     p.b_k_seg_stride = L.Nw;
-    return launch_tc<false, false>(dz_map(s, l), L.map_W, p, epi, s->sms, st);
+    et::tc::EpiMaps em;
+    const CUtensorMap& gout = P.map_Gout;                     // G_l lives in layer l-1's buffer
+    const CUtensorMap& skip = need_skip ? g_map(s, L.consumer + 1) : gout;
+    if (!need_act) {                                          // G_l = acc (+ skip)
+      et::DgradEpiS<1> epi;
+      epi.has_in[0] = need_skip; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
+      epi.mul_act = false; epi.act_prev = P.act;
+      em.in[0] = skip; em.out[0] = gout; em.in[1] = gout; em.out[1] = gout;
+      return launch_tc<false, false>(L.bn_dgrad, dz_map(s, l), L.map_W, em, p, epi, s->sms, st);
+    }
+    if (!need_skip && !need_G) {                              // dZ_{l-1} = acc * act'(Z_{l-1})
+      et::DgradEpiS<1> epi;
+      epi.has_in[0] = true; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
+      epi.mul_act = true; epi.act_prev = P.act;
+      em.in[0] = P.map_Z; em.out[0] = P.map_dZ; em.in[1] = P.map_Z; em.out[1] = P.map_dZ;
+      return launch_tc<false, false>(L.bn_dgrad, dz_map(s, l), L.map_W, em, p, epi, s->sms, st);
+    }
+    et::DgradEpiS<2> epi;                                     // both G_l and dZ_{l-1}
+    epi.has_in[0] = need_skip; epi.has_in[1] = true; epi.has_out[0] = need_G; epi.has_out[1] = true;
+    epi.mul_act = false; epi.act_prev = P.act;
+    em.in[0] = skip; em.out[0] = gout; em.in[1] = P.map_Z; em.out[1] = P.map_dZ;
+    return launch_tc<false, false>(L.bn_dgrad, dz_map(s, l), L.map_W, em, p, epi, s->sms, st);
   } else {
+    et::DgradEpi<T> epi;
+    epi.skip = need_skip ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
+    epi.act_prev = P.act;
+    epi.ld = L.K;
+    if (!need_act) {
+      epi.Zprev = nullptr;
+      epi.outG = (T*)s->at(P.off_G_out);
+      epi.outdZ = nullptr;
+    } else {
+      epi.Zprev = (const T*)s->at(P.off_Z);
+      epi.outdZ = (T*)s->at(P.off_dZ);
+      epi.outG = need_G ? (T*)s->at(P.off_G_out) : nullptr;
+    }
     et::simt::Params p;
     p.rows = (int)s->M; p.cols = L.K; p.kc = L.Nw; p.segs = L.fold;
     p.sa_i = L.Nw; p.sa_k = 1;
@@ -289,7 +351,9 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
       split = L.split;
       et::tc::Params p = tc_params(s, L.K, L.N, (int)s->M, 1, split);
       p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
-      ET_TRY((launch_tc<true, true>(a_map(s, l), dz_map(s, l), p, epi, s->sms, st)));
+      et::tc::EpiMaps em;
+      em.in[0] = em.in[1] = em.out[0] = em.out[1] = L.map_W;          // unused by the direct epilogue
+      ET_TRY((launch_tc<true, true>(L.bn_wgrad, a_map(s, l), dz_map(s, l), em, p, epi, s->sms, st)));
     } else {
       et::simt::Params p;
       p.rows = L.K; p.cols = L.N; p.kc = (int)s->M; p.segs = 1;
@@ -370,7 +434,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
     if (delta != nullptr) CU_TRY(cudaMemsetAsync(importance_dev, 0, sizeof(float) * 2 * L, st));
   } else {
     if constexpr (is_bf16<T>::value) {
-      if (s->ly[L - 1].act == ET_ACT_NONE && s->map_dy_ptr != dY) {
+      if (s->map_dy_ptr != dY) {
         ET_TRY(make_map(&s->map_dy, dY, s->out_width(), s->M));
         s->map_dy_ptr = dY;
       }
@@ -436,6 +500,10 @@ template <typename T>
 et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
   if constexpr (is_bf16<T>::value) {
     if (s->x != x || !s->forwarded) ET_TRY(make_map(&s->map_x, x, s->ly[0].K, s->M));
+    if (s->map_y_ptr != y) {
+      ET_TRY(make_map(&s->map_y, y, s->out_width(), s->M));
+      s->map_y_ptr = y;
+    }
   }
   s->x = x;
   for (int l = 0; l < s->L; ++l) ET_TRY(run_forward_layer<T>(s, l, y, st));
@@ -492,7 +560,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     }
     if (dtype == ET_BF16) {
       if (y.K % 8 || y.N % 8 || y.Nw % 8) { err = ET_ERR_UNSUPPORTED; break; }
-      if (y.fold > 1 && y.Nw % et::tc::BN) { err = ET_ERR_UNSUPPORTED; break; }
+      if (y.fold > 1 && y.Nw % 256) { err = ET_ERR_UNSUPPORTED; break; }
     }
   }
   if (err != ET_OK) { delete s; return err; }
@@ -511,8 +579,22 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (l < L - 1) { y.off_a_out = take(act_bytes); y.off_G_out = take(act_bytes); }
     if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
     if (dtype == ET_BF16) {
-      const int tiles = ceil_div(y.K, et::tc::BM) * ceil_div(y.N, et::tc::BN);
-      y.split = choose_split(tiles, ceil_div(M, et::tc::BK), s->sms);
+      const int kb_n = ceil_div(y.Nw, et::tc::BK) * y.fold;
+      y.bn_fwd = choose_tiles((int)M, y.Nw, ceil_div(y.K, et::tc::BK) * y.fold, s->sms, false).bn;
+      y.bn_dgrad = choose_tiles((int)M, y.K, kb_n, s->sms, false).bn;
+      TilePlan w = choose_tiles(y.K, y.N, ceil_div(M, et::tc::BK), s->sms, true);
+      if (y.fold > 1 && y.Nw % w.bn != 0) {                     // a folded wgrad tile must not straddle slices
+        w.bn = 256;
+        TilePlan best{256, 1}; double bc = -1;
+        for (int sp = 1; sp <= 16; ++sp) {
+          const int kbt = ceil_div(M, et::tc::BK), kbs = ceil_div(kbt, sp);
+          if (sp > kbt || (long long)(sp - 1) * kbs >= kbt) continue;
+          const double c = (double)ceil_div((long long)ceil_div(y.K, et::tc::BM) * ceil_div(y.N, 256) * sp, s->sms) * (kbs + 6);
+          if (bc < 0 || c < bc) { bc = c; best = {256, sp}; }
+        }
+        w = best;
+      }
+      y.bn_wgrad = w.bn; y.split = w.split;
     }
     max_partial = std::max(max_partial, (size_t)y.split * y.K * y.N * sizeof(float));
     max_biaspart = std::max(max_biaspart, (size_t)chunks * y.Nw * sizeof(float));
@@ -563,9 +645,14 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
     for (int l = 0; l < s->L; ++l) {
       LayerRT& y = s->ly[l];
       ET_TRY(make_map(&y.map_W, y.W, y.N, y.K));
-      if (l >= 1) ET_TRY(make_map(&y.map_a, s->at(s->ly[l - 1].off_a_out), y.K, s->M));
-      if (y.act != ET_ACT_NONE) ET_TRY(make_map(&y.map_dz, s->at(y.off_dZ), y.Nw, s->M));
-      else if (l < s->L - 1) ET_TRY(make_map(&y.map_dz, s->at(y.off_G_out), y.Nw, s->M));
+      if (l < s->L - 1) {
+        ET_TRY(make_map(&y.map_aout, s->at(y.off_a_out), y.Nw, s->M));
+        ET_TRY(make_map(&y.map_Gout, s->at(y.off_G_out), y.Nw, s->M));
+      }
+      if (y.act != ET_ACT_NONE) {
+        ET_TRY(make_map(&y.map_Z, s->at(y.off_Z), y.Nw, s->M));
+        ET_TRY(make_map(&y.map_dZ, s->at(y.off_dZ), y.Nw, s->M));
+      }
     }
   }
   CU_TRY(cudaMemsetAsync(s->at(s->off_status), 0, 256, st));
@@ -575,6 +662,7 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   s->bound = true;
   s->forwarded = false;
   s->map_dy_ptr = nullptr;
+  s->map_y_ptr = nullptr;
   s->x = nullptr;
   return ET_OK;
 }

@@ -7,6 +7,13 @@
 //   forward  Z  = a  * W      A = a   K-major,   B = W   MN-major
 //   dgrad    dX = dZ * W^T    A = dZ  K-major,   B = W   K-major
 //   wgrad    dW = a^T * dZ    A = a   MN-major,  B = dZ  MN-major   (contraction over tokens)
+//
+// Epilogues that read or write bf16 tensors (forward, dgrad) move them with TMA through
+// 128-byte-swizzled shared-memory chunks of 128 rows x 64 columns: a loader warp prefetches the
+// operand chunks (skip gradient, pre-activation, residual) while the main loop of the tile is
+// still running, the four epilogue warps combine them with the accumulator in place, and one
+// thread stores the chunk back with TMA.  Global traffic is therefore fully coalesced although
+// each epilogue thread owns one accumulator row.
 #pragma once
 
 #include <cuda.h>
@@ -18,18 +25,30 @@ namespace et {
 namespace tc {
 
 constexpr int BM = 128;          // output rows per tile  (UMMA M)
-constexpr int BN = 256;          // output cols per tile  (UMMA N)
 constexpr int BK = 64;           // contraction elements per stage = one 128-byte swizzle row
 constexpr int UK = 16;           // contraction elements per tcgen05.mma (bf16)
-constexpr int STAGES = 4;
-constexpr int ACC_STAGES = 2;    // 2 x 256 fp32 columns = all 512 TMEM columns
-constexpr int THREADS = 192;     // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-5: epilogue
+constexpr int ACC_STAGES = 2;    // accumulator stages at TMEM columns 0 and 256
+constexpr int ACC_STRIDE = 256;
+constexpr int THREADS = 224;     // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-5: epilogue, warp 6: epilogue loader
+constexpr uint32_t CHUNK_BYTES = 64 * BK * 2;       // one TMA box: 64 rows of 128 B
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
-constexpr uint32_t B_STAGE_BYTES = BN * BK * 2;
-constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-constexpr uint32_t CHUNK_BYTES = 64 * BK * 2;   // one TMA box: 64 rows of 128 B
-constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t EPI_CHUNK_BYTES = BM * 64 * 2;   // 128 rows x 64 bf16 columns
+constexpr int EPI_SETS = 3;      // staged-epilogue buffer sets: one being combined, one being stored, one being loaded
 constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t SMEM_LIMIT = 227 * 1024;
+constexpr uint32_t SMEM_SLACK = 1024 /*alignment*/ + 256 /*barriers*/;
+
+template <int BN, int SLOTS>
+struct Cfg {
+  static constexpr uint32_t B_STAGE_BYTES = BN * BK * 2;
+  static constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+  static constexpr uint32_t EPI_BYTES = (uint32_t)EPI_SETS * SLOTS * EPI_CHUNK_BYTES;
+  static constexpr int STAGES_FIT = (int)((SMEM_LIMIT - SMEM_SLACK - EPI_BYTES) / STAGE_BYTES);
+  static constexpr int STAGES = STAGES_FIT > 6 ? 6 : STAGES_FIT;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + SMEM_SLACK;
+  static_assert(STAGES >= 3, "too few pipeline stages");
+  static_assert(BN % 64 == 0 && BN >= 64 && BN <= 256, "tile width");
+};
 
 // Bounded waits: a wait that has not succeeded after this many polls gives up, records
 // where, and the CTA winds down.  Each poll may block inside try_wait for a while, so the
@@ -42,6 +61,7 @@ enum StatusCode : uint32_t {
   kTimeoutMma = 2,
   kTimeoutEpilogue = 3,
   kTimeoutDrain = 4,
+  kTimeoutEpiLoader = 5,
 };
 
 struct Params {
@@ -55,6 +75,13 @@ struct Params {
   int b_mn_seg_stride;       // added to B's mn coordinate per segment  (forward through a fold)
   int b_mn_wrap;             // B's mn coordinate taken modulo this, 0 = off (wgrad through a fold)
   uint32_t* status;          // device word, 0 = ok; first failure wins
+};
+
+// Tensor maps of the staged epilogue: per slot one optional input and one optional output,
+// all [rows x cols] bf16 row-major with the output's shape.
+struct EpiMaps {
+  CUtensorMap in[2];
+  CUtensorMap out[2];
 };
 
 // --------------------------------------------------------------------------- PTX wrappers
@@ -98,6 +125,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -146,7 +186,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lead_bytes
 
 // Instruction descriptor for kind::f16: fp32 accumulate (bits 4-5 = 1), bf16 A and B
 // (bits 7-9, 10-12 = 1), operand major-ness (bits 15, 16), N/8 (bits 17-22), M/16 (bits 24-28).
-template <bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN>
 __host__ __device__ constexpr uint32_t make_idesc() {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
          ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -156,22 +196,64 @@ template <class Epi>
 __device__ __forceinline__ void epi_set_split(Epi&, int) {}
 __device__ __forceinline__ void epi_set_split(PartialEpi& e, int s) { e.split = s; }
 
+// 16-byte piece `piece` (0..7) of row `row` (0..127) inside a staged 128 x 64 bf16 chunk.
+__device__ __forceinline__ uint32_t epi_chunk_off(int row, int piece) {
+  return (uint32_t)((row >> 6) * CHUNK_BYTES + (row & 63) * 128 + ((piece ^ (row & 7)) << 4));
+}
+__device__ __forceinline__ void lds_row32(const uint8_t* chunk, int row, int half, float (&v)[32]) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint4 q = *reinterpret_cast<const uint4*>(chunk + epi_chunk_off(row, half * 4 + j));
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[j * 8 + 2 * i] = __uint_as_float(w[i] << 16);
+      v[j * 8 + 2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+}
+__device__ __forceinline__ void sts_row32(uint8_t* chunk, int row, int half, const float (&v)[32]) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint4 q;
+    q.x = pack_bf16x2(v[j * 8 + 0], v[j * 8 + 1]);
+    q.y = pack_bf16x2(v[j * 8 + 2], v[j * 8 + 3]);
+    q.z = pack_bf16x2(v[j * 8 + 4], v[j * 8 + 5]);
+    q.w = pack_bf16x2(v[j * 8 + 6], v[j * 8 + 7]);
+    *reinterpret_cast<uint4*>(chunk + epi_chunk_off(row, half * 4 + j)) = q;
+  }
+}
+
 // --------------------------------------------------------------------------- the kernel
-template <bool A_MN, bool B_MN, class Epi>
+// Epi::kSlots == 0: direct epilogue, Epi::operator()<32>(row, col0, n, acc) stores by itself.
+// Epi::kSlots  > 0: staged epilogue, Epi::combine(col0, acc, s0, s1) turns the accumulator and
+//                   the slots' input values into the slots' output values, in place; the flags
+//                   Epi::has_in[s] / has_out[s] say which slots carry an input / an output.
+template <int BN, bool A_MN, bool B_MN, class Epi>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const Params p, const Epi epi_in) {
+               const __grid_constant__ EpiMaps emaps, const Params p, const Epi epi_in) {
+  constexpr int SLOTS = Epi::kSlots;
+  using C = Cfg<BN, SLOTS>;
+  constexpr int STAGES = C::STAGES;
+  constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES;
+  constexpr int NCHUNK = BN / 64;
+
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzle atoms need 1024-B alignment
   uint8_t* gen_base = smem_raw + (base - raw);
-  const uint32_t bars = base + STAGES * STAGE_BYTES;
-  // barrier slots (8 B each): full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
+  const uint32_t epi_base = base + STAGES * STAGE_BYTES;        // [2 buffer sets][SLOTS][EPI_CHUNK_BYTES]
+  const uint32_t bars = epi_base + C::EPI_BYTES;
+  // barrier slots (8 B each)
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto acc_full_bar = [&](int s) { return bars + 8u * (2 * STAGES + s); };
-  auto acc_empty_bar = [&](int s) { return bars + 8u * (2 * STAGES + ACC_STAGES + s); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + STAGES * STAGE_BYTES + 128);
+  auto acc_empty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 2 + s); };
+  auto in_full_bar = [&](int s) { return bars + 8u * (2 * STAGES + 4 + s); };
+  auto in_empty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 4 + EPI_SETS + s); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(
+      gen_base + STAGES * STAGE_BYTES + C::EPI_BYTES + 8 * (2 * STAGES + 4 + 2 * EPI_SETS));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5;
@@ -179,10 +261,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int s = 0; s < ACC_STAGES; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), 4); }
+    for (int s = 0; s < EPI_SETS; ++s) { mbar_init(in_full_bar(s), 1); mbar_init(in_empty_bar(s), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    fence_async_smem();
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -251,7 +334,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc<A_MN, B_MN>();
+      constexpr uint32_t idesc = make_idesc<BN, A_MN, B_MN>();
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -264,7 +347,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, kTimeoutMma);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_STRIDE);
         for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, kTimeoutMma);
           if (!ok) break;
@@ -286,12 +369,67 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
       }
     }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ epilogue operand loader
+    if constexpr (SLOTS > 0) {
+      if (lane == 0) {
+        uint32_t tx = 0;
+#pragma unroll
+        for (int s = 0; s < SLOTS; ++s) tx += epi_in.has_in[s] ? EPI_CHUNK_BYTES : 0u;
+        int bs = 0;                                   // buffer set of the next chunk
+        uint32_t use = 0;                             // how often that set has been used before
+        uint32_t fills[EPI_SETS];
+#pragma unroll
+        for (int i = 0; i < EPI_SETS; ++i) fills[i] = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+          const int t = u % tiles;
+          const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+          for (int c = 0; c < NCHUNK; ++c) {
+            const int col0 = n0 + c * 64;
+            if (col0 >= p.cols) break;
+            ok = mbar_wait(in_empty_bar(bs), (use & 1u) ^ 1u, abort_flag, p.status, kTimeoutEpiLoader);
+            if (!ok) break;
+            const uint32_t bar = in_full_bar(bs);
+            if (tx > 0) {
+              mbar_expect_tx(bar, tx);
+#pragma unroll
+              for (int s = 0; s < SLOTS; ++s) {
+                if (!epi_in.has_in[s]) continue;
+                const uint32_t dst = epi_base + (bs * SLOTS + s) * EPI_CHUNK_BYTES;
+                tma_load_2d(dst, &emaps.in[s], bar, col0, m0);
+                tma_load_2d(dst + CHUNK_BYTES, &emaps.in[s], bar, col0, m0 + 64);
+              }
+              ++fills[bs];
+            } else {
+              mbar_arrive(bar);                       // nothing to fetch: just pass the buffer on
+            }
+            if (++bs == EPI_SETS) { bs = 0; ++use; }
+          }
+        }
+        if (!ok && tx > 0) {
+#pragma unroll
+          for (int b = 0; b < EPI_SETS; ++b) {
+            if (fills[b] == 0) continue;
+            const uint32_t par = (fills[b] - 1u) & 1u;
+            bool landed = false;
+            for (uint32_t it = 0; it < (1u << 20) && !landed; ++it) landed = mbar_try_wait(in_full_bar(b), par);
+            if (!landed) atomicCAS(p.status, 0u, (uint32_t)kTimeoutDrain);
+          }
+        }
+      }
+    }
   } else {
-    // ------------------------------------------------------------------ epilogue (4 warps)
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
     Epi epi = epi_in;
     const int quad = warp & 3;                      // TMEM lanes this warp may read: 32*quad ...
+    const int trow = quad * 32 + lane;              // row inside the tile
+    const bool leader = (warp == 2 && lane == 0);   // issues the TMA stores
     int acc = 0;
     uint32_t acc_phase = 0;
+    int bs = 0;                                     // staged path: buffer set of the next chunk,
+    uint32_t use = 0;                               // how often it has been used before,
+    bool first_chunk = true;                        // and whether any chunk has been stored yet
     bool ok = true;
     for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
       const int sp = u / tiles, t = u - sp * tiles;
@@ -300,20 +438,70 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, p.status, kTimeoutEpilogue);
       if (!ok) break;
       tc_fence_after();
-      const int row = m0 + quad * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * ACC_STRIDE);
+      if constexpr (SLOTS == 0) {
+        const int row = m0 + trow;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        float v[32];
-        tmem_ld32(taddr + c * 32, v);               // warp-collective: every lane takes part
-        const int col0 = n0 + c * 32;
-        const int n = p.cols - col0;
-        if (row < p.rows && n > 0) epi.template operator()<32>(row, col0, n, v);
+        for (int c = 0; c < BN / 32; ++c) {
+          float v[32];
+          tmem_ld32(taddr + c * 32, v);             // warp-collective: every lane takes part
+          const int col0 = n0 + c * 32;
+          const int nv = p.cols - col0;
+          if (row < p.rows && nv > 0) epi.template operator()<32>(row, col0, nv, v);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+      } else {
+        int nch = 0;
+#pragma unroll
+        for (int c = 0; c < NCHUNK; ++c) nch += (n0 + c * 64 < p.cols) ? 1 : 0;
+#pragma unroll 1
+        for (int c = 0; c < nch; ++c) {
+          const int col0 = n0 + c * 64;
+          ok = mbar_wait(in_full_bar(bs), use & 1u, abort_flag, p.status, kTimeoutEpilogue);
+          if (!ok) break;
+          uint8_t* buf0 = gen_base + STAGES * STAGE_BYTES + (bs * SLOTS + 0) * EPI_CHUNK_BYTES;
+          uint8_t* buf1 = gen_base + STAGES * STAGE_BYTES + (bs * SLOTS + (SLOTS - 1)) * EPI_CHUNK_BYTES;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float v[32], s0[32], s1[32];
+            tmem_ld32(taddr + c * 64 + h * 32, v);
+            if (c == nch - 1 && h == 1) {           // last read of this accumulator: hand it back
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+            }
+            if (epi.has_in[0]) lds_row32(buf0, trow, h, s0);
+            if (SLOTS > 1 && epi.has_in[SLOTS - 1]) lds_row32(buf1, trow, h, s1);
+            epi.combine(col0 + h * 32, p.cols - (col0 + h * 32), v, s0, s1);
+            if (epi.has_out[0]) sts_row32(buf0, trow, h, s0);
+            if (SLOTS > 1 && epi.has_out[SLOTS - 1]) sts_row32(buf1, trow, h, s1);
+          }
+          fence_async_smem();                       // generic-proxy writes -> visible to the TMA engine
+          epi_bar_sync();
+          if (leader) {
+#pragma unroll
+            for (int s = 0; s < SLOTS; ++s) {
+              if (!epi.has_out[s]) continue;
+              const uint32_t src = epi_base + (bs * SLOTS + s) * EPI_CHUNK_BYTES;
+              tma_store_2d(&emaps.out[s], src, col0, m0);
+              if (m0 + 64 < p.rows) tma_store_2d(&emaps.out[s], src + CHUNK_BYTES, col0, m0 + 64);
+            }
+            tma_store_commit();
+            if (!first_chunk) {
+              tma_store_wait_read<1>();             // the previous chunk's stores have read their buffers
+              mbar_arrive(in_empty_bar(bs == 0 ? EPI_SETS - 1 : bs - 1));
+            }
+          }
+          first_chunk = false;
+          if (++bs == EPI_SETS) { bs = 0; ++use; }
+        }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar(acc));
       if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+    }
+    if constexpr (SLOTS > 0) {
+      if (leader) tma_store_wait_all();             // shared memory must outlive the last store's reads
     }
   }
 
