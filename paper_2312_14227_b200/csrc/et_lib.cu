@@ -2,6 +2,8 @@
 // from the selection mask, kernel launches.  No device memory is allocated here.
 #include <algorithm>
 #include <atomic>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <type_traits>
@@ -59,13 +61,14 @@ EncodeTiledFn get_encode_fn() {
   }
   return fn;
 }
-// Row-major bf16 matrix [outer x inner], box 64 x 64, 128-byte swizzle, zero fill outside.
-et_status make_map(CUtensorMap* m, const void* ptr, int inner, long long outer) {
+// Row-major bf16 matrix [outer x inner]: box of 64 columns x box_rows rows, 128-byte swizzle,
+// zero fill outside.
+et_status make_map(CUtensorMap* m, const void* ptr, int inner, long long outer, int box_rows = 64) {
   EncodeTiledFn fn = get_encode_fn();
   if (fn == nullptr) return ET_ERR_CUDA;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
   cuuint64_t strides[1] = {(cuuint64_t)inner * 2};
-  cuuint32_t box[2] = {64, 64};
+  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -75,6 +78,47 @@ et_status make_map(CUtensorMap* m, const void* ptr, int inner, long long outer) 
     return ET_ERR_CUDA;
   }
   return ET_OK;
+}
+// The same matrix seen as [inner/64 chunks][outer][64]: one box = `depth` chunks of 64 columns x
+// 64 rows, which is how an MN-major operand tile lies in shared memory.  inner % 64 == 0.
+et_status make_map3(CUtensorMap* m, const void* ptr, int inner, long long outer, int depth) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return ET_ERR_CUDA;
+  cuuint64_t dims[3] = {64, (cuuint64_t)outer, (cuuint64_t)(inner / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)inner * 2, 128};
+  cuuint32_t box[3] = {64, 64, (cuuint32_t)depth};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda = (int)cudaErrorInvalidValue;
+    return ET_ERR_CUDA;
+  }
+  return ET_OK;
+}
+// All the views of one bf16 activation / gradient / weight matrix that the GEMMs use.
+struct TMaps {
+  CUtensorMap b64;     // 64 x 64 boxes: MN-major operand fetched chunk by chunk
+  CUtensorMap b128;    // 64 columns x 128 rows: K-major A tile, epilogue chunks
+  CUtensorMap c3[2];   // 3-D, depth 2 and 4: MN-major operand tile in one copy (width % 64 == 0)
+  bool has3 = false;
+};
+et_status make_tmaps(TMaps* t, const void* ptr, int inner, long long outer) {
+  ET_TRY(make_map(&t->b64, ptr, inner, outer, 64));
+  ET_TRY(make_map(&t->b128, ptr, inner, outer, 128));
+  t->has3 = inner % 64 == 0;
+  if (t->has3) {
+    ET_TRY(make_map3(&t->c3[0], ptr, inner, outer, 2));
+    ET_TRY(make_map3(&t->c3[1], ptr, inner, outer, 4));
+  }
+  return ET_OK;
+}
+// MN-major operand of `chunks` 64-wide chunks: the 3-D view if there is one, else the 64 x 64 view.
+const CUtensorMap& mn_map(const TMaps& t, int chunks, int* use3d) {
+  if (t.has3 && (chunks == 2 || chunks == 4)) { *use3d = 1; return t.c3[chunks == 2 ? 0 : 1]; }
+  *use3d = 0;
+  return t.b64;
 }
 
 struct LayerRT {
@@ -88,9 +132,11 @@ struct LayerRT {
   size_t off_dZ = 0;        // dZ_l              (act != none)
   int split = 1;            // wgrad contraction splits
   int bn_fwd = 256, bn_dgrad = 256, bn_wgrad = 256;   // tile widths chosen per GEMM
+  bool pair_fwd = false, pair_dgrad = false, pair_wgrad = false;   // CTA-pair (cta_group::2) tiles
   int imp_count_w = 0, imp_count_b = 0;
   // bf16 stacks: one TMA descriptor per tensor (the caller's x, y and dY get theirs per call)
-  CUtensorMap map_W, map_aout, map_Gout, map_Z, map_dZ;
+  TMaps map_W, map_aout, map_Gout, map_Z, map_dZ;
+  CUtensorMap map_Wd;       // W as the K-major B of the dgrad GEMM: one box = the CTA's whole B tile
 };
 
 }  // namespace
@@ -110,7 +156,7 @@ struct et_stack {
   char* ws = nullptr;
   bool bound = false, forwarded = false;
   const void* x = nullptr;
-  CUtensorMap map_x, map_y, map_dy;
+  TMaps map_x, map_y, map_dy;
   const void* map_dy_ptr = nullptr;
   const void* map_y_ptr = nullptr;
   // optional per-kernel timing
@@ -128,22 +174,35 @@ namespace {
 
 using et::bf16;
 
-// Tile width and contraction split of one GEMM: minimise (waves of work units over the SMs) x
-// (k-blocks per unit + fixed per-unit cost) x (tile width), i.e. the time of the slowest SM.
-struct TilePlan { int bn; int split; };
-TilePlan choose_tiles(int rows, int cols, int kb_total, int sms, bool allow_split) {
-  TilePlan best{256, 1};
+// Tile shape and contraction split of one GEMM.  Model: an SM spends, per 64-deep k-block of
+// its tile, the larger of the tensor-pipe time and the time to pull the operands from L2
+// (about 10.5 TB/s over all SMs, measured with this kernel); a unit costs (k-blocks + a fixed
+// prologue/epilogue allowance) of those; the GEMM takes as many unit times as the busiest SM
+// gets units.  A CTA pair (cta_group::2) loads half of B per CTA and so moves fewer L2 bytes per
+// flop; a 192-wide pair tile needs 32-row B boxes and therefore a K-major B (dgrad only).
+struct TilePlan { int bn; int split; bool pair; };
+TilePlan choose_tiles(int rows, int cols, int kb_total, int sms, bool allow_split, bool b_k_major, int n_multiple) {
+  TilePlan best{256, 1, false};
   double best_cost = -1.0;
-  const int bns[3] = {256, 192, 128};
-  for (int bn : bns) {
-    const long long tiles = (long long)ceil_div(rows, et::tc::BM) * ceil_div(cols, bn);
-    const int smax = allow_split ? std::min(16, kb_total) : 1;
-    for (int s = 1; s <= smax; ++s) {
-      const int kbs = ceil_div(kb_total, s);
-      if ((long long)(s - 1) * kbs >= kb_total) continue;      // an empty split
-      const long long waves = ceil_div(tiles * s, sms);
-      const double cost = (double)waves * (kbs + 6) * (bn + 32);
-      if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = {bn, s}; }
+  const double sm_flops = 10.5e12, sm_l2_bytes = 10.5e12 / 148.0;
+  for (int pair = 0; pair < 2; ++pair) {
+    for (int bn : {256, 192, 128}) {
+      if (pair && bn == 192 && !b_k_major) continue;
+      if (n_multiple > 0 && n_multiple % bn != 0) continue;          // a folded wgrad tile must not straddle slices
+      const int tile_m = pair ? 256 : 128;
+      const long long tiles = (long long)ceil_div(rows, tile_m) * ceil_div(cols, bn);
+      const int workers = pair ? sms / 2 : sms;
+      const double flops = 2.0 * 128 * bn * 64;                      // per CTA per k-block
+      const double bytes = 128.0 * 128 + (pair ? bn / 2 : bn) * 128.0;
+      const double kb_time = std::max(flops / sm_flops, bytes / sm_l2_bytes);
+      const int smax = allow_split ? std::min(16, kb_total) : 1;
+      for (int sp = 1; sp <= smax; ++sp) {
+        const int kbs = ceil_div(kb_total, sp);
+        if ((long long)(sp - 1) * kbs >= kb_total) continue;         // an empty split
+        const long long waves = ceil_div(tiles * sp, workers);
+        const double cost = (double)waves * (kbs + 6) * kb_time;
+        if (best_cost < 0 || cost < best_cost * 0.999) { best_cost = cost; best = {bn, sp, pair != 0}; }
+      }
     }
   }
   return best;
@@ -184,36 +243,62 @@ template <typename T> const T* dz_src(const et_stack* s, int l, const void* dY) 
   const LayerRT& y = s->ly[l];
   return y.act != ET_ACT_NONE ? (const T*)s->at(y.off_dZ) : grad_act<T>(s, l + 1, dY);
 }
-const CUtensorMap& a_map(const et_stack* s, int l) { return l == 0 ? s->map_x : s->ly[l - 1].map_aout; }   // a_l
-const CUtensorMap& g_map(const et_stack* s, int i) { return i == s->L ? s->map_dy : s->ly[i - 1].map_Gout; }  // G_i
-const CUtensorMap& dz_map(const et_stack* s, int l) {                                                         // dZ_l
+const TMaps& a_map(const et_stack* s, int l) { return l == 0 ? s->map_x : s->ly[l - 1].map_aout; }   // a_l
+const TMaps& g_map(const et_stack* s, int i) { return i == s->L ? s->map_dy : s->ly[i - 1].map_Gout; }  // G_i
+const TMaps& dz_map(const et_stack* s, int l) {                                                         // dZ_l
   return s->ly[l].act != ET_ACT_NONE ? s->ly[l].map_dZ : g_map(s, l + 1);
 }
 
 // ---- GEMM launches ---------------------------------------------------------------------------
-template <int BN, bool A_MN, bool B_MN, class Epi>
+template <int BN, bool A_MN, bool B_MN, bool PAIR, class Epi>
 et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em, et::tc::Params p,
                        const Epi& epi, int sms, cudaStream_t st) {
-  auto kern = et::tc::gemm_tc_kernel<BN, A_MN, B_MN, Epi>;
-  using C = et::tc::Cfg<BN, Epi::kSlots>;
+  auto kern = et::tc::gemm_tc_kernel<BN, A_MN, B_MN, Epi, PAIR>;
+  using C = et::tc::Cfg<BN, Epi::kSlots, PAIR>;
   static bool attr_done = false;
+  static int max_clusters = 0;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  cfg.blockDim = dim3(et::tc::THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = st;
+  if (PAIR) {
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+  }
   if (!attr_done) {
     CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
+    if (PAIR) {
+      cfg.gridDim = dim3(sms & ~1);
+      if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) != cudaSuccess || max_clusters < 1) {
+        (void)cudaGetLastError();
+        max_clusters = sms / 2;
+      }
+    }
     attr_done = true;
   }
+  p.tiles_m = ceil_div(p.rows, PAIR ? 2 * et::tc::BM : et::tc::BM);
   p.tiles_n = ceil_div(p.cols, BN);
   const int units = p.tiles_m * p.tiles_n * p.split;
-  const int grid = std::min(units, sms);
-  kern<<<grid, et::tc::THREADS, C::SMEM_BYTES, st>>>(ma, mb, em, p, epi);
+  cfg.gridDim = PAIR ? dim3(2 * std::min(units, max_clusters)) : dim3(std::min(units, sms));
+  CU_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, em, p, epi));
   return after_launch();
 }
 template <bool A_MN, bool B_MN, class Epi>
-et_status launch_tc(int bn, const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em,
+et_status launch_tc(int bn, bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em,
                     const et::tc::Params& p, const Epi& epi, int sms, cudaStream_t st) {
-  if (bn == 128) return launch_tc_bn<128, A_MN, B_MN>(ma, mb, em, p, epi, sms, st);
-  // two staged slots leave too little shared memory for a 256-wide operand ring
-  if (bn == 192 || Epi::kSlots == 2) return launch_tc_bn<192, A_MN, B_MN>(ma, mb, em, p, epi, sms, st);
-  if constexpr (Epi::kSlots < 2) return launch_tc_bn<256, A_MN, B_MN>(ma, mb, em, p, epi, sms, st);
+  if (pair) {
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st);
+    if constexpr (!B_MN) {
+      if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st);
+    }
+    return launch_tc_bn<256, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st);
+  }
+  if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+  // two staged slots leave too little shared memory for a 256-wide single-CTA operand ring
+  if (bn == 192 || Epi::kSlots == 2) return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+  if constexpr (Epi::kSlots < 2) return launch_tc_bn<256, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
   return ET_ERR_UNSUPPORTED;
 }
 template <typename T, class Epi>
@@ -226,13 +311,13 @@ et_status launch_simt(const T* A, const T* B, const et::simt::Params& p, const E
 et::tc::Params tc_params(const et_stack* s, int rows, int cols, int contraction, int fold, int split) {
   et::tc::Params p;
   p.rows = rows; p.cols = cols;
-  p.tiles_m = ceil_div(rows, et::tc::BM);
-  p.tiles_n = 0;                       // set at launch from the tile width
+  p.tiles_m = 0; p.tiles_n = 0;        // set at launch from the tile shape
   p.split = split;
   p.kb_per_seg = ceil_div(contraction, et::tc::BK);
   p.kb_total = p.kb_per_seg * fold;
   p.kb_per_split = ceil_div(p.kb_total, split);
   p.b_k_seg_stride = 0; p.b_mn_seg_stride = 0; p.b_mn_wrap = 0;
+  p.a_3d = 0; p.b_3d = 0;
   p.status = (uint32_t*)s->at(s->off_status);
   return p;
 }
@@ -246,11 +331,13 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
     et::tc::Params p = tc_params(s, (int)s->M, L.Nw, L.K, L.fold, 1);
     p.b_mn_seg_stride = L.Nw;
     et::tc::EpiMaps em;
-    const CUtensorMap& out = l == s->L - 1 ? s->map_y : L.map_aout;
-    em.in[0] = L.residual_src >= 0 ? a_map(s, L.residual_src) : out;
+    const CUtensorMap& out = (l == s->L - 1 ? s->map_y : L.map_aout).b128;
+    em.in[0] = L.residual_src >= 0 ? a_map(s, L.residual_src).b128 : out;
     em.out[0] = out;
     em.in[1] = out;
-    em.out[1] = L.act != ET_ACT_NONE ? L.map_Z : out;
+    em.out[1] = L.act != ET_ACT_NONE ? L.map_Z.b128 : out;
+    const int bnh = L.pair_fwd ? L.bn_fwd / 2 : L.bn_fwd;
+    const CUtensorMap& wmap = mn_map(L.map_W, bnh / 64, &p.b_3d);
     auto fill = [&](auto& epi) {
       epi.has_in[0] = L.residual_src >= 0; epi.has_in[1] = false;
       epi.has_out[0] = true; epi.has_out[1] = L.act != ET_ACT_NONE;
@@ -258,10 +345,10 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
     };
     if (L.act != ET_ACT_NONE) {
       et::FwdEpiS<2> epi; fill(epi);
-      return launch_tc<false, true>(L.bn_fwd, a_map(s, l), L.map_W, em, p, epi, s->sms, st);
+      return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st);
     }
     et::FwdEpiS<1> epi; fill(epi);
-    return launch_tc<false, true>(L.bn_fwd, a_map(s, l), L.map_W, em, p, epi, s->sms, st);
+    return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st);
   } else {
     et::FwdEpi<T> epi;
     epi.bias = (const T*)L.b;
@@ -292,27 +379,30 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st) {
     et::tc::Params p = tc_params(s, (int)s->M, L.K, L.Nw, L.fold, 1);
     p.b_k_seg_stride = L.Nw;
     et::tc::EpiMaps em;
-    const CUtensorMap& gout = P.map_Gout;                     // G_l lives in layer l-1's buffer
-    const CUtensorMap& skip = need_skip ? g_map(s, L.consumer + 1) : gout;
+    const CUtensorMap& gout = P.map_Gout.b128;                // G_l lives in layer l-1's buffer
+    const CUtensorMap& wmap = L.map_Wd;
+    const CUtensorMap& skip = need_skip ? g_map(s, L.consumer + 1).b128 : gout;
+    const CUtensorMap& zmap = P.map_Z.b128;
+    const CUtensorMap& dzout = P.map_dZ.b128;
     if (!need_act) {                                          // G_l = acc (+ skip)
       et::DgradEpiS<1> epi;
       epi.has_in[0] = need_skip; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = false; epi.act_prev = P.act;
       em.in[0] = skip; em.out[0] = gout; em.in[1] = gout; em.out[1] = gout;
-      return launch_tc<false, false>(L.bn_dgrad, dz_map(s, l), L.map_W, em, p, epi, s->sms, st);
+      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
     }
     if (!need_skip && !need_G) {                              // dZ_{l-1} = acc * act'(Z_{l-1})
       et::DgradEpiS<1> epi;
       epi.has_in[0] = true; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = true; epi.act_prev = P.act;
-      em.in[0] = P.map_Z; em.out[0] = P.map_dZ; em.in[1] = P.map_Z; em.out[1] = P.map_dZ;
-      return launch_tc<false, false>(L.bn_dgrad, dz_map(s, l), L.map_W, em, p, epi, s->sms, st);
+      em.in[0] = zmap; em.out[0] = dzout; em.in[1] = zmap; em.out[1] = dzout;
+      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
     }
     et::DgradEpiS<2> epi;                                     // both G_l and dZ_{l-1}
     epi.has_in[0] = need_skip; epi.has_in[1] = true; epi.has_out[0] = need_G; epi.has_out[1] = true;
     epi.mul_act = false; epi.act_prev = P.act;
-    em.in[0] = skip; em.out[0] = gout; em.in[1] = P.map_Z; em.out[1] = P.map_dZ;
-    return launch_tc<false, false>(L.bn_dgrad, dz_map(s, l), L.map_W, em, p, epi, s->sms, st);
+    em.in[0] = skip; em.out[0] = gout; em.in[1] = zmap; em.out[1] = dzout;
+    return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
   } else {
     et::DgradEpi<T> epi;
     epi.skip = need_skip ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
@@ -352,8 +442,11 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
       et::tc::Params p = tc_params(s, L.K, L.N, (int)s->M, 1, split);
       p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
       et::tc::EpiMaps em;
-      em.in[0] = em.in[1] = em.out[0] = em.out[1] = L.map_W;          // unused by the direct epilogue
-      ET_TRY((launch_tc<true, true>(L.bn_wgrad, a_map(s, l), dz_map(s, l), em, p, epi, s->sms, st)));
+      em.in[0] = em.in[1] = em.out[0] = em.out[1] = L.map_W.b64;      // unused by the direct epilogue
+      const int bnh = L.pair_wgrad ? L.bn_wgrad / 2 : L.bn_wgrad;
+      const CUtensorMap& amap = mn_map(a_map(s, l), 2, &p.a_3d);
+      const CUtensorMap& bmap = mn_map(dz_map(s, l), bnh / 64, &p.b_3d);
+      ET_TRY((launch_tc<true, true>(L.bn_wgrad, L.pair_wgrad, amap, bmap, em, p, epi, s->sms, st)));
     } else {
       et::simt::Params p;
       p.rows = L.K; p.cols = L.N; p.kc = (int)s->M; p.segs = 1;
@@ -435,7 +528,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
   } else {
     if constexpr (is_bf16<T>::value) {
       if (s->map_dy_ptr != dY) {
-        ET_TRY(make_map(&s->map_dy, dY, s->out_width(), s->M));
+        ET_TRY(make_tmaps(&s->map_dy, dY, s->out_width(), s->M));
         s->map_dy_ptr = dY;
       }
     }
@@ -499,9 +592,9 @@ et_status validate_backward_args(const et_stack* s, const void* dY, const uint8_
 template <typename T>
 et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
   if constexpr (is_bf16<T>::value) {
-    if (s->x != x || !s->forwarded) ET_TRY(make_map(&s->map_x, x, s->ly[0].K, s->M));
+    if (s->x != x || !s->forwarded) ET_TRY(make_tmaps(&s->map_x, x, s->ly[0].K, s->M));
     if (s->map_y_ptr != y) {
-      ET_TRY(make_map(&s->map_y, y, s->out_width(), s->M));
+      ET_TRY(make_tmaps(&s->map_y, y, s->out_width(), s->M));
       s->map_y_ptr = y;
     }
   }
@@ -580,21 +673,22 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
     if (dtype == ET_BF16) {
       const int kb_n = ceil_div(y.Nw, et::tc::BK) * y.fold;
-      y.bn_fwd = choose_tiles((int)M, y.Nw, ceil_div(y.K, et::tc::BK) * y.fold, s->sms, false).bn;
-      y.bn_dgrad = choose_tiles((int)M, y.K, kb_n, s->sms, false).bn;
-      TilePlan w = choose_tiles(y.K, y.N, ceil_div(M, et::tc::BK), s->sms, true);
-      if (y.fold > 1 && y.Nw % w.bn != 0) {                     // a folded wgrad tile must not straddle slices
-        w.bn = 256;
-        TilePlan best{256, 1}; double bc = -1;
-        for (int sp = 1; sp <= 16; ++sp) {
-          const int kbt = ceil_div(M, et::tc::BK), kbs = ceil_div(kbt, sp);
-          if (sp > kbt || (long long)(sp - 1) * kbs >= kbt) continue;
-          const double c = (double)ceil_div((long long)ceil_div(y.K, et::tc::BM) * ceil_div(y.N, 256) * sp, s->sms) * (kbs + 6);
-          if (bc < 0 || c < bc) { bc = c; best = {256, sp}; }
+      const TilePlan f = choose_tiles((int)M, y.Nw, ceil_div(y.K, et::tc::BK) * y.fold, s->sms, false, false, 0);
+      const TilePlan d = choose_tiles((int)M, y.K, kb_n, s->sms, false, true, 0);
+      const TilePlan w = choose_tiles(y.K, y.N, ceil_div(M, et::tc::BK), s->sms, true, false, y.fold > 1 ? y.Nw : 0);
+      y.bn_fwd = f.bn; y.pair_fwd = f.pair;
+      y.bn_dgrad = d.bn; y.pair_dgrad = d.pair;
+      y.bn_wgrad = w.bn; y.pair_wgrad = w.pair; y.split = w.split;
+      if (const char* force = getenv("ET_DEBUG_TILES")) {          // debug: "<bn>,<pair>[,<split>]" for every GEMM
+        int fb = 0, fp = 0, fs = 0;
+        if (sscanf(force, "%d,%d,%d", &fb, &fp, &fs) >= 2 && (fb == 128 || fb == 192 || fb == 256)) {
+          y.bn_dgrad = fb; y.pair_dgrad = fp != 0;
+          const int fbm = (fb == 192) ? 256 : fb;                   // MN-major B has no 192-wide pair tile
+          y.bn_fwd = fp ? fbm : fb; y.pair_fwd = fp != 0;
+          if (y.fold == 1 || y.Nw % (fp ? fbm : fb) == 0) { y.bn_wgrad = fp ? fbm : fb; y.pair_wgrad = fp != 0; }
+          if (fs > 0) y.split = std::min(fs, ceil_div(M, et::tc::BK));
         }
-        w = best;
       }
-      y.bn_wgrad = w.bn; y.split = w.split;
     }
     max_partial = std::max(max_partial, (size_t)y.split * y.K * y.N * sizeof(float));
     max_biaspart = std::max(max_biaspart, (size_t)chunks * y.Nw * sizeof(float));
@@ -644,14 +738,15 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   if (s->dtype == ET_BF16) {
     for (int l = 0; l < s->L; ++l) {
       LayerRT& y = s->ly[l];
-      ET_TRY(make_map(&y.map_W, y.W, y.N, y.K));
+      ET_TRY(make_tmaps(&y.map_W, y.W, y.N, y.K));
+      ET_TRY(make_map(&y.map_Wd, y.W, y.N, y.K, y.pair_dgrad ? y.bn_dgrad / 2 : y.bn_dgrad));
       if (l < s->L - 1) {
-        ET_TRY(make_map(&y.map_aout, s->at(y.off_a_out), y.Nw, s->M));
-        ET_TRY(make_map(&y.map_Gout, s->at(y.off_G_out), y.Nw, s->M));
+        ET_TRY(make_tmaps(&y.map_aout, s->at(y.off_a_out), y.Nw, s->M));
+        ET_TRY(make_tmaps(&y.map_Gout, s->at(y.off_G_out), y.Nw, s->M));
       }
       if (y.act != ET_ACT_NONE) {
-        ET_TRY(make_map(&y.map_Z, s->at(y.off_Z), y.Nw, s->M));
-        ET_TRY(make_map(&y.map_dZ, s->at(y.off_dZ), y.Nw, s->M));
+        ET_TRY(make_tmaps(&y.map_Z, s->at(y.off_Z), y.Nw, s->M));
+        ET_TRY(make_tmaps(&y.map_dZ, s->at(y.off_dZ), y.Nw, s->M));
       }
     }
   }

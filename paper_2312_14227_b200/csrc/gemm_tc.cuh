@@ -8,6 +8,12 @@
 //   dgrad    dX = dZ * W^T    A = dZ  K-major,   B = W   K-major
 //   wgrad    dW = a^T * dZ    A = a   MN-major,  B = dZ  MN-major   (contraction over tokens)
 //
+// PAIR = true runs two CTAs of a cluster as one unit (tcgen05 cta_group::2): a 256-row tile whose
+// B operand is split between the two CTAs' shared memories, so each CTA fetches half as many B
+// bytes from L2 per flop.  CTA 0 of the pair issues the MMAs; every load of either CTA reports
+// to CTA 0's "full" barrier; MMA completion is signalled to both CTAs' "empty" / "accumulator
+// full" barriers; both CTAs' epilogue warps report to CTA 0's "accumulator empty" barrier.
+//
 // Epilogues that read or write bf16 tensors (forward, dgrad) move them with TMA through
 // 128-byte-swizzled shared-memory chunks of 128 rows x 64 columns: a loader warp prefetches the
 // operand chunks (skip gradient, pre-activation, residual) while the main loop of the tile is
@@ -38,9 +44,10 @@ constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t SMEM_LIMIT = 227 * 1024;
 constexpr uint32_t SMEM_SLACK = 1024 /*alignment*/ + 256 /*barriers*/;
 
-template <int BN, int SLOTS>
+template <int BN, int SLOTS, bool PAIR>
 struct Cfg {
-  static constexpr uint32_t B_STAGE_BYTES = BN * BK * 2;
+  static constexpr int BNH = PAIR ? BN / 2 : BN;                 // B columns this CTA loads
+  static constexpr uint32_t B_STAGE_BYTES = BNH * BK * 2;
   static constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
   static constexpr uint32_t EPI_BYTES = (uint32_t)EPI_SETS * SLOTS * EPI_CHUNK_BYTES;
   static constexpr int STAGES_FIT = (int)((SMEM_LIMIT - SMEM_SLACK - EPI_BYTES) / STAGE_BYTES);
@@ -48,6 +55,7 @@ struct Cfg {
   static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + SMEM_SLACK;
   static_assert(STAGES >= 3, "too few pipeline stages");
   static_assert(BN % 64 == 0 && BN >= 64 && BN <= 256, "tile width");
+  static_assert(BNH % 32 == 0, "half tile width");
 };
 
 // Bounded waits: a wait that has not succeeded after this many polls gives up, records
@@ -74,11 +82,13 @@ struct Params {
   int b_k_seg_stride;        // added to B's k coordinate per segment   (dgrad through a fold)
   int b_mn_seg_stride;       // added to B's mn coordinate per segment  (forward through a fold)
   int b_mn_wrap;             // B's mn coordinate taken modulo this, 0 = off (wgrad through a fold)
+  int a_3d, b_3d;            // MN-major operand fetched by one 3-D copy (all 64-wide chunks at once)
+                             // instead of one 2-D copy per chunk; needs its width to be a multiple of 64
   uint32_t* status;          // device word, 0 = ok; first failure wins
 };
 
 // Tensor maps of the staged epilogue: per slot one optional input and one optional output,
-// all [rows x cols] bf16 row-major with the output's shape.
+// all [rows x cols] bf16 row-major with the output's shape, boxes of 64 columns x 128 rows.
 struct EpiMaps {
   CUtensorMap in[2];
   CUtensorMap out[2];
@@ -125,6 +135,57 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
 }
+// Pair variant: the copy lands in this CTA's shared memory, its bytes are reported to the barrier
+// at the same offset in CTA 0 of the pair (cluster shared addresses carry the CTA rank in bit 24).
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar & kPeerBitMask), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar & kPeerBitMask), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `cta` of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t cta) {
+  asm volatile(
+      "{\n\t.reg .b32 rem;\n\t"
+      "mapa.shared::cluster.u32 rem, %0, %1;\n\t"
+      "mbarrier.arrive.shared::cluster.b64 _, [rem];\n\t}"
+      ::"r"(bar), "r"(cta)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {     // arrives in both CTAs of the pair
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3)
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1)
@@ -168,7 +229,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
-// Every operand stage is a sequence of 8-KB chunks, one TMA box each: 64 rows of 128 B.
+// Every operand stage is a sequence of 8-KB chunks of 64 rows of 128 B.
 //   K-major  : a row holds 64 contraction elements of one mn index; 8-row groups are 1024 B
 //              apart (stride offset); the leading offset is unused with swizzling (set 1).
 //   MN-major : a row holds 64 mn elements of one k; 8 k-rows form a 1024-B group (stride
@@ -186,10 +247,10 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lead_bytes
 
 // Instruction descriptor for kind::f16: fp32 accumulate (bits 4-5 = 1), bf16 A and B
 // (bits 7-9, 10-12 = 1), operand major-ness (bits 15, 16), N/8 (bits 17-22), M/16 (bits 24-28).
-template <int BN, bool A_MN, bool B_MN>
+template <int MM, int BN, bool A_MN, bool B_MN>
 __host__ __device__ constexpr uint32_t make_idesc() {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((A_MN ? 1u : 0u) << 15) | ((B_MN ? 1u : 0u) << 16) |
-         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(MM >> 4) << 24);
 }
 
 template <class Epi>
@@ -229,12 +290,19 @@ __device__ __forceinline__ void sts_row32(uint8_t* chunk, int row, int half, con
 // Epi::kSlots  > 0: staged epilogue, Epi::combine(col0, acc, s0, s1) turns the accumulator and
 //                   the slots' input values into the slots' output values, in place; the flags
 //                   Epi::has_in[s] / has_out[s] say which slots carry an input / an output.
-template <int BN, bool A_MN, bool B_MN, class Epi>
+template <int BN, bool A_MN, bool B_MN, class Epi, bool PAIR>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ EpiMaps emaps, const Params p, const Epi epi_in) {
   constexpr int SLOTS = Epi::kSlots;
-  using C = Cfg<BN, SLOTS>;
+  using C = Cfg<BN, SLOTS, PAIR>;
+  constexpr int BNH = C::BNH;
+  static_assert(BNH % 64 == 0 || !B_MN, "an MN-major B needs whole 64-element chunks per CTA");
+  constexpr int TILE_M = PAIR ? 2 * BM : BM;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const bool leader_cta = rank == 0;
+  const int unit0 = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int unit_step = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   constexpr int STAGES = C::STAGES;
   constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES;
   constexpr int NCHUNK = BN / 64;
@@ -261,19 +329,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), PAIR ? 8 : 4); }
     for (int s = 0; s < EPI_SETS; ++s) { mbar_init(in_full_bar(s), 1); mbar_init(in_empty_bar(s), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                   ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();          // the peer's barriers exist before anything targets them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -289,9 +364,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      auto load = [&](uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1) {
+        if constexpr (PAIR) tma_load_2d_pair(dst, m, bar, c0, c1);
+        else tma_load_2d(dst, m, bar, c0, c1);
+      };
+      auto load3 = [&](uint32_t dst, const CUtensorMap* m, uint32_t bar, int c0, int c1, int c2) {
+        if constexpr (PAIR) tma_load_3d_pair(dst, m, bar, c0, c1, c2);
+        else tma_load_3d(dst, m, bar, c0, c1, c2);
+      };
+      for (int u = unit0; u < units && ok; u += unit_step) {
         const int sp = u / tiles, t = u - sp * tiles;
-        const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+        const int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
         const int kb0 = sp * p.kb_per_split;
         const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -300,20 +383,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int seg = kb / p.kb_per_seg, kk = (kb - seg * p.kb_per_seg) * BK;
           const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
           const uint32_t bar = full_bar(stage);
-          mbar_expect_tx(bar, STAGE_BYTES);
-          // every tensor map has a 64 x 64 box: one box = one 8-KB chunk of 64 rows of 128 B
+          // in a pair, CTA 0 announces the bytes of both CTAs' copies
+          if (leader_cta) mbar_expect_tx(bar, (PAIR ? 2u : 1u) * STAGE_BYTES);
+          // Few, large copies: issuing a TMA copy costs the producer thread far more than
+          // the copy's size does.  K-major operands come as one box of 64 k x (tile rows);
+          // MN-major operands as one 3-D box (64 mn, 64 k, chunks) when their width allows.
+          if constexpr (!A_MN) {
+            load(sa, &map_a, bar, kk, m0);
+          } else if (p.a_3d) {
+            load3(sa, &map_a, bar, 0, kk, m0 >> 6);
+          } else {
 #pragma unroll
-          for (int c = 0; c < BM / 64; ++c) {
-            if (A_MN) tma_load_2d(sa + c * CHUNK_BYTES, &map_a, bar, m0 + c * 64, kk);
-            else      tma_load_2d(sa + c * CHUNK_BYTES, &map_a, bar, kk, m0 + c * 64);
+            for (int c = 0; c < BM / 64; ++c) load(sa + c * CHUNK_BYTES, &map_a, bar, m0 + c * 64, kk);
           }
           const int bk = kk + seg * p.b_k_seg_stride;
           int bn = p.b_mn_wrap > 0 ? n0 % p.b_mn_wrap : n0;
-          bn += seg * p.b_mn_seg_stride;
+          bn += seg * p.b_mn_seg_stride + (int)rank * BNH;
+          if constexpr (!B_MN) {
+            load(sb, &map_b, bar, bk, bn);
+          } else if (p.b_3d) {
+            load3(sb, &map_b, bar, 0, bk, bn >> 6);
+          } else {
 #pragma unroll
-          for (int c = 0; c < BN / 64; ++c) {
-            if (B_MN) tma_load_2d(sb + c * CHUNK_BYTES, &map_b, bar, bn + c * 64, bk);
-            else      tma_load_2d(sb + c * CHUNK_BYTES, &map_b, bar, bk, bn + c * 64);
+            for (int c = 0; c < BNH / 64; ++c) load(sb + c * CHUNK_BYTES, &map_b, bar, bn + c * 64, bk);
           }
           ++fills[stage];
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -321,26 +413,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
       if (!ok) {
         // wind-down: let every copy this thread issued land before the CTA's shared memory goes away
+        if (leader_cta) {
 #pragma unroll
-        for (int s = 0; s < STAGES; ++s) {
-          if (fills[s] == 0) continue;
-          const uint32_t par = (fills[s] - 1u) & 1u;
-          bool landed = false;
-          for (uint32_t it = 0; it < (1u << 20) && !landed; ++it) landed = mbar_try_wait(full_bar(s), par);
-          if (!landed) atomicCAS(p.status, 0u, (uint32_t)kTimeoutDrain);
+          for (int s = 0; s < STAGES; ++s) {
+            if (fills[s] == 0) continue;
+            const uint32_t par = (fills[s] - 1u) & 1u;
+            bool landed = false;
+            for (uint32_t it = 0; it < (1u << 20) && !landed; ++it) landed = mbar_try_wait(full_bar(s), par);
+            if (!landed) atomicCAS(p.status, 0u, (uint32_t)kTimeoutDrain);
+          }
+        } else {
+          for (int it = 0; it < 2000; ++it) __nanosleep(1000);   // CTA 1 has no barrier of its own to watch
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc<BN, A_MN, B_MN>();
+    if (lane == 0 && leader_cta) {
+      constexpr uint32_t idesc = make_idesc<TILE_M, BN, A_MN, B_MN>();
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      for (int u = unit0; u < units && ok; u += unit_step) {
         const int sp = u / tiles;
         const int kb0 = sp * p.kb_per_split;
         const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
@@ -359,13 +455,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // MN-major: 16 k-rows = two 1024-B groups further.
             const uint64_t da = A_MN ? make_desc(sa + k * 2048, CHUNK_BYTES, 1024) : make_desc(sa + k * 32, 16, 1024);
             const uint64_t db = B_MN ? make_desc(sb + k * 2048, CHUNK_BYTES, 1024) : make_desc(sb + k * 32, 16, 1024);
-            tc_mma(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+            if constexpr (PAIR) tc_mma_pair(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+            else tc_mma(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           }
-          tc_commit(empty_bar(stage));              // frees the stage once these MMAs have read it
+          // frees the stage (in both CTAs of a pair) once these MMAs have read it
+          if constexpr (PAIR) tc_commit_pair(empty_bar(stage)); else tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(acc_full_bar(acc));               // accumulator complete
+        if constexpr (PAIR) tc_commit_pair(acc_full_bar(acc)); else tc_commit(acc_full_bar(acc));   // accumulator complete
         if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -382,9 +480,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
         for (int i = 0; i < EPI_SETS; ++i) fills[i] = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        for (int u = unit0; u < units && ok; u += unit_step) {
           const int t = u % tiles;
-          const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+          const int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
           for (int c = 0; c < NCHUNK; ++c) {
             const int col0 = n0 + c * 64;
             if (col0 >= p.cols) break;
@@ -397,8 +495,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int s = 0; s < SLOTS; ++s) {
                 if (!epi_in.has_in[s]) continue;
                 const uint32_t dst = epi_base + (bs * SLOTS + s) * EPI_CHUNK_BYTES;
-                tma_load_2d(dst, &emaps.in[s], bar, col0, m0);
-                tma_load_2d(dst + CHUNK_BYTES, &emaps.in[s], bar, col0, m0 + 64);
+                tma_load_2d(dst, &emaps.in[s], bar, col0, m0);       // one box of 64 columns x 128 rows
               }
               ++fills[bs];
             } else {
@@ -431,9 +528,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint32_t use = 0;                               // how often it has been used before,
     bool first_chunk = true;                        // and whether any chunk has been stored yet
     bool ok = true;
-    for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+    auto release_acc = [&](int a) {
+      if constexpr (PAIR) mbar_arrive_remote(acc_empty_bar(a), 0u);
+      else mbar_arrive(acc_empty_bar(a));
+    };
+    for (int u = unit0; u < units && ok; u += unit_step) {
       const int sp = u / tiles, t = u - sp * tiles;
-      const int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+      const int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
       epi_set_split(epi, sp);
       ok = mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, p.status, kTimeoutEpilogue);
       if (!ok) break;
@@ -451,7 +552,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+        if (lane == 0) release_acc(acc);
       } else {
         int nch = 0;
 #pragma unroll
@@ -470,7 +571,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (c == nch - 1 && h == 1) {           // last read of this accumulator: hand it back
               tc_fence_before();
               __syncwarp();
-              if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+              if (lane == 0) release_acc(acc);
             }
             if (epi.has_in[0]) lds_row32(buf0, trow, h, s0);
             if (SLOTS > 1 && epi.has_in[SLOTS - 1]) lds_row32(buf1, trow, h, s1);
@@ -485,8 +586,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int s = 0; s < SLOTS; ++s) {
               if (!epi.has_out[s]) continue;
               const uint32_t src = epi_base + (bs * SLOTS + s) * EPI_CHUNK_BYTES;
-              tma_store_2d(&emaps.out[s], src, col0, m0);
-              if (m0 + 64 < p.rows) tma_store_2d(&emaps.out[s], src + CHUNK_BYTES, col0, m0 + 64);
+              if (m0 < p.rows) tma_store_2d(&emaps.out[s], src, col0, m0);
             }
             tma_store_commit();
             if (!first_chunk) {
@@ -507,9 +607,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();          // neither CTA leaves while the other may still touch it
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if constexpr (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
