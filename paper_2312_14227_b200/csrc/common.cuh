@@ -48,6 +48,33 @@ __device__ __forceinline__ float act_grad(float z, int act) {
   return 1.0f;
 }
 
+// bf16-storage variants: tanh from the MUFU unit (tanh.approx.f32, relative error about 2^-11,
+// below the 2^-9 rounding of the bf16 value the result is stored as).
+__device__ __forceinline__ float tanh_fast(float u) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  return t;
+}
+__device__ __forceinline__ float act_apply_fast(float z, int act) {
+  if (act == kActGelu) {
+    const float c0 = 0.7978845608028654f, c1 = 0.044715f;
+    return 0.5f * z * (1.0f + tanh_fast(c0 * (z + c1 * z * z * z)));
+  }
+  if (act == kActRelu) return z > 0.0f ? z : 0.0f;
+  return z;
+}
+__device__ __forceinline__ float act_grad_fast(float z, int act) {
+  if (act == kActGelu) {
+    const float c0 = 0.7978845608028654f, c1 = 0.044715f;
+    const float z2 = z * z;
+    const float t = tanh_fast(c0 * (z + c1 * z * z2));
+    const float du = c0 * (1.0f + 3.0f * c1 * z2);
+    return 0.5f * (1.0f + t) + 0.5f * z * (1.0f - t * t) * du;
+  }
+  if (act == kActRelu) return z > 0.0f ? 1.0f : 0.0f;
+  return 1.0f;
+}
+
 // ---- row segments: NV consecutive elements of one row, vectorised when aligned ----------
 // `n` = how many of the NV elements exist (ragged right edge); the rest read as 0.
 template <int NV>

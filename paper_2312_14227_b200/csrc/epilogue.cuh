@@ -99,7 +99,7 @@ struct FwdEpiS {
     }
     const bool res = has_in[0];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) s0[i] = act_apply(v[i], act) + (res ? s0[i] : 0.0f);
+    for (int i = 0; i < 32; ++i) s0[i] = act_apply_fast(v[i], act) + (res ? s0[i] : 0.0f);
   }
 };
 
@@ -118,7 +118,7 @@ struct DgradEpiS {
     if constexpr (SLOTS == 1) {
       if (mul_act) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) s0[i] = v[i] * act_grad(s0[i], act_prev);
+        for (int i = 0; i < 32; ++i) s0[i] = v[i] * act_grad_fast(s0[i], act_prev);
       } else {
         const bool skip = has_in[0];
 #pragma unroll
@@ -130,7 +130,7 @@ struct DgradEpiS {
       for (int i = 0; i < 32; ++i) {
         const float g = v[i] + (skip ? s0[i] : 0.0f);
         s0[i] = g;
-        s1[i] = g * act_grad(s1[i], act_prev);
+        s1[i] = g * act_grad_fast(s1[i], act_prev);
       }
     }
   }

@@ -295,11 +295,18 @@ et_status launch_tc(int bn, bool pair, const CUtensorMap& ma, const CUtensorMap&
     }
     return launch_tc_bn<256, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st);
   }
-  if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
-  // two staged slots leave too little shared memory for a 256-wide single-CTA operand ring
-  if (bn == 192 || Epi::kSlots == 2) return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
-  if constexpr (Epi::kSlots < 2) return launch_tc_bn<256, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
-  return ET_ERR_UNSUPPORTED;
+  // staged epilogues take 64 KB of shared memory per slot: a single CTA keeps a deep enough
+  // operand ring only with narrower tiles
+  if constexpr (Epi::kSlots == 2) {
+    return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+  } else if constexpr (Epi::kSlots == 1) {
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+    return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+  } else {
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+    if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+    return launch_tc_bn<256, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+  }
 }
 template <typename T, class Epi>
 et_status launch_simt(const T* A, const T* B, const et::simt::Params& p, const Epi& epi, cudaStream_t st) {

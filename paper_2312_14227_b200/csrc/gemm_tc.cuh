@@ -15,11 +15,13 @@
 // full" barriers; both CTAs' epilogue warps report to CTA 0's "accumulator empty" barrier.
 //
 // Epilogues that read or write bf16 tensors (forward, dgrad) move them with TMA through
-// 128-byte-swizzled shared-memory chunks of 128 rows x 64 columns: a loader warp prefetches the
-// operand chunks (skip gradient, pre-activation, residual) while the main loop of the tile is
-// still running, the four epilogue warps combine them with the accumulator in place, and one
-// thread stores the chunk back with TMA.  Global traffic is therefore fully coalesced although
-// each epilogue thread owns one accumulator row.
+// 128-byte-swizzled shared-memory chunks of 128 rows x 64 columns.  Two groups of four epilogue
+// warps each take every other chunk of a tile; per group one extra thread does all the TMA work:
+// it prefetches the operand chunks (skip gradient, pre-activation, residual) while the main
+// loop of the tile is still running, and stores a chunk once the group's 128 threads have
+// combined it with the accumulator in place.  The epilogue warps therefore never wait for a
+// copy they issued themselves, and global traffic is fully coalesced although each epilogue
+// thread owns one accumulator row.
 #pragma once
 
 #include <cuda.h>
@@ -35,11 +37,13 @@ constexpr int BK = 64;           // contraction elements per stage = one 128-byt
 constexpr int UK = 16;           // contraction elements per tcgen05.mma (bf16)
 constexpr int ACC_STAGES = 2;    // accumulator stages at TMEM columns 0 and 256
 constexpr int ACC_STRIDE = 256;
-constexpr int THREADS = 224;     // warp 0: TMA, warp 1: MMA + TMEM alloc, warps 2-5: epilogue, warp 6: epilogue loader
+constexpr int THREADS = 384;     // warp 0: TMA producer, warp 1: MMA + TMEM alloc, warps 2-9: two epilogue groups,
+                                 // warps 10-11: one TMA thread per epilogue group
+constexpr int EPI_GROUPS = 2;
 constexpr uint32_t CHUNK_BYTES = 64 * BK * 2;       // one TMA box: 64 rows of 128 B
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
 constexpr uint32_t EPI_CHUNK_BYTES = BM * 64 * 2;   // 128 rows x 64 bf16 columns
-constexpr int EPI_SETS = 3;      // staged-epilogue buffer sets: one being combined, one being stored, one being loaded
+constexpr int EPI_SETS = 2;      // staged-epilogue buffer sets per group: one being combined, one in flight
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t SMEM_LIMIT = 227 * 1024;
 constexpr uint32_t SMEM_SLACK = 1024 /*alignment*/ + 256 /*barriers*/;
@@ -49,7 +53,7 @@ struct Cfg {
   static constexpr int BNH = PAIR ? BN / 2 : BN;                 // B columns this CTA loads
   static constexpr uint32_t B_STAGE_BYTES = BNH * BK * 2;
   static constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-  static constexpr uint32_t EPI_BYTES = (uint32_t)EPI_SETS * SLOTS * EPI_CHUNK_BYTES;
+  static constexpr uint32_t EPI_BYTES = (uint32_t)EPI_GROUPS * EPI_SETS * SLOTS * EPI_CHUNK_BYTES;
   static constexpr int STAGES_FIT = (int)((SMEM_LIMIT - SMEM_SLACK - EPI_BYTES) / STAGE_BYTES);
   static constexpr int STAGES = STAGES_FIT > 6 ? 6 : STAGES_FIT;
   static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + SMEM_SLACK;
@@ -69,7 +73,7 @@ enum StatusCode : uint32_t {
   kTimeoutMma = 2,
   kTimeoutEpilogue = 3,
   kTimeoutDrain = 4,
-  kTimeoutEpiLoader = 5,
+  kTimeoutEpiTma = 5,
 };
 
 struct Params {
@@ -198,7 +202,6 @@ __device__ __forceinline__ void tma_store_wait_read() {
 }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -226,6 +229,38 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Two 32-column reads in flight, one wait.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, float (&v)[32]) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+// The "+r" constraints tie the wait to the registers the loads write: the compiler may not read
+// them earlier or move the wait past their first use.
+__device__ __forceinline__ void tmem_ld_wait(float (&a)[32], float (&b)[32]) {
+  uint32_t* x = reinterpret_cast<uint32_t*>(a);
+  uint32_t* y = reinterpret_cast<uint32_t*>(b);
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(x[0]), "+r"(x[1]), "+r"(x[2]), "+r"(x[3]), "+r"(x[4]), "+r"(x[5]), "+r"(x[6]), "+r"(x[7]),
+                 "+r"(x[8]), "+r"(x[9]), "+r"(x[10]), "+r"(x[11]), "+r"(x[12]), "+r"(x[13]), "+r"(x[14]), "+r"(x[15]),
+                 "+r"(x[16]), "+r"(x[17]), "+r"(x[18]), "+r"(x[19]), "+r"(x[20]), "+r"(x[21]), "+r"(x[22]), "+r"(x[23]),
+                 "+r"(x[24]), "+r"(x[25]), "+r"(x[26]), "+r"(x[27]), "+r"(x[28]), "+r"(x[29]), "+r"(x[30]), "+r"(x[31])
+               :: "memory");
+  asm volatile(""
+               : "+r"(y[0]), "+r"(y[1]), "+r"(y[2]), "+r"(y[3]), "+r"(y[4]), "+r"(y[5]), "+r"(y[6]), "+r"(y[7]),
+                 "+r"(y[8]), "+r"(y[9]), "+r"(y[10]), "+r"(y[11]), "+r"(y[12]), "+r"(y[13]), "+r"(y[14]), "+r"(y[15]),
+                 "+r"(y[16]), "+r"(y[17]), "+r"(y[18]), "+r"(y[19]), "+r"(y[20]), "+r"(y[21]), "+r"(y[22]), "+r"(y[23]),
+                 "+r"(y[24]), "+r"(y[25]), "+r"(y[26]), "+r"(y[27]), "+r"(y[28]), "+r"(y[29]), "+r"(y[30]), "+r"(y[31])
+               :: "memory");
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
@@ -311,17 +346,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzle atoms need 1024-B alignment
   uint8_t* gen_base = smem_raw + (base - raw);
-  const uint32_t epi_base = base + STAGES * STAGE_BYTES;        // [2 buffer sets][SLOTS][EPI_CHUNK_BYTES]
+  const uint32_t epi_base = base + STAGES * STAGE_BYTES;        // [group][buffer set][slot][EPI_CHUNK_BYTES]
   const uint32_t bars = epi_base + C::EPI_BYTES;
   // barrier slots (8 B each)
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto acc_full_bar = [&](int s) { return bars + 8u * (2 * STAGES + s); };
   auto acc_empty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 2 + s); };
-  auto in_full_bar = [&](int s) { return bars + 8u * (2 * STAGES + 4 + s); };
-  auto in_empty_bar = [&](int s) { return bars + 8u * (2 * STAGES + 4 + EPI_SETS + s); };
+  // per epilogue group g and buffer set b: "operands have landed" and "result is in place"
+  auto in_full_bar = [&](int g, int b) { return bars + 8u * (2 * STAGES + 4 + g * EPI_SETS + b); };
+  auto out_ready_bar = [&](int g, int b) { return bars + 8u * (2 * STAGES + 4 + (EPI_GROUPS + g) * EPI_SETS + b); };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(
-      gen_base + STAGES * STAGE_BYTES + C::EPI_BYTES + 8 * (2 * STAGES + 4 + 2 * EPI_SETS));
+      gen_base + STAGES * STAGE_BYTES + C::EPI_BYTES + 8 * (2 * STAGES + 4 + 2 * EPI_GROUPS * EPI_SETS));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5;
@@ -329,8 +365,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), PAIR ? 8 : 4); }
-    for (int s = 0; s < EPI_SETS; ++s) { mbar_init(in_full_bar(s), 1); mbar_init(in_empty_bar(s), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), PAIR ? 16 : 8); }
+    for (int g = 0; g < EPI_GROUPS; ++g)
+      for (int b = 0; b < EPI_SETS; ++b) { mbar_init(in_full_bar(g, b), 1); mbar_init(out_ready_bar(g, b), 128); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -467,66 +504,97 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
       }
     }
-  } else if (warp == 6) {
-    // ------------------------------------------------------------------ epilogue operand loader
+  } else if (warp >= 2 + 4 * EPI_GROUPS) {
+    // ------------------------------------------------------------------ epilogue TMA thread of group g
     if constexpr (SLOTS > 0) {
-      if (lane == 0) {
+      const int g = warp - (2 + 4 * EPI_GROUPS);
+      if (lane == 0 && g < EPI_GROUPS) {
         uint32_t tx = 0;
 #pragma unroll
         for (int s = 0; s < SLOTS; ++s) tx += epi_in.has_in[s] ? EPI_CHUNK_BYTES : 0u;
-        int bs = 0;                                   // buffer set of the next chunk
-        uint32_t use = 0;                             // how often that set has been used before
-        uint32_t fills[EPI_SETS];
+        // The group's chunks, in order, are numbered j = 0, 1, ...; chunk j uses buffer set j % 2.
+        // fetch(j) may start once the store of chunk j - 2 has finished reading that set.
+        auto chunk_coords = [&](int j, int* m0, int* col0) -> bool {   // j-th chunk of this group, if any
+          int seen = 0;
+          for (int u = unit0; u < units; u += unit_step) {
+            const int t = u % tiles;
+            const int n0 = (t % p.tiles_n) * BN;
+            int here = 0;
 #pragma unroll
-        for (int i = 0; i < EPI_SETS; ++i) fills[i] = 0;
-        bool ok = true;
-        for (int u = unit0; u < units && ok; u += unit_step) {
-          const int t = u % tiles;
-          const int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
-          for (int c = 0; c < NCHUNK; ++c) {
-            const int col0 = n0 + c * 64;
-            if (col0 >= p.cols) break;
-            ok = mbar_wait(in_empty_bar(bs), (use & 1u) ^ 1u, abort_flag, p.status, kTimeoutEpiLoader);
-            if (!ok) break;
-            const uint32_t bar = in_full_bar(bs);
-            if (tx > 0) {
-              mbar_expect_tx(bar, tx);
-#pragma unroll
-              for (int s = 0; s < SLOTS; ++s) {
-                if (!epi_in.has_in[s]) continue;
-                const uint32_t dst = epi_base + (bs * SLOTS + s) * EPI_CHUNK_BYTES;
-                tma_load_2d(dst, &emaps.in[s], bar, col0, m0);       // one box of 64 columns x 128 rows
-              }
-              ++fills[bs];
-            } else {
-              mbar_arrive(bar);                       // nothing to fetch: just pass the buffer on
+            for (int c = 0; c < NCHUNK; ++c) here += ((c & 1) == g && n0 + c * 64 < p.cols) ? 1 : 0;
+            if (j < seen + here) {
+              const int c = g + 2 * (j - seen);
+              *m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM;
+              *col0 = n0 + c * 64;
+              return true;
             }
-            if (++bs == EPI_SETS) { bs = 0; ++use; }
+            seen += here;
           }
-        }
-        if (!ok && tx > 0) {
+          return false;
+        };
+        auto fetch = [&](int j) {
+          int m0, col0;
+          if (!chunk_coords(j, &m0, &col0)) return;
+          const int b = j & 1;
+          const uint32_t bar = in_full_bar(g, b);
+          if (tx > 0) {
+            mbar_expect_tx(bar, tx);
 #pragma unroll
-          for (int b = 0; b < EPI_SETS; ++b) {
-            if (fills[b] == 0) continue;
-            const uint32_t par = (fills[b] - 1u) & 1u;
+            for (int s = 0; s < SLOTS; ++s) {
+              if (!epi_in.has_in[s]) continue;
+              const uint32_t dst = epi_base + (uint32_t)(((g * EPI_SETS + b) * SLOTS + s) * EPI_CHUNK_BYTES);
+              tma_load_2d(dst, &emaps.in[s], bar, col0, m0);       // one box of 64 columns x 128 rows
+            }
+          } else {
+            mbar_arrive(bar);                                      // nothing to fetch: hand the set over
+          }
+        };
+        fetch(0);
+        fetch(1);
+        bool ok = true;
+        int fetched = 2;
+        for (int j = 0; ok; ++j) {
+          int m0, col0;
+          if (!chunk_coords(j, &m0, &col0)) break;
+          const int b = j & 1;
+          ok = mbar_wait(out_ready_bar(g, b), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, kTimeoutEpiTma);
+          if (!ok) break;
+          if (m0 < p.rows) {
+#pragma unroll
+            for (int s = 0; s < SLOTS; ++s) {
+              if (!epi_in.has_out[s]) continue;
+              const uint32_t src = epi_base + (uint32_t)(((g * EPI_SETS + b) * SLOTS + s) * EPI_CHUNK_BYTES);
+              tma_store_2d(&emaps.out[s], src, col0, m0);
+            }
+          }
+          tma_store_commit();
+          tma_store_wait_read<0>();                   // the set may be overwritten from here on
+          fetch(j + 2);
+          fetched = j + 3;
+        }
+        tma_store_wait_all();                         // shared memory must outlive the last store
+        if (!ok && tx > 0) {
+          // wind-down: copies already requested must land before the CTA's shared memory goes away
+          for (int j = max(0, fetched - 2); j < fetched; ++j) {
+            int m0, col0;
+            if (!chunk_coords(j, &m0, &col0)) continue;
             bool landed = false;
-            for (uint32_t it = 0; it < (1u << 20) && !landed; ++it) landed = mbar_try_wait(in_full_bar(b), par);
+            for (uint32_t it = 0; it < (1u << 20) && !landed; ++it)
+              landed = mbar_try_wait(in_full_bar(g, j & 1), (uint32_t)(j >> 1) & 1u);
             if (!landed) atomicCAS(p.status, 0u, (uint32_t)kTimeoutDrain);
           }
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue warps 2..9
     Epi epi = epi_in;
+    const int g = (warp - 2) >> 2;                  // epilogue group: takes the tile's chunks c with c % 2 == g
     const int quad = warp & 3;                      // TMEM lanes this warp may read: 32*quad ...
     const int trow = quad * 32 + lane;              // row inside the tile
-    const bool leader = (warp == 2 && lane == 0);   // issues the TMA stores
     int acc = 0;
     uint32_t acc_phase = 0;
-    int bs = 0;                                     // staged path: buffer set of the next chunk,
-    uint32_t use = 0;                               // how often it has been used before,
-    bool first_chunk = true;                        // and whether any chunk has been stored yet
+    int j = 0;                                      // staged path: running chunk number of this group
     bool ok = true;
     auto release_acc = [&](int a) {
       if constexpr (PAIR) mbar_arrive_remote(acc_empty_bar(a), 0u);
@@ -543,36 +611,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if constexpr (SLOTS == 0) {
         const int row = m0 + trow;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-          float v[32];
-          tmem_ld32(taddr + c * 32, v);             // warp-collective: every lane takes part
-          const int col0 = n0 + c * 32;
-          const int nv = p.cols - col0;
-          if (row < p.rows && nv > 0) epi.template operator()<32>(row, col0, nv, v);
+        for (int c = g; c < NCHUNK; c += EPI_GROUPS) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float v[32];
+            tmem_ld32(taddr + c * 64 + h * 32, v);  // warp-collective: every lane takes part
+            const int col0 = n0 + c * 64 + h * 32;
+            const int nv = p.cols - col0;
+            if (row < p.rows && nv > 0) epi.template operator()<32>(row, col0, nv, v);
+          }
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) release_acc(acc);
       } else {
-        int nch = 0;
+        int nch = 0;                                // this group's chunks in this tile
 #pragma unroll
-        for (int c = 0; c < NCHUNK; ++c) nch += (n0 + c * 64 < p.cols) ? 1 : 0;
+        for (int c = 0; c < NCHUNK; ++c) nch += ((c & 1) == g && n0 + c * 64 < p.cols) ? 1 : 0;
+        if (nch == 0) {                             // nothing to read, but the accumulator still has to be handed back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) release_acc(acc);
+        }
 #pragma unroll 1
-        for (int c = 0; c < nch; ++c) {
+        for (int i = 0; i < nch; ++i, ++j) {
+          const int c = g + 2 * i;
           const int col0 = n0 + c * 64;
-          ok = mbar_wait(in_full_bar(bs), use & 1u, abort_flag, p.status, kTimeoutEpilogue);
+          const int b = j & 1;
+          float v0[32], v1[32];
+          tmem_ld32_issue(taddr + c * 64, v0);
+          tmem_ld32_issue(taddr + c * 64 + 32, v1);
+          tmem_ld_wait(v0, v1);
+          if (i == nch - 1) {                       // last read of this accumulator by this warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) release_acc(acc);
+          }
+          ok = mbar_wait(in_full_bar(g, b), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, kTimeoutEpilogue);
           if (!ok) break;
-          uint8_t* buf0 = gen_base + STAGES * STAGE_BYTES + (bs * SLOTS + 0) * EPI_CHUNK_BYTES;
-          uint8_t* buf1 = gen_base + STAGES * STAGE_BYTES + (bs * SLOTS + (SLOTS - 1)) * EPI_CHUNK_BYTES;
+          uint8_t* buf0 = gen_base + STAGES * STAGE_BYTES + ((g * EPI_SETS + b) * SLOTS + 0) * EPI_CHUNK_BYTES;
+          uint8_t* buf1 = gen_base + STAGES * STAGE_BYTES + ((g * EPI_SETS + b) * SLOTS + (SLOTS - 1)) * EPI_CHUNK_BYTES;
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
-            float v[32], s0[32], s1[32];
-            tmem_ld32(taddr + c * 64 + h * 32, v);
-            if (c == nch - 1 && h == 1) {           // last read of this accumulator: hand it back
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) release_acc(acc);
-            }
+            float (&v)[32] = h == 0 ? v0 : v1;
+            float s0[32], s1[32];
             if (epi.has_in[0]) lds_row32(buf0, trow, h, s0);
             if (SLOTS > 1 && epi.has_in[SLOTS - 1]) lds_row32(buf1, trow, h, s1);
             epi.combine(col0 + h * 32, p.cols - (col0 + h * 32), v, s0, s1);
@@ -580,28 +662,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (SLOTS > 1 && epi.has_out[SLOTS - 1]) sts_row32(buf1, trow, h, s1);
           }
           fence_async_smem();                       // generic-proxy writes -> visible to the TMA engine
-          epi_bar_sync();
-          if (leader) {
-#pragma unroll
-            for (int s = 0; s < SLOTS; ++s) {
-              if (!epi.has_out[s]) continue;
-              const uint32_t src = epi_base + (bs * SLOTS + s) * EPI_CHUNK_BYTES;
-              if (m0 < p.rows) tma_store_2d(&emaps.out[s], src, col0, m0);
-            }
-            tma_store_commit();
-            if (!first_chunk) {
-              tma_store_wait_read<1>();             // the previous chunk's stores have read their buffers
-              mbar_arrive(in_empty_bar(bs == 0 ? EPI_SETS - 1 : bs - 1));
-            }
-          }
-          first_chunk = false;
-          if (++bs == EPI_SETS) { bs = 0; ++use; }
+          mbar_arrive(out_ready_bar(g, b));         // 128 arrivals: the group's TMA thread may store the chunk
         }
       }
       if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
-    }
-    if constexpr (SLOTS > 0) {
-      if (leader) tma_store_wait_all();             // shared memory must outlive the last store's reads
     }
   }
 
