@@ -414,10 +414,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
         const int kb0 = sp * p.kb_per_split;
         const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+        int seg = kb0 / p.kb_per_seg, kk = (kb0 - seg * p.kb_per_seg) * BK;   // fold segment, k offset inside it
         for (int kb = kb0; kb < kb1; ++kb) {
           ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, kTimeoutProducer);
           if (!ok) break;
-          const int seg = kb / p.kb_per_seg, kk = (kb - seg * p.kb_per_seg) * BK;
           const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
           const uint32_t bar = full_bar(stage);
           // in a pair, CTA 0 announces the bytes of both CTAs' copies
@@ -446,6 +446,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           ++fills[stage];
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          kk += BK;
+          if (kk == p.kb_per_seg * BK) { kk = 0; ++seg; }
         }
       }
       if (!ok) {
