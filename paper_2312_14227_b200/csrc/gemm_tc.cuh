@@ -470,6 +470,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && leader_cta) {
       constexpr uint32_t idesc = make_idesc<TILE_M, BN, A_MN, B_MN>();
+      const uint64_t desc_a0 = A_MN ? make_desc(base, CHUNK_BYTES, 1024) : make_desc(base, 16, 1024);
+      const uint64_t desc_b0 = B_MN ? make_desc(base + A_STAGE_BYTES, CHUNK_BYTES, 1024)
+                                    : make_desc(base + A_STAGE_BYTES, 16, 1024);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -487,15 +490,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           ok = mbar_wait(full_bar(stage), phase, abort_flag, p.status, kTimeoutMma);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+          // descriptors of this stage: the address field (16-byte units) is the only part that
+          // moves.  K-major: 16 elements = 32 B further along the swizzled row per MMA;
+          // MN-major: 16 k-rows = two 1024-B groups further.
+          const uint64_t da = desc_a0 + (uint64_t)((uint32_t)stage * (STAGE_BYTES >> 4));
+          const uint64_t db = desc_b0 + (uint64_t)((uint32_t)stage * (STAGE_BYTES >> 4));
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k) {
-            // K-major: 16 elements = 32 B further along the swizzled row.
-            // MN-major: 16 k-rows = two 1024-B groups further.
-            const uint64_t da = A_MN ? make_desc(sa + k * 2048, CHUNK_BYTES, 1024) : make_desc(sa + k * 32, 16, 1024);
-            const uint64_t db = B_MN ? make_desc(sb + k * 2048, CHUNK_BYTES, 1024) : make_desc(sb + k * 32, 16, 1024);
-            if constexpr (PAIR) tc_mma_pair(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-            else tc_mma(d_tmem, da, db, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+            constexpr uint32_t step_a = (A_MN ? 2048u : 32u) >> 4, step_b = (B_MN ? 2048u : 32u) >> 4;
+            const uint32_t accumulate = (kb > kb0 || k > 0) ? 1u : 0u;
+            if constexpr (PAIR) tc_mma_pair(d_tmem, da + k * step_a, db + k * step_b, idesc, accumulate);
+            else tc_mma(d_tmem, da + k * step_a, db + k * step_b, idesc, accumulate);
           }
           // frees the stage (in both CTAs of a pair) once these MMAs have read it
           if constexpr (PAIR) tc_commit_pair(empty_bar(stage)); else tc_commit(empty_bar(stage));
@@ -516,28 +521,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int s = 0; s < SLOTS; ++s) tx += epi_in.has_in[s] ? EPI_CHUNK_BYTES : 0u;
         // The group's chunks, in order, are numbered j = 0, 1, ...; chunk j uses buffer set j % 2.
         // fetch(j) may start once the store of chunk j - 2 has finished reading that set.
-        auto chunk_coords = [&](int j, int* m0, int* col0) -> bool {   // j-th chunk of this group, if any
-          int seen = 0;
-          for (int u = unit0; u < units; u += unit_step) {
-            const int t = u % tiles;
-            const int n0 = (t % p.tiles_n) * BN;
-            int here = 0;
-#pragma unroll
-            for (int c = 0; c < NCHUNK; ++c) here += ((c & 1) == g && n0 + c * 64 < p.cols) ? 1 : 0;
-            if (j < seen + here) {
-              const int c = g + 2 * (j - seen);
-              *m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM;
-              *col0 = n0 + c * 64;
+        // Two cursors walk the same chunk sequence: one for fetches (two chunks ahead), one for stores.
+        struct Cursor {
+          int u, c, m0, n0;
+          bool fresh;
+        };
+        auto advance = [&](Cursor& k, int* m0, int* col0) -> bool {      // next chunk of this group, if any
+          while (k.u < units) {
+            if (k.fresh) {
+              const int t = k.u % tiles;
+              k.m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM;
+              k.n0 = (t % p.tiles_n) * BN;
+              k.c = g;
+              k.fresh = false;
+            }
+            if (k.c < NCHUNK && k.n0 + k.c * 64 < p.cols) {
+              *m0 = k.m0;
+              *col0 = k.n0 + k.c * 64;
+              k.c += EPI_GROUPS;
               return true;
             }
-            seen += here;
+            k.u += unit_step;
+            k.fresh = true;
           }
           return false;
         };
-        auto fetch = [&](int j) {
+        Cursor fc{unit0, 0, 0, 0, true}, sc{unit0, 0, 0, 0, true};
+        int fetched = 0;                                                 // chunks requested so far
+        auto fetch = [&]() {
           int m0, col0;
-          if (!chunk_coords(j, &m0, &col0)) return;
-          const int b = j & 1;
+          if (!advance(fc, &m0, &col0)) return;
+          const int b = fetched & 1;
+          ++fetched;
           const uint32_t bar = in_full_bar(g, b);
           if (tx > 0) {
             mbar_expect_tx(bar, tx);
@@ -551,13 +566,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_arrive(bar);                                      // nothing to fetch: hand the set over
           }
         };
-        fetch(0);
-        fetch(1);
+        fetch();
+        fetch();
         bool ok = true;
-        int fetched = 2;
-        for (int j = 0; ok; ++j) {
+        int j = 0;
+        for (;; ++j) {
           int m0, col0;
-          if (!chunk_coords(j, &m0, &col0)) break;
+          if (!advance(sc, &m0, &col0)) break;
           const int b = j & 1;
           ok = mbar_wait(out_ready_bar(g, b), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, kTimeoutEpiTma);
           if (!ok) break;
@@ -571,18 +586,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           tma_store_commit();
           tma_store_wait_read<0>();                   // the set may be overwritten from here on
-          fetch(j + 2);
-          fetched = j + 3;
+          fetch();
         }
         tma_store_wait_all();                         // shared memory must outlive the last store
         if (!ok && tx > 0) {
           // wind-down: copies already requested must land before the CTA's shared memory goes away
-          for (int j = max(0, fetched - 2); j < fetched; ++j) {
-            int m0, col0;
-            if (!chunk_coords(j, &m0, &col0)) continue;
+          for (int f = max(j, fetched - 2); f < fetched; ++f) {
             bool landed = false;
             for (uint32_t it = 0; it < (1u << 20) && !landed; ++it)
-              landed = mbar_try_wait(in_full_bar(g, j & 1), (uint32_t)(j >> 1) & 1u);
+              landed = mbar_try_wait(in_full_bar(g, f & 1), (uint32_t)(f >> 1) & 1u);
             if (!landed) atomicCAS(p.status, 0u, (uint32_t)kTimeoutDrain);
           }
         }
