@@ -484,7 +484,7 @@ et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   ET_TRY(after_launch());
   ++*launches;
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l + 1];
-  et::bias_finish_kernel<T><<<L.imp_count_b, et::kEltThreads, 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
+  et::bias_finish_kernel<T><<<L.imp_count_b, dim3(32, 8), 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
                                                                        (T*)L.b, lr, sgd ? 1 : 0);
   ++*launches;
   return after_launch();
@@ -700,7 +700,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     max_partial = std::max(max_partial, (size_t)y.split * y.K * y.N * sizeof(float));
     max_biaspart = std::max(max_biaspart, (size_t)chunks * y.Nw * sizeof(float));
     y.imp_count_w = ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
-    y.imp_count_b = ceil_div(y.N, et::kEltThreads);
+    y.imp_count_b = ceil_div(y.N, et::kBiasCols);
     s->imp_offs[2 * l] = imp_total; s->imp_counts[2 * l] = y.imp_count_w; imp_total += y.imp_count_w;
     s->imp_offs[2 * l + 1] = imp_total; s->imp_counts[2 * l + 1] = y.imp_count_b; imp_total += y.imp_count_b;
   }

@@ -54,6 +54,7 @@ wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_
 
 // ---- bias gradient, stage 1: column sums of one chunk of rows ------------------------------
 // grid (ceil(width / 256), ceil(M / kColsumRows)); block (32, 8): x -> 8 columns, y -> row phase.
+// Each thread keeps four independent 16-byte loads in flight.
 template <typename T>
 __global__ void __launch_bounds__(256)
 colsum_partial_kernel(const T* __restrict__ dZ, int M, int width, float* __restrict__ part) {
@@ -66,9 +67,20 @@ colsum_partial_kernel(const T* __restrict__ dZ, int M, int width, float* __restr
   for (int i = 0; i < kVec; ++i) acc[i] = 0.0f;
   const int n = width - col0;
   if (n > 0) {
-    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
+    const T* base = dZ + col0;
+    int r = r0 + threadIdx.y;
+    for (; r + 24 < r1; r += 32) {
+      float v[4][kVec];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) load_seg<kVec>(base + (size_t)(r + 8 * q) * width, n, v[q]);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int i = 0; i < kVec; ++i) acc[i] += v[q][i];
+    }
+    for (; r < r1; r += 8) {
       float v[kVec];
-      load_seg<kVec>(dZ + (size_t)r * width + col0, n, v);
+      load_seg<kVec>(base + (size_t)r * width, n, v);
 #pragma unroll
       for (int i = 0; i < kVec; ++i) acc[i] += v[i];
     }
@@ -87,26 +99,38 @@ colsum_partial_kernel(const T* __restrict__ dZ, int M, int width, float* __restr
 }
 
 // ---- bias gradient, stage 2: sum the chunks, then grad / importance / SGD -----------------
-// One thread per bias element j in [0, fold*width); column = j mod width (a folded layer's
-// dZ is the same gradient repeated for each slice).
+// Block (32, 8) handles kBiasCols bias elements j in [0, fold*width): x -> element, y -> which
+// chunks (y, y+8, ...) this thread adds; a fixed-order shared-memory sum joins the eight.
+// column = j mod width (a folded layer's dZ is the same gradient repeated for each slice).
+constexpr int kBiasCols = 32;
 template <typename T>
-__global__ void __launch_bounds__(kEltThreads)
+__global__ void __launch_bounds__(256)
 bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
                    float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
                    T* __restrict__ b, float lr, int do_sgd) {
-  const int j = blockIdx.x * kEltThreads + threadIdx.x;
-  float dot = 0.0f;
+  __shared__ float sm[8][kBiasCols + 1];
+  const int j = blockIdx.x * kBiasCols + threadIdx.x;
+  float g = 0.0f;
   if (j < count) {
     const int col = j % width;
-    float g = 0.0f;
-    for (int c = 0; c < chunks; ++c) g += part[(size_t)c * width + col];
-    if (grad != nullptr) grad[j] = g;
-    if (delta != nullptr) dot = g * to_f32(delta[j]);
-    if (do_sgd) b[j] = from_f32<T>(fmaf(-lr, g, to_f32(b[j])));
+    for (int c = threadIdx.y; c < chunks; c += 8) g += part[(size_t)c * width + col];
   }
-  if (delta != nullptr) {
-    dot = block_sum(dot);
-    if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
+  sm[threadIdx.y][threadIdx.x] = g;
+  __syncthreads();
+  float dot = 0.0f;
+  if (threadIdx.y == 0) {
+    if (j < count) {
+      g = 0.0f;
+#pragma unroll
+      for (int y = 0; y < 8; ++y) g += sm[y][threadIdx.x];
+      if (grad != nullptr) grad[j] = g;
+      if (delta != nullptr) dot = g * to_f32(delta[j]);
+      if (do_sgd) b[j] = from_f32<T>(fmaf(-lr, g, to_f32(b[j])));
+    }
+    if (delta != nullptr) {                           // one warp: fixed shuffle tree
+      dot = warp_sum(dot);
+      if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
+    }
   }
 }
 
