@@ -71,7 +71,10 @@ typedef enum {
 } et_cost_variant;
 
 enum {
-  ET_FLAG_FUSE_SGD = 1u    /* et_backward_elastic also applies w <- w - lr*g to selected tensors */
+  ET_FLAG_FUSE_SGD = 1u,   /* et_backward_elastic also applies w <- w - lr*g to selected tensors */
+  ET_FLAG_DELTA_IS_SNAPSHOT = 2u  /* delta[k] is a copy of tensor k taken earlier; the update of Eq. 2 is
+                                     dw = (current tensor) - delta[k], formed on the fly (Section 3.1: the
+                                     weight update accumulated since the start of the evaluation period) */
 };
 
 typedef struct {
@@ -135,7 +138,8 @@ et_status et_loss_mse_grad(et_stack* s, const void* y, const void* target, void*
  *              NULL when the gradient itself is not wanted.  Entries of unselected
  *              tensors are ignored and their buffers never touched.
  *   delta      host array of 2L device pointers, storage dtype, same shapes as the
- *              tensors (or NULL array): the recent update dw of Eq. 2.  If given,
+ *              tensors (or NULL array): the recent update dw of Eq. 2 (or, with
+ *              ET_FLAG_DELTA_IS_SNAPSHOT, the earlier weights it is measured from).  If given,
  *              importance_dev must be given too, and every selected tensor needs an entry.
  *   importance_dev  device float[2L]: S_k for selected tensors, 0 for the others.
  *   flags, lr  ET_FLAG_FUSE_SGD applies w <- w - lr*g (Section 2.2's weight update) to

@@ -281,3 +281,80 @@ def select_by_depth_knapsack(I, qw, qy, budget: int, variant: int = STRICT) -> f
                 knap[w:] = np.maximum(knap[w:], knap[:-w] + I[i])
         best = max(best, I[d] + knap[cap])
     return float(best)
+
+
+def select_depth_knapsack_mask(I, qw, qy, budget: int, variant: int = STRICT):
+    """Optimum AND a mask attaining it, for instances too large to enumerate: for every
+    candidate deepest tensor d (selected by definition) a 0/1 knapsack with back-pointers over
+    the tensors after d.  Used by the training-schedule oracle; checked against brute force."""
+    I = np.asarray(I, dtype=np.float64)
+    qw = np.asarray(qw, dtype=np.int64)
+    qy = np.asarray(qy, dtype=np.int64)
+    n = len(I)
+    best_val, best_mask = 0.0, np.zeros(n, dtype=np.uint8)
+    for d in range(n):
+        fixed = int(qw[d] + qy[d + 1:].sum() + (qy[d] if variant == INCLUSIVE else 0))
+        cap = budget - fixed
+        if cap < 0:
+            continue
+        items = [i for i in range(d + 1, n) if I[i] > 0]
+        table = np.zeros((len(items) + 1, cap + 1))
+        for r, i in enumerate(items):
+            w = int(qw[i])
+            table[r + 1] = table[r]
+            if w <= cap:
+                cand = np.full(cap + 1, -np.inf)
+                cand[w:] = table[r][:cap + 1 - w] + I[i]
+                table[r + 1] = np.maximum(table[r], cand)
+        val = I[d] + table[len(items)][cap]
+        if val > best_val:
+            mask = np.zeros(n, dtype=np.uint8)
+            mask[d] = 1
+            c = cap
+            for r in range(len(items), 0, -1):
+                if table[r][c] != table[r - 1][c]:
+                    i = items[r - 1]
+                    mask[i] = 1
+                    c -= int(qw[i])
+            best_val, best_mask = float(val), mask
+    return best_mask, best_val
+
+
+def train_schedule(layers, W, b, x, target, lr: float, steps: int, period: int, window: int,
+                   rho: float, t_dw, t_dy, t_fwd: float = 0.0, Tq: int = 1000, variant: int = STRICT):
+    """Elastic training schedule (Section 3.1): each period of `period` steps starts with
+    `window` steps in which every tensor is trained; the weight change accumulated over the
+    window, measured at the window's last step before that step's own update, gives the
+    importances S_k = sum g * (w_now - w_window_start) of Eq. (2); -S_k (a loss decrease counts as
+    positive, Section 4) goes to the selector at budget rho; the remaining steps of the period
+    train the selected tensors only.  Plain SGD, one fixed batch.
+    Returns per-step losses, per-step masks and the importances of every evaluation."""
+    L = len(layers)
+    W = [np.array(w_, dtype=np.float64) for w_ in W]
+    b = [np.array(b_, dtype=np.float64) for b_ in b]
+    losses, masks, evaluations = [], [], []
+    mask = np.ones(2 * L, dtype=np.uint8)
+    qw, qy, budget = quantise(t_dw, t_dy, t_fwd, rho, Tq)
+    snap = None
+    for step in range(steps):
+        phase = step % period
+        if phase == 0:
+            mask = np.ones(2 * L, dtype=np.uint8)
+            snap = [p.copy() for p in tensors_of(W, b)]
+        saved = forward(layers, W, b, x)
+        loss, dY = mse_loss_grad(saved.a[-1], target)
+        grads, _ = backward_masked(layers, W, saved, dY, mask)
+        losses.append(loss)
+        masks.append(mask.copy())
+        params = tensors_of(W, b)
+        new_mask = None
+        if phase == window - 1:
+            delta = [p - s for p, s in zip(params, snap)]
+            S = importance(grads, delta, mask)
+            evaluations.append(S)
+            new_mask, _ = select_depth_knapsack_mask(-S, qw, qy, budget, variant)
+        new = sgd_masked(params, grads, mask, lr)
+        W, b = list(new[0::2]), list(new[1::2])
+        if new_mask is not None:
+            mask = new_mask
+    return dict(losses=np.array(losses), masks=masks, importances=evaluations, W=W, b=b)

@@ -21,6 +21,7 @@ ET_F32, ET_BF16 = 0, 1
 ET_ACT_NONE, ET_ACT_GELU_TANH, ET_ACT_RELU = 0, 1, 2
 ET_COST_STRICT, ET_COST_INCLUSIVE = 0, 1
 ET_FLAG_FUSE_SGD = 1
+ET_FLAG_DELTA_IS_SNAPSHOT = 2
 ET_ERR_INVALID_ARG, ET_ERR_SHAPE, ET_ERR_DTYPE, ET_ERR_STATE = 1, 2, 3, 4
 ET_ERR_WORKSPACE, ET_ERR_UNSUPPORTED, ET_ERR_CUDA, ET_ERR_TIMEOUT = 5, 6, 7, 8
 ET_ERR_TOO_LARGE = 9

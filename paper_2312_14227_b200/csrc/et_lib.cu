@@ -159,6 +159,7 @@ struct et_stack {
   TMaps map_x, map_y, map_dy;
   const void* map_dy_ptr = nullptr;
   const void* map_y_ptr = nullptr;
+  bool delta_is_snapshot = false;      // per call: the delta tensors hold a weight snapshot
   // optional per-kernel timing
   bool timing = false;
   struct Timed { int cls; cudaEvent_t e0, e1; };
@@ -467,7 +468,8 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   TimedLaunch tl(s, ET_K_WGRAD_REDUCE, st);
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
   et::wgrad_reduce_kernel<T><<<L.imp_count_w, et::kEltThreads, 0, st>>>(partial, split, count, count, grad, delta, imp,
-                                                                        (T*)L.W, lr, sgd ? 1 : 0);
+                                                                        (T*)L.W, lr, sgd ? 1 : 0,
+                                                                        s->delta_is_snapshot ? 1 : 0);
   ++*launches;
   return after_launch();
 }
@@ -485,7 +487,7 @@ et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   ++*launches;
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l + 1];
   et::bias_finish_kernel<T><<<L.imp_count_b, dim3(32, 8), 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
-                                                                       (T*)L.b, lr, sgd ? 1 : 0);
+                                                                       (T*)L.b, lr, sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0);
   ++*launches;
   return after_launch();
 }
@@ -514,6 +516,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
   for (int l = 0; l < L; ++l)
     if (mask[2 * l] || mask[2 * l + 1]) { d = l; break; }
   const bool sgd = (flags & ET_FLAG_FUSE_SGD) != 0;
+  s->delta_is_snapshot = delta != nullptr && (flags & ET_FLAG_DELTA_IS_SNAPSHOT) != 0;
   int launches = 0;
   double flops = 0.0;
 
@@ -802,7 +805,7 @@ et_status et_backward_elastic(et_stack* s, const void* dY, const uint8_t* mask, 
                               uint32_t flags, float lr, et_exec_report* report, void* stream) {
   ET_TRY(validate_backward_args(s, dY, mask, n_tensors, delta, importance_dev));
   if ((uintptr_t)dY & 15) return ET_ERR_INVALID_ARG;
-  if (flags & ~(uint32_t)ET_FLAG_FUSE_SGD) return ET_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(ET_FLAG_FUSE_SGD | ET_FLAG_DELTA_IS_SNAPSHOT)) return ET_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   return s->dtype == ET_BF16
              ? backward_impl<bf16>(s, dY, mask, grads, delta, importance_dev, flags, lr, report, st)
@@ -813,7 +816,7 @@ et_status et_backward_elastic_host(et_stack* s, const void* dY_host, const uint8
                                    float* const* grads, const void* const* delta, float* importance_host,
                                    uint32_t flags, float lr, et_exec_report* report, void* stream) {
   ET_TRY(validate_backward_args(s, dY_host, mask, n_tensors, delta, importance_host));
-  if (flags & ~(uint32_t)ET_FLAG_FUSE_SGD) return ET_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(ET_FLAG_FUSE_SGD | ET_FLAG_DELTA_IS_SNAPSHOT)) return ET_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   void* dY = s->at(s->off_dy_stage);
   float* imp = (float*)s->at(s->off_imp_stage);

@@ -15,13 +15,14 @@ constexpr int kColsumRows = 128;                // rows per column-sum chunk
 // ---- weight gradient: sum the K-split partials, then everything that consumes g ----------
 //   g = sum_s partial[s]                       (fixed order s = 0, 1, ...)
 //   grad        <- g                           if grad != nullptr
-//   imp_part[b] <- sum over this block of g * delta     if delta != nullptr   (Eq. 2)
+//   imp_part[b] <- sum over this block of g * dw        if delta != nullptr   (Eq. 2);
+//                  dw = delta, or W - delta when delta holds a snapshot of W
 //   W           <- W - lr * g                  if do_sgd   (fp32 arithmetic, one rounding)
 template <typename T>
 __global__ void __launch_bounds__(kEltThreads)
 wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_t count,
                     float* grad /* may alias partial: each thread reads its elements before writing them */, const T* __restrict__ delta, float* __restrict__ imp_part,
-                    T* __restrict__ W, float lr, int do_sgd) {
+                    T* __restrict__ W, float lr, int do_sgd, int delta_is_snapshot) {
   const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
   float dot = 0.0f;
   if (i0 < count) {
@@ -36,6 +37,12 @@ wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_
     if (grad != nullptr) store_seg<kVec>(grad + i0, n, g);
     if (delta != nullptr) {
       load_seg<kVec>(delta + i0, n, t);
+      if (delta_is_snapshot) {                        // dw = current weight - weight at the window start
+        float w[kVec];
+        load_seg<kVec>(W + i0, n, w);
+#pragma unroll
+        for (int i = 0; i < kVec; ++i) t[i] = w[i] - t[i];
+      }
 #pragma unroll
       for (int i = 0; i < kVec; ++i) dot = fmaf(g[i], t[i], dot);
     }
@@ -107,7 +114,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
                    float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
-                   T* __restrict__ b, float lr, int do_sgd) {
+                   T* __restrict__ b, float lr, int do_sgd, int delta_is_snapshot) {
   __shared__ float sm[8][kBiasCols + 1];
   const int j = blockIdx.x * kBiasCols + threadIdx.x;
   float g = 0.0f;
@@ -124,7 +131,7 @@ bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int co
 #pragma unroll
       for (int y = 0; y < 8; ++y) g += sm[y][threadIdx.x];
       if (grad != nullptr) grad[j] = g;
-      if (delta != nullptr) dot = g * to_f32(delta[j]);
+      if (delta != nullptr) dot = g * (delta_is_snapshot ? to_f32(b[j]) - to_f32(delta[j]) : to_f32(delta[j]));
       if (do_sgd) b[j] = from_f32<T>(fmaf(-lr, g, to_f32(b[j])));
     }
     if (delta != nullptr) {                           // one warp: fixed shuffle tree

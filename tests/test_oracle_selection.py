@@ -118,3 +118,44 @@ def test_quantise_eq_8():
     qw, qy, budget = orc.quantise([1.0, 2.5, 0.49], [0.5, 0.0, 0.51], t_fwd=0.0, rho=0.5, Tq=10)
     # T = 5, Z = 2
     assert qw.tolist() == [2, 5, 0] and qy.tolist() == [1, 0, 1] and budget == 5
+
+
+@pytest.mark.parametrize("variant", [orc.STRICT, orc.INCLUSIVE])
+def test_knapsack_mask_matches_bruteforce(variant):
+    rng = np.random.default_rng(40 + variant)
+    for trial in range(40):
+        n = int(rng.integers(1, 11))
+        I, qw, qy = wl.selector_instance(rng, n, t_max=12)
+        if trial % 3 == 0:
+            I[rng.integers(0, n)] = -0.2
+        qw, qy = qw.astype(np.int64), qy.astype(np.int64)
+        budget = int(rng.integers(0, int(qw.sum() + qy.sum()) + 2))
+        mask, val = orc.select_depth_knapsack_mask(I, qw, qy, budget, variant)
+        _, want = orc.select_bruteforce(I, qw, qy, budget, variant)
+        assert abs(val - want) < 1e-12
+        assert orc.t_selective(mask, qw, qy, variant) <= budget
+        assert abs(I[mask.astype(bool)].sum() - val) < 1e-12
+
+
+def test_train_schedule_structure_and_progress():
+    layers = wl.vit_blocks(2, 8, 16)
+    w = wl.small_stack(layers, 12, wl.DT_F32, 3, w_std=0.3)
+    L = len(layers)
+    t_dw = np.array([2.0 * ly.in_features * ly.out_features if t % 2 == 0 else ly.out_features
+                     for ly in layers for t in range(2)])
+    t_dy = np.array([2.0 * ly.in_features * ly.out_features if t % 2 == 0 else 0.0
+                     for ly in layers for t in range(2)])
+    out = orc.train_schedule(w.layers, w.W, w.b, w.x, w.target, lr=0.05, steps=24, period=8, window=3,
+                             rho=0.4, t_dw=t_dw, t_dy=t_dy, Tq=200)
+    assert out["losses"][-1] < out["losses"][0]
+    assert len(out["importances"]) == 3
+    for step, m in enumerate(out["masks"]):
+        if step % 8 < 3:
+            assert m.all()                                   # every tensor trains during the window
+        else:
+            assert not m.all()                               # rho = 0.4 cannot afford everything
+            assert orc.t_selective(m, t_dw, t_dy) <= 0.4 * (t_dw.sum() + t_dy.sum()) * 1.05
+            if step % 8 > 3:
+                assert np.array_equal(m, out["masks"][step - 1])   # masks only change at a reselection
+    # importances of useful updates are negative sums (the loss went down along them)
+    assert (np.concatenate(out["importances"]) <= 1e-12).mean() > 0.8
