@@ -78,6 +78,21 @@ struct DgradEpi {
 // which it replaces by the output values (on exit).  has_in / has_out tell the kernel which
 // slots to load and store.
 
+// Column sums over a warp's 32 rows: on entry lane r holds 32 consecutive columns of row r; on exit
+// lane i's v[0] is the sum over the 32 rows of column i.  31 shuffles (halving exchange).
+__device__ __forceinline__ void warp_column_sums(float (&v)[32], int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int k = 0; k < off; ++k) {
+      const float send = upper ? v[k] : v[k + off];
+      const float keep = upper ? v[k + off] : v[k];
+      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+}
+
 // Forward.  slot 0: in = residual a_j (optional), out = a_{l+1}.  slot 1 (SLOTS == 2): out = Z.
 template <int SLOTS>
 struct FwdEpiS {
@@ -101,18 +116,32 @@ struct FwdEpiS {
 #pragma unroll
     for (int i = 0; i < 32; ++i) s0[i] = act_apply_fast(v[i], act) + (res ? s0[i] : 0.0f);
   }
+  __device__ __forceinline__ void column_sums(int, int, int, float (&)[32], float (&)[32], int) const {}
 };
 
 // Error-gradient pass.  SLOTS == 2: slot 0: in = skip gradient (optional), out = G_l (optional);
 // slot 1: in = Z_{l-1}, out = dZ_{l-1} = G_l * act'(Z_{l-1}).
 // SLOTS == 1, mul_act == false: in = skip (optional), out = G_l = acc + skip.
 // SLOTS == 1, mul_act == true : in = Z_{l-1}, out = dZ_{l-1} = acc * act'(Z_{l-1}).
+// colsum != nullptr: the column sums of dZ_{l-1} over each warp's 32 rows are written to
+// colsum[row_block][column] as well -- the bias gradient of layer l-1 without re-reading dZ_{l-1}.
 template <int SLOTS>
 struct DgradEpiS {
   static constexpr int kSlots = SLOTS;
   bool has_in[2], has_out[2];
   bool mul_act;
   int act_prev;
+  float* colsum;     // [row blocks of 32][ld] or nullptr
+  int ld;
+
+  // s0 / s1 as combine() left them; destroys them.  row_block = (first row of the warp) / 32.
+  __device__ __forceinline__ void column_sums(int row_block, int col0, int nv, float (&s0)[32], float (&s1)[32],
+                                              int lane) const {
+    if (colsum == nullptr) return;
+    float (&dz)[32] = SLOTS == 1 ? s0 : s1;
+    warp_column_sums(dz, lane);
+    if (lane < nv) colsum[(size_t)row_block * ld + col0 + lane] = dz[0];
+  }
 
   __device__ __forceinline__ void combine(int, int, float (&v)[32], float (&s0)[32], float (&s1)[32]) const {
     if constexpr (SLOTS == 1) {

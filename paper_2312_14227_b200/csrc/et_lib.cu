@@ -375,8 +375,16 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
 }
 
 // G_l = dZ_l W_l^T (+ skip gradient), dZ_{l-1} = G_l * act'(Z_{l-1});  l >= 1
+// Row blocks of 32 that the dgrad GEMM of layer l writes fused column sums for.
+int dgrad_row_blocks(const et_stack* s, int l) {
+  const int tile_m = s->ly[l].pair_dgrad ? 2 * et::tc::BM : et::tc::BM;
+  return ceil_div(s->M, tile_m) * (tile_m / 32);
+}
+
+// want_colsum: also leave the column sums of dZ_{l-1} (layer l-1's bias gradient) in the bias
+// partial buffer (tensor-core path only).
 template <typename T>
-et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st) {
+et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, bool want_colsum = false) {
   TimedLaunch tl(s, ET_K_DGRAD, st);
   const LayerRT& L = s->ly[l];
   const LayerRT& P = s->ly[l - 1];
@@ -396,6 +404,7 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st) {
       et::DgradEpiS<1> epi;
       epi.has_in[0] = need_skip; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = false; epi.act_prev = P.act;
+      epi.colsum = want_colsum ? (float*)s->at(s->off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = skip; em.out[0] = gout; em.in[1] = gout; em.out[1] = gout;
       return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
     }
@@ -403,12 +412,14 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st) {
       et::DgradEpiS<1> epi;
       epi.has_in[0] = true; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = true; epi.act_prev = P.act;
+      epi.colsum = want_colsum ? (float*)s->at(s->off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = zmap; em.out[0] = dzout; em.in[1] = zmap; em.out[1] = dzout;
       return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
     }
     et::DgradEpiS<2> epi;                                     // both G_l and dZ_{l-1}
     epi.has_in[0] = need_skip; epi.has_in[1] = true; epi.has_out[0] = need_G; epi.has_out[1] = true;
     epi.mul_act = false; epi.act_prev = P.act;
+    epi.colsum = want_colsum ? (float*)s->at(s->off_biaspart) : nullptr; epi.ld = L.K;
     em.in[0] = skip; em.out[0] = gout; em.in[1] = zmap; em.out[1] = dzout;
     return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
   } else {
@@ -474,17 +485,22 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   return after_launch();
 }
 
+// fused_chunks > 0: the column partials (that many row blocks) were already written by the dgrad
+// GEMM of the layer above; only the finishing kernel runs.
 template <typename T>
 et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
-                          int* launches, cudaStream_t st) {
+                          int* launches, cudaStream_t st, int fused_chunks = 0) {
   TimedLaunch tl(s, ET_K_BGRAD, st);
   const LayerRT& L = s->ly[l];
   float* part = (float*)s->at(s->off_biaspart);
-  const int chunks = ceil_div(s->M, et::kColsumRows);
-  dim3 grid(ceil_div(L.Nw, 256), chunks), block(32, 8);
-  et::colsum_partial_kernel<T><<<grid, block, 0, st>>>(dz_src<T>(s, l, dY), (int)s->M, L.Nw, part);
-  ET_TRY(after_launch());
-  ++*launches;
+  int chunks = fused_chunks;
+  if (fused_chunks == 0) {
+    chunks = ceil_div(s->M, et::kColsumRows);
+    dim3 grid(ceil_div(L.Nw, 256), chunks), block(32, 8);
+    et::colsum_partial_kernel<T><<<grid, block, 0, st>>>(dz_src<T>(s, l, dY), (int)s->M, L.Nw, part);
+    ET_TRY(after_launch());
+    ++*launches;
+  }
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l + 1];
   et::bias_finish_kernel<T><<<L.imp_count_b, dim3(32, 8), 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
                                                                        (T*)L.b, lr, sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0);
@@ -554,8 +570,15 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
     for (int l = L - 1; l >= d; --l) {
       const LayerRT& Y = s->ly[l];
       const double gemm = 2.0 * (double)s->M * Y.K * Y.N;
+      if (mask[2 * l + 1]) {
+        // On the tensor-core path the column partials of dZ_l were left by dgrad(l+1) one
+        // iteration ago; they must be consumed before dgrad(l) reuses the buffer for dZ_{l-1}.
+        const int fused = (is_bf16<T>::value && l < L - 1) ? dgrad_row_blocks(s, l + 1) : 0;
+        ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
+                                  delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, st, fused));
+      }
       if (l > d) {                        // reads the old W_l: must precede this layer's update
-        ET_TRY(run_dgrad_layer<T>(s, l, dY, st));
+        ET_TRY(run_dgrad_layer<T>(s, l, dY, st, mask[2 * (l - 1) + 1] != 0));
         ++launches;
         flops += gemm;
       }
@@ -563,10 +586,6 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         ET_TRY(run_wgrad_layer<T>(s, l, dY, grads ? grads[2 * l] : nullptr,
                                   delta ? (const T*)delta[2 * l] : nullptr, sgd, lr, &launches, st));
         flops += gemm;
-      }
-      if (mask[2 * l + 1]) {
-        ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
-                                  delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, st));
       }
     }
     if (delta != nullptr) {
@@ -702,6 +721,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     }
     max_partial = std::max(max_partial, (size_t)y.split * y.K * y.N * sizeof(float));
     max_biaspart = std::max(max_biaspart, (size_t)chunks * y.Nw * sizeof(float));
+    max_biaspart = std::max(max_biaspart, (size_t)(ceil_div(M, 256) * 8 + 8) * std::max(y.Nw, y.K) * sizeof(float));
     y.imp_count_w = ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
     y.imp_count_b = ceil_div(y.N, et::kBiasCols);
     s->imp_offs[2 * l] = imp_total; s->imp_counts[2 * l] = y.imp_count_w; imp_total += y.imp_count_w;

@@ -674,6 +674,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             epi.combine(col0 + h * 32, p.cols - (col0 + h * 32), v, s0, s1);
             if (epi.has_out[0]) sts_row32(buf0, trow, h, s0);
             if (SLOTS > 1 && epi.has_out[SLOTS - 1]) sts_row32(buf1, trow, h, s1);
+            epi.column_sums((m0 >> 5) + quad, col0 + h * 32, p.cols - (col0 + h * 32), s0, s1, lane);
           }
           fence_async_smem();                       // generic-proxy writes -> visible to the TMA engine
           mbar_arrive(out_ready_bar(g, b));         // 128 arrivals: the group's TMA thread may store the chunk
