@@ -48,6 +48,22 @@ def _peaks():
     return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
 
 
+def _dgrad_traffic():
+    """DRAM bytes per dgrad launch from the committed ncu capture, or None once the GEMM sources
+    have changed since the counters were taken."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "dgrad_dram_traffic.json")) as f:
+            rec = json.load(f)
+        h = hashlib.sha256()
+        for name in ("gemm_tc.cuh", "epilogue.cuh"):
+            with open(os.path.join(ROOT, "paper_2312_14227_b200", "csrc", name), "rb") as f:
+                h.update(f.read())
+        return rec["bytes_per_launch"] if h.hexdigest() == rec["source_sha256"] else None
+    except (OSError, KeyError, ValueError):
+        return None
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
 
@@ -265,7 +281,8 @@ def run_own(args):
     e2e_value = world * flops / (e2e_ms * 1e-3) / 1e12
     clocks = sampler.stop()     # sampled from the full-backprop run to the end of the end-to-end run
 
-    # per-kernel-class device time over the same steps (event pair around every launch)
+    # per-kernel-class device time over the same steps (event pair around every launch; while
+    # this is on, the library keeps all kernels on one stream so that a pair brackets one kernel)
     et.et_timing_enable(stack, True)
     inst_ms, _ = timed(lambda: step(w.mask), args.steps, 1)
     classes = et.et_timing_read(stack)
@@ -340,7 +357,8 @@ def run_own(args):
         "gpu_launches": int(launches),
         "roofline": {"kernel": "gemm_tc_kernel<dgrad>", "bound": "tensor", "achieved": dg_tf,
                      "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": dg_tf / peaks["tf_sustained"],
-                     "peak_source": peaks["source"] + " (sustained cuBLAS bf16)", "traffic": None},
+                     "peak_source": peaks["source"] + " (sustained cuBLAS bf16)", "traffic": _dgrad_traffic(),
+                     "traffic_note": "DRAM bytes per launch, mean over the dgrad GEMMs of one block (ncu, cold cache)"},
         "kernels": kernels,
     }
     if world == 1:

@@ -148,7 +148,11 @@ et_status et_loss_mse_grad(et_stack* s, const void* y, const void* target, void*
  *   report     host, optional.
  * Nothing is launched for layers below the deepest selected one; with an empty mask
  * nothing is launched at all except zeroing importance_dev.  Needs a preceding
- * et_forward_stack on the same stack. */
+ * et_forward_stack on the same stack.
+ * The error-gradient chain runs on an internal high-priority stream that forks from and joins
+ * back into `stream` inside the call (weight gradients fill the SMs the chain leaves idle); to
+ * the caller everything is ordered on `stream`.  ET_SINGLE_STREAM=1 in the environment keeps
+ * all kernels on `stream`. */
 et_status et_backward_elastic(et_stack* s, const void* dY, const uint8_t* mask, int32_t n_tensors,
                               float* const* grads, const void* const* delta,
                               float* importance_dev, uint32_t flags, float lr,
@@ -245,7 +249,9 @@ typedef enum {
 } et_kernel_class;
 
 /* on != 0: every kernel this stack launches from now on is bracketed by a pair of CUDA
- * events on its stream (host objects; no device memory).  on == 0: stop and drop them. */
+ * events on its stream (host objects; no device memory), and the backward pass keeps all its
+ * kernels on the caller's stream, one after the other, so that a pair brackets exactly one
+ * kernel's run.  on == 0: stop and drop them. */
 et_status et_timing_enable(et_stack* s, int32_t on);
 /* Waits for the recorded events, adds up device time (milliseconds) and launch counts per
  * class into ms[ET_K_CLASSES] / launches[ET_K_CLASSES] (either may be NULL), and clears the

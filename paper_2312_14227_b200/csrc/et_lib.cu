@@ -160,6 +160,11 @@ struct et_stack {
   const void* map_dy_ptr = nullptr;
   const void* map_y_ptr = nullptr;
   bool delta_is_snapshot = false;      // per call: the delta tensors hold a weight snapshot
+  // second stream: the error-gradient chain runs here while weight gradients run on the caller's
+  cudaStream_t chain_stream = nullptr;
+  std::vector<cudaEvent_t> chain_ev;   // [l] = dgrad(l) finished; [L] = top-layer dZ ready; [L+1] = join
+  cudaEvent_t fork_ev = nullptr;
+  int two_streams = -1;                // -1 = not set up yet, 0 = off, 1 = on
   // optional per-kernel timing
   bool timing = false;
   struct Timed { int cls; cudaEvent_t e0, e1; };
@@ -447,7 +452,7 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
 // dW_l = a_l^T dZ_l as split partials, then the reducer with grad / importance / SGD.
 template <typename T>
 et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
-                          int* launches, cudaStream_t st) {
+                          int* launches, cudaStream_t st, cudaEvent_t before_reduce = nullptr) {
   const LayerRT& L = s->ly[l];
   float* partial = (float*)s->at(s->off_partial);
   const size_t count = (size_t)L.K * L.N;
@@ -476,6 +481,7 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   }
   ++*launches;
   if (grad == nullptr && delta == nullptr && !sgd) return ET_OK;     // nothing consumes g
+  if (before_reduce != nullptr) CU_TRY(cudaStreamWaitEvent(st, before_reduce, 0));
   TimedLaunch tl(s, ET_K_WGRAD_REDUCE, st);
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
   et::wgrad_reduce_kernel<T><<<L.imp_count_w, et::kEltThreads, 0, st>>>(partial, split, count, count, grad, delta, imp,
@@ -523,6 +529,36 @@ et_status check_ready(const et_stack* s, const uint8_t* mask, int n_tensors) {
   return ET_OK;
 }
 
+// The dgrad chain dZ_{L-1} -> dZ_{L-2} -> ... is the critical path of the backward pass; weight
+// gradients only hang off it.  Running the chain on its own high-priority stream lets weight-gradient
+// CTAs fill the SMs a chain kernel leaves idle in its last wave and during its prologue and drain.
+// Streams and events are host objects (no device memory).  ET_SINGLE_STREAM=1 turns this off.
+bool setup_two_streams(et_stack* s) {
+  if (s->two_streams >= 0) return s->two_streams == 1;
+  s->two_streams = 0;
+  if (getenv("ET_SINGLE_STREAM") != nullptr) return false;
+  int least = 0, greatest = 0;
+  if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+  if (cudaStreamCreateWithPriority(&s->chain_stream, cudaStreamNonBlocking, greatest) != cudaSuccess) {
+    (void)cudaGetLastError();
+    s->chain_stream = nullptr;
+    return false;
+  }
+  s->chain_ev.assign(s->L + 2, nullptr);
+  bool ok = cudaEventCreateWithFlags(&s->fork_ev, cudaEventDisableTiming) == cudaSuccess;
+  for (auto& e : s->chain_ev) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) { (void)cudaGetLastError(); return false; }
+  s->two_streams = 1;
+  return true;
+}
+void destroy_two_streams(et_stack* s) {
+  for (auto e : s->chain_ev) if (e != nullptr) cudaEventDestroy(e);
+  s->chain_ev.clear();
+  if (s->fork_ev != nullptr) cudaEventDestroy(s->fork_ev);
+  if (s->chain_stream != nullptr) cudaStreamDestroy(s->chain_stream);
+  s->fork_ev = nullptr; s->chain_stream = nullptr; s->two_streams = -1;
+}
+
 template <typename T>
 et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float* const* grads,
                         const void* const* delta, float* importance_dev, uint32_t flags, float lr,
@@ -558,15 +594,22 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         s->map_dy_ptr = dY;
       }
     }
+    const bool two = !s->timing && setup_two_streams(s);   // per-kernel timing wants kernels one at a time
+    cudaStream_t cs = two ? s->chain_stream : st;          // stream of the error-gradient chain
+    if (two) {
+      CU_TRY(cudaEventRecord(s->fork_ev, st));
+      CU_TRY(cudaStreamWaitEvent(cs, s->fork_ev, 0));
+    }
     const LayerRT& top = s->ly[L - 1];
     if (top.act != ET_ACT_NONE) {
-      TimedLaunch tl(s, ET_K_OTHER, st);
+      TimedLaunch tl(s, ET_K_OTHER, cs);
       const size_t count = (size_t)s->M * top.N;
-      et::act_backward_kernel<T><<<ceil_div(count, et::kEltThreads * et::kVec), et::kEltThreads, 0, st>>>(
+      et::act_backward_kernel<T><<<ceil_div(count, et::kEltThreads * et::kVec), et::kEltThreads, 0, cs>>>(
           (const T*)dY, (const T*)s->at(top.off_Z), (T*)s->at(top.off_dZ), count, top.act);
       ET_TRY(after_launch());
       ++launches;
     }
+    if (two) CU_TRY(cudaEventRecord(s->chain_ev[L], cs));  // dZ_{L-1} is ready
     for (int l = L - 1; l >= d; --l) {
       const LayerRT& Y = s->ly[l];
       const double gemm = 2.0 * (double)s->M * Y.K * Y.N;
@@ -575,18 +618,26 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         // iteration ago; they must be consumed before dgrad(l) reuses the buffer for dZ_{l-1}.
         const int fused = (is_bf16<T>::value && l < L - 1) ? dgrad_row_blocks(s, l + 1) : 0;
         ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
-                                  delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, st, fused));
+                                  delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, cs, fused));
       }
-      if (l > d) {                        // reads the old W_l: must precede this layer's update
-        ET_TRY(run_dgrad_layer<T>(s, l, dY, st, mask[2 * (l - 1) + 1] != 0));
+      if (l > d) {
+        ET_TRY(run_dgrad_layer<T>(s, l, dY, cs, mask[2 * (l - 1) + 1] != 0));
+        if (two) CU_TRY(cudaEventRecord(s->chain_ev[l], cs));   // dZ_{l-1} ready, W_l no longer needed
         ++launches;
         flops += gemm;
       }
       if (mask[2 * l]) {
+        // needs dZ_l (left by dgrad(l+1)); its update of W_l has to wait until dgrad(l) has read W_l
+        if (two) CU_TRY(cudaStreamWaitEvent(st, s->chain_ev[l + 1], 0));
         ET_TRY(run_wgrad_layer<T>(s, l, dY, grads ? grads[2 * l] : nullptr,
-                                  delta ? (const T*)delta[2 * l] : nullptr, sgd, lr, &launches, st));
+                                  delta ? (const T*)delta[2 * l] : nullptr, sgd, lr, &launches, st,
+                                  (two && l > d) ? s->chain_ev[l] : nullptr));
         flops += gemm;
       }
+    }
+    if (two) {
+      CU_TRY(cudaEventRecord(s->chain_ev[L + 1], cs));
+      CU_TRY(cudaStreamWaitEvent(st, s->chain_ev[L + 1], 0));
     }
     if (delta != nullptr) {
       TimedLaunch tl(s, ET_K_OTHER, st);
@@ -745,6 +796,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
 et_status et_stack_destroy(et_stack* s) {
   if (s == nullptr) return ET_ERR_INVALID_ARG;
   et_timing_enable(s, 0);
+  destroy_two_streams(s);
   delete s;
   return ET_OK;
 }
