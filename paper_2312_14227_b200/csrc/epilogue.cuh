@@ -146,8 +146,17 @@ struct DgradEpiS {
   __device__ __forceinline__ void combine(int, int, float (&v)[32], float (&s0)[32], float (&s1)[32]) const {
     if constexpr (SLOTS == 1) {
       if (mul_act) {
+        if (act_prev == kActGelu) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) s0[i] = v[i] * act_grad_fast(s0[i], act_prev);
+          for (int i = 0; i < 32; i += 2) {
+            const float2 d = gelu_tanh_grad_x2(s0[i], s0[i + 1]);
+            s0[i] = v[i] * d.x;
+            s0[i + 1] = v[i + 1] * d.y;
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) s0[i] = v[i] * act_grad_fast(s0[i], act_prev);
+        }
       } else {
         const bool skip = has_in[0];
 #pragma unroll
