@@ -371,6 +371,82 @@ def run_own(args):
         dist.destroy_process_group()
 
 
+def run_side(args):
+    """Side reports for the other workload shapes (not the benchmark line): one JSON line each.
+    resnet: ResNet-50 conv4_x 1x1 stack, elastic vs full step time (launch-bound GEMMs).
+    schedule: ViT-L-shaped stack, the 200-iteration elastic schedule (10-step all-tensor window every
+    50 steps, importances from the weight change over the window, selector at rho = 0.4 on
+    measured per-tensor times) against 200 full-backprop iterations."""
+    import torch
+    import paper_2312_14227_b200 as et
+    from paper_2312_14227_b200.elastic_loop import ElasticLoop
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    w = wl.resnet_1x1() if args.workload == "resnet" else wl.vit_l()
+    tdt = torch.bfloat16
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
+    stack = et.et_stack_create(w.layers, w.M, w.dtype)
+    W, b = [to_dev(a) for a in w.W], [to_dev(a) for a in w.b]
+    ws = torch.empty(et.et_stack_workspace_bytes(stack), dtype=torch.uint8, device=dev)
+    et.et_stack_bind(stack, W, b, ws)
+    x, target = to_dev(w.x), to_dev(w.target)
+    y = torch.empty((w.M, w.layers[-1].out_width), dtype=tdt, device=dev)
+    dY = torch.empty_like(y)
+    et.et_forward_stack(stack, x, y)
+    et.et_loss_mse_grad(stack, y, target, dY, None)
+    torch.cuda.synchronize()
+    if args.workload == "resnet":
+        rep = et.Report(w.L)
+        delta = [to_dev(d) for d in wl.draw_delta(w, 5)]
+        imp = torch.zeros(2 * w.L, dtype=torch.float32, device=dev)
+
+        def timed(mask):
+            for _ in range(5):
+                et.et_backward_elastic(stack, dY, mask, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(args.steps):
+                et.et_backward_elastic(stack, dY, mask, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps, rep.flops_executed, rep.launches
+
+        ms, fl, n = timed(w.mask)
+        fms, ffl, fn = timed(np.ones(2 * w.L, dtype=np.uint8))
+        print(json.dumps({"report": "resnet50_conv4_1x1_bf16", "elastic_ms": ms, "elastic_tflops": fl / ms / 1e9,
+                          "elastic_launches": n, "full_ms": fms, "full_tflops": ffl / fms / 1e9, "full_launches": fn,
+                          "selected_tensors": int(w.mask.sum())}))
+        return
+    t_dw, t_dy, t_fwd = et.et_profile_costs(stack, x, y, dY, iters=10)
+    loop = ElasticLoop(stack, W, b, x, target, w.lr, 50, 10, 0.4, t_dw, t_dy, t_fwd=t_fwd, Tq=1000, master=True)
+    W0, b0 = [t.clone() for t in W], [t.clone() for t in b]
+
+    def restore():
+        for dst, src in zip(W + b, W0 + b0):
+            dst.copy_(src)
+        for dst, src in zip(loop.W32 + loop.b32, W0 + b0):
+            dst.copy_(src)
+
+    loop.run(10, elastic=False)                                   # warm-up
+    restore()
+    full = loop.run(200, elastic=False, time_steps=True)
+    restore()
+    el = loop.run(200, elastic=True, time_steps=True)
+    T_full = t_fwd + t_dw.sum() + t_dy.sum()
+    est = [t_fwd + et.et_time_selective(m, t_dw, t_dy) for m in el["masks"]]
+    print(json.dumps({"report": "vit_l_linear_bf16 elastic schedule, 200 iterations", "rho": 0.4,
+                      "full_ms_per_step": full["ms_per_step"], "elastic_ms_per_step": el["ms_per_step"],
+                      "ratio": el["ms_per_step"] / full["ms_per_step"],
+                      "model_estimate_ratio": float(np.mean(est) / T_full),
+                      "selected_tensors_per_period": [int(m.sum()) for m in el["masks"][10::50]],
+                      "selector_ms": el["dp_ms"], "profiled_full_step_ms": float(T_full),
+                      "loss_first_last": [float(el["losses"][0]), float(el["losses"][-1])],
+                      "note": "includes forward, loss, host selector and snapshot copies; bf16 storage "
+                              "with fp32 master weights"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -380,9 +456,13 @@ def main():
     ap.add_argument("--blocks", type=int, default=12, help="transformer blocks of the stack (12 = the benchmark workload)")
     ap.add_argument("--profile", action="store_true",
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "schedule"],
+                    help="vit_b = the benchmark line; resnet / schedule = side reports for the other shapes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup
-    if args.impl == "reference":
+    if args.workload != "vit_b":
+        run_side(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_own(args)

@@ -115,6 +115,16 @@ et_status et_stack_workspace_bytes(const et_stack* s, size_t* bytes);
 et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* workspace,
                         size_t workspace_bytes, void* stream);
 
+/* Optional fp32 master copies for ET_BF16 stacks (the paper trains in fp32, Section 7; bf16
+ * storage alone rounds an update lr*g away when it is below half an ulp of the weight).
+ * W32, b32: host arrays of L device float* holding the same values as W, b (caller-owned,
+ * caller-initialised), or both NULL to detach.  While attached, every masked update
+ * (ET_FLAG_FUSE_SGD, et_sgd_masked) is applied to the master in fp32 and the bf16 tensor is
+ * rewritten as its rounding; ET_FLAG_DELTA_IS_SNAPSHOT then expects fp32 snapshots of the
+ * masters in `delta`.  Unselected tensors and their masters are never written.  Call after
+ * et_stack_bind (which detaches). */
+et_status et_stack_bind_master(et_stack* s, float* const* W32, float* const* b32);
+
 /* ---- forward and loss (precede the hot path; Eq. 3's T_forward) -------------------- */
 
 /* x: device [M x in_features(0)], y: device [M x width(a_L)], storage dtype.  Saves every

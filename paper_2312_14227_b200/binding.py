@@ -44,6 +44,7 @@ _SIGS = {
     "et_stack_destroy": [_vp],
     "et_stack_workspace_bytes": [_vp, C.POINTER(C.c_size_t)],
     "et_stack_bind": [_vp, _vp, _vp, _vp, C.c_size_t, _vp],
+    "et_stack_bind_master": [_vp, _vp, _vp],
     "et_forward_stack": [_vp, _vp, _vp, _vp],
     "et_loss_mse_grad": [_vp, _vp, _vp, _vp, _vp, _vp],
     "et_backward_elastic": [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _u32, _f32, _vp, _vp],
@@ -220,6 +221,12 @@ def et_stack_bind(s: Stack, W, b, workspace, workspace_bytes: Optional[int] = No
     s._keep = [list(W), list(b), workspace]          # keep the tensors alive while bound
     _check(_lib.et_stack_bind(s.handle, _ptr_array(W, s.L), _ptr_array(b, s.L), _ptr(workspace),
                               workspace_bytes, _stream_ptr(stream)), "et_stack_bind")
+
+
+def et_stack_bind_master(s: Stack, W32, b32):
+    s._keep_master = [list(W32), list(b32)] if W32 is not None else None
+    _check(_lib.et_stack_bind_master(s.handle, _ptr_array(W32, s.L) if W32 is not None else None,
+                                     _ptr_array(b32, s.L) if b32 is not None else None), "et_stack_bind_master")
 
 
 def et_forward_stack(s: Stack, x, y, stream=None):

@@ -126,6 +126,8 @@ struct LayerRT {
   int consumer = -1;        // layer whose residual reads a_l (its output gradient joins G_l), or -1
   void* W = nullptr;
   void* b = nullptr;
+  float* W32 = nullptr;     // optional fp32 master copies (et_stack_bind_master)
+  float* b32 = nullptr;
   size_t off_a_out = 0;     // a_{l+1}           (unused for the last layer: that is the caller's y)
   size_t off_Z = 0;         // Z_l               (act != none)
   size_t off_G_out = 0;     // G_{l+1}           (unused for the last layer: that is the caller's dY)
@@ -486,7 +488,7 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
   et::wgrad_reduce_kernel<T><<<L.imp_count_w, et::kEltThreads, 0, st>>>(partial, split, count, count, grad, delta, imp,
                                                                         (T*)L.W, lr, sgd ? 1 : 0,
-                                                                        s->delta_is_snapshot ? 1 : 0);
+                                                                        s->delta_is_snapshot ? 1 : 0, L.W32);
   ++*launches;
   return after_launch();
 }
@@ -509,7 +511,7 @@ et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   }
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l + 1];
   et::bias_finish_kernel<T><<<L.imp_count_b, dim3(32, 8), 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
-                                                                       (T*)L.b, lr, sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0);
+                                                                       (T*)L.b, lr, sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0, L.b32);
   ++*launches;
   return after_launch();
 }
@@ -816,7 +818,7 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   cudaStream_t st = (cudaStream_t)stream;
   s->bound = false;
   s->ws = (char*)workspace;
-  for (int l = 0; l < s->L; ++l) { s->ly[l].W = W[l]; s->ly[l].b = b[l]; }
+  for (int l = 0; l < s->L; ++l) { s->ly[l].W = W[l]; s->ly[l].b = b[l]; s->ly[l].W32 = nullptr; s->ly[l].b32 = nullptr; }
   if (s->dtype == ET_BF16) {
     for (int l = 0; l < s->L; ++l) {
       LayerRT& y = s->ly[l];
@@ -841,6 +843,22 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   s->map_dy_ptr = nullptr;
   s->map_y_ptr = nullptr;
   s->x = nullptr;
+  return ET_OK;
+}
+
+et_status et_stack_bind_master(et_stack* s, float* const* W32, float* const* b32) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  if (s->dtype != ET_BF16) return ET_ERR_DTYPE;
+  if ((W32 == nullptr) != (b32 == nullptr)) return ET_ERR_INVALID_ARG;
+  if (W32 != nullptr)
+    for (int l = 0; l < s->L; ++l)
+      if (W32[l] == nullptr || b32[l] == nullptr || ((uintptr_t)W32[l] & 15) || ((uintptr_t)b32[l] & 15))
+        return ET_ERR_INVALID_ARG;
+  for (int l = 0; l < s->L; ++l) {
+    s->ly[l].W32 = W32 ? W32[l] : nullptr;
+    s->ly[l].b32 = b32 ? b32[l] : nullptr;
+  }
   return ET_OK;
 }
 
@@ -946,9 +964,10 @@ et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
     const bool is_w = (t & 1) == 0;
     const size_t count = is_w ? (size_t)y.K * y.N : (size_t)y.N;
     void* w = is_w ? y.W : y.b;
+    float* m = is_w ? y.W32 : y.b32;
     const int blocks = ceil_div(count, et::kEltThreads * et::kVec);
-    if (s->dtype == ET_BF16) et::sgd_kernel<bf16><<<blocks, et::kEltThreads, 0, st>>>((bf16*)w, grads[t], count, lr);
-    else                     et::sgd_kernel<float><<<blocks, et::kEltThreads, 0, st>>>((float*)w, grads[t], count, lr);
+    if (s->dtype == ET_BF16) et::sgd_kernel<bf16><<<blocks, et::kEltThreads, 0, st>>>((bf16*)w, grads[t], count, lr, m);
+    else                     et::sgd_kernel<float><<<blocks, et::kEltThreads, 0, st>>>((float*)w, grads[t], count, lr, m);
     ET_TRY(after_launch());
   }
   return ET_OK;

@@ -18,16 +18,18 @@ constexpr int kColsumRows = 128;                // rows per column-sum chunk
 //   imp_part[b] <- sum over this block of g * dw        if delta != nullptr   (Eq. 2);
 //                  dw = delta, or W - delta when delta holds a snapshot of W
 //   W           <- W - lr * g                  if do_sgd   (fp32 arithmetic, one rounding)
+//   master != nullptr: the weight lives in fp32 there (W is its rounded copy): the update and
+//                  the snapshot difference use it, and a snapshot `delta` is fp32 as well
 template <typename T>
 __global__ void __launch_bounds__(kEltThreads)
 wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_t count,
                     float* grad /* may alias partial: each thread reads its elements before writing them */, const T* __restrict__ delta, float* __restrict__ imp_part,
-                    T* __restrict__ W, float lr, int do_sgd, int delta_is_snapshot) {
+                    T* __restrict__ W, float lr, int do_sgd, int delta_is_snapshot, float* __restrict__ master) {
   const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
   float dot = 0.0f;
   if (i0 < count) {
     const int n = (int)min((size_t)kVec, count - i0);
-    float g[kVec], t[kVec];
+    float g[kVec], t[kVec], w[kVec];
     load_seg<kVec>(partial + i0, n, g);
     for (int s = 1; s < splits; ++s) {
       load_seg<kVec>(partial + (size_t)s * split_stride + i0, n, t);
@@ -35,22 +37,27 @@ wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_
       for (int i = 0; i < kVec; ++i) g[i] += t[i];
     }
     if (grad != nullptr) store_seg<kVec>(grad + i0, n, g);
+    if (do_sgd || (delta != nullptr && delta_is_snapshot)) {      // the current weight is needed
+      if (master != nullptr) load_seg<kVec>(master + i0, n, w);
+      else load_seg<kVec>(W + i0, n, w);
+    }
     if (delta != nullptr) {
-      load_seg<kVec>(delta + i0, n, t);
       if (delta_is_snapshot) {                        // dw = current weight - weight at the window start
-        float w[kVec];
-        load_seg<kVec>(W + i0, n, w);
+        if (master != nullptr) load_seg<kVec>(reinterpret_cast<const float*>(delta) + i0, n, t);
+        else load_seg<kVec>(delta + i0, n, t);
 #pragma unroll
         for (int i = 0; i < kVec; ++i) t[i] = w[i] - t[i];
+      } else {
+        load_seg<kVec>(delta + i0, n, t);
       }
 #pragma unroll
       for (int i = 0; i < kVec; ++i) dot = fmaf(g[i], t[i], dot);
     }
     if (do_sgd) {
-      load_seg<kVec>(W + i0, n, t);
 #pragma unroll
-      for (int i = 0; i < kVec; ++i) t[i] = fmaf(-lr, g[i], t[i]);
-      store_seg<kVec>(W + i0, n, t);
+      for (int i = 0; i < kVec; ++i) w[i] = fmaf(-lr, g[i], w[i]);
+      if (master != nullptr) store_seg<kVec>(master + i0, n, w);
+      store_seg<kVec>(W + i0, n, w);
     }
   }
   if (delta != nullptr) {
@@ -114,7 +121,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
                    float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
-                   T* __restrict__ b, float lr, int do_sgd, int delta_is_snapshot) {
+                   T* __restrict__ b, float lr, int do_sgd, int delta_is_snapshot, float* __restrict__ master) {
   __shared__ float sm[8][kBiasCols + 1];
   const int j = blockIdx.x * kBiasCols + threadIdx.x;
   float g = 0.0f;
@@ -131,8 +138,21 @@ bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int co
 #pragma unroll
       for (int y = 0; y < 8; ++y) g += sm[y][threadIdx.x];
       if (grad != nullptr) grad[j] = g;
-      if (delta != nullptr) dot = g * (delta_is_snapshot ? to_f32(b[j]) - to_f32(delta[j]) : to_f32(delta[j]));
-      if (do_sgd) b[j] = from_f32<T>(fmaf(-lr, g, to_f32(b[j])));
+      float w = 0.0f;
+      if (do_sgd || (delta != nullptr && delta_is_snapshot)) w = master != nullptr ? master[j] : to_f32(b[j]);
+      if (delta != nullptr) {
+        float dw;
+        if (delta_is_snapshot)
+          dw = w - (master != nullptr ? reinterpret_cast<const float*>(delta)[j] : to_f32(delta[j]));
+        else
+          dw = to_f32(delta[j]);
+        dot = g * dw;
+      }
+      if (do_sgd) {
+        w = fmaf(-lr, g, w);
+        if (master != nullptr) master[j] = w;
+        b[j] = from_f32<T>(w);
+      }
     }
     if (delta != nullptr) {                           // one warp: fixed shuffle tree
       dot = warp_sum(dot);
@@ -178,15 +198,17 @@ importance_kernel(const float* __restrict__ grad, const T* __restrict__ delta, s
 // ---- stand-alone masked SGD on one selected tensor -----------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(kEltThreads)
-sgd_kernel(T* __restrict__ w, const float* __restrict__ grad, size_t count, float lr) {
+sgd_kernel(T* __restrict__ w, const float* __restrict__ grad, size_t count, float lr, float* __restrict__ master) {
   const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
   if (i0 >= count) return;
   const int n = (int)min((size_t)kVec, count - i0);
   float g[kVec], t[kVec];
   load_seg<kVec>(grad + i0, n, g);
-  load_seg<kVec>(w + i0, n, t);
+  if (master != nullptr) load_seg<kVec>(master + i0, n, t);
+  else load_seg<kVec>(w + i0, n, t);
 #pragma unroll
   for (int i = 0; i < kVec; ++i) t[i] = fmaf(-lr, g[i], t[i]);
+  if (master != nullptr) store_seg<kVec>(master + i0, n, t);
   store_seg<kVec>(w + i0, n, t);
 }
 

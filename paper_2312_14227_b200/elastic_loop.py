@@ -16,7 +16,7 @@ from . import binding as et
 
 class ElasticLoop:
     def __init__(self, stack, W, b, x, target, lr, period, window, rho, t_dw, t_dy, t_fwd=0.0, Tq=1000,
-                 variant=et.ET_COST_STRICT, stream=None):
+                 variant=et.ET_COST_STRICT, stream=None, master=False):
         self.stack, self.W, self.b, self.x, self.target = stack, W, b, x, target
         self.lr, self.period, self.window, self.rho = float(lr), int(period), int(window), float(rho)
         self.t_dw, self.t_dy, self.t_fwd, self.Tq, self.variant = t_dw, t_dy, float(t_fwd), int(Tq), variant
@@ -26,7 +26,14 @@ class ElasticLoop:
         self.y = torch.empty((stack.M, stack.out_width), dtype=x.dtype, device=dev)
         self.dY = torch.empty_like(self.y)
         self.params = [t for pair in zip(W, b) for t in pair]
-        self.snap = [torch.empty_like(p) for p in self.params]
+        # master=True: fp32 master copies of bf16 parameters; updates and snapshots then live in fp32
+        self.master = None
+        if master:
+            self.W32 = [t.float() for t in W]
+            self.b32 = [t.float() for t in b]
+            et.et_stack_bind_master(stack, self.W32, self.b32)
+            self.master = [t for pair in zip(self.W32, self.b32) for t in pair]
+        self.snap = [torch.empty_like(p) for p in (self.master or self.params)]
         self.imp = torch.zeros(2 * self.L, dtype=torch.float32, device=dev)
         self.mask = np.ones(2 * self.L, dtype=np.uint8)
 
@@ -45,7 +52,7 @@ class ElasticLoop:
             phase = step % self.period
             if elastic and phase == 0:
                 self.mask = np.ones(2 * self.L, dtype=np.uint8)
-                for s_, p_ in zip(self.snap, self.params):
+                for s_, p_ in zip(self.snap, self.master or self.params):
                     s_.copy_(p_)
             et.et_forward_stack(self.stack, self.x, self.y, stream=self.stream)
             et.et_loss_mse_grad(self.stack, self.y, self.target, self.dY, losses[step:step + 1], stream=self.stream)
@@ -54,6 +61,7 @@ class ElasticLoop:
                 et.et_backward_elastic(self.stack, self.dY, self.mask, None, self.snap, self.imp,
                                        flags | et.ET_FLAG_DELTA_IS_SNAPSHOT, self.lr, None, stream=self.stream)
                 S = self.imp.cpu().numpy().astype(np.float64)          # synchronises
+                S = np.nan_to_num(S, nan=0.0, posinf=0.0, neginf=0.0)  # a diverged run must not stop the selector
                 evaluations.append(S)
                 import time
                 t0 = time.perf_counter()

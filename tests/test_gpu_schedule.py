@@ -48,6 +48,32 @@ def test_schedule_fp32_reduced_twin_matches_oracle_trajectory():
         assert np.abs(h.to_np(p) - final[t]).max() <= 1e-3
 
 
+def test_schedule_bf16_with_master_weights_follows_oracle():
+    import gpu_harness as h
+    # bf16 storage and tensor-core kernels, fp32 master weights: the schedule still follows the
+    # float64 run closely (without master weights most updates would be rounded away)
+    layers = wl.vit_blocks(4, 256, 512)
+    w = wl.small_stack(layers, 394, wl.DT_BF16, 23, w_std=0.02)
+    steps, period, window, rho, Tq = 60, 30, 6, 0.5, 300
+    t_dw, t_dy = flop_costs(w.layers, w.M)
+    ref = orc.train_schedule(w.layers, w.W, w.b, w.x, w.target, w.lr, steps, period, window, rho, t_dw, t_dy, Tq=Tq)
+    run = h.GpuRun(w)
+    loop = ElasticLoop(run.stack, run.W, run.b, run.x, run.target, w.lr, period, window, rho, t_dw, t_dy, Tq=Tq,
+                       master=True)
+    got = loop.run(steps)
+    assert et.et_device_status(run.stack) == et.ET_OK
+    np.testing.assert_allclose(got["losses"], ref["losses"], rtol=2e-2)
+    assert got["losses"][-1] < got["losses"][0]
+    for S_gpu, S_ref in zip(got["importances"], ref["importances"]):
+        assert np.abs(S_gpu - S_ref).max() <= 5e-2 * np.abs(S_ref).max()
+    final = orc.tensors_of(ref["W"], ref["b"])
+    for t, p in enumerate(loop.master):
+        assert np.abs(h.to_np(p) - final[t]).max() <= 2e-3
+    # the bf16 tensors are the roundings of their masters
+    for p16, p32 in zip(run.params(), loop.master):
+        assert torch.equal(p16, p32.to(torch.bfloat16))
+
+
 def test_selector_on_measured_costs_bf16():
     import gpu_harness as h
     # per-tensor times measured with CUDA events, seeded Uniform(0,1) importances, budgets as a

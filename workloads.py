@@ -164,7 +164,9 @@ def vit_l(seed: int = 3, params: bool = True, n_blocks: int = 24, tokens: int = 
     rng = np.random.default_rng(seed)
     layers = vit_blocks(n_blocks, d, ffn)
     mask = np.ones(2 * len(layers), dtype=np.uint8)
-    return _finish("vit_l_linear_bf16", layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
+    # std 0.01: without normalisation layers 24 blocks of std-0.02 kernels at d = 1024 multiply the
+    # activation variance by about 1.9 per block (5e6 overall); 0.01 keeps it near 3x overall
+    return _finish("vit_l_linear_bf16", layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.01, params=params)
 
 
 def resnet_1x1(seed: int = 2, p_select: float = 0.5, n_blocks: int = 6, tokens: int = 32 * 14 * 14,
