@@ -415,8 +415,36 @@ def run_side(args):
 
         ms, fl, n = timed(w.mask)
         fms, ffl, fn = timed(np.ones(2 * w.L, dtype=np.uint8))
+
+        # the same elastic step replayed from a CUDA graph (the caller captures the library call)
+        def graph_ms(mask):
+            cap = torch.cuda.Stream()
+            cap.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(cap):
+                et.et_backward_elastic(stack, dY, mask, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep, stream=cap)
+                cap.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=cap):
+                    et.et_backward_elastic(stack, dY, mask, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep, stream=cap)
+                for _ in range(5):
+                    g.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                cap.synchronize()
+                e0.record(cap)
+                for _ in range(args.steps):
+                    g.replay()
+                e1.record(cap)
+                cap.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        try:
+            gms, gfms = graph_ms(w.mask), graph_ms(np.ones(2 * w.L, dtype=np.uint8))
+        except Exception as exc:                      # report, do not hide
+            gms = gfms = None
+            print("graph capture failed:", exc, file=sys.stderr)
         print(json.dumps({"report": "resnet50_conv4_1x1_bf16", "elastic_ms": ms, "elastic_tflops": fl / ms / 1e9,
                           "elastic_launches": n, "full_ms": fms, "full_tflops": ffl / fms / 1e9, "full_launches": fn,
+                          "elastic_graph_ms": gms, "full_graph_ms": gfms,
                           "selected_tensors": int(w.mask.sum())}))
         return
     t_dw, t_dy, t_fwd = et.et_profile_costs(stack, x, y, dY, iters=10)
