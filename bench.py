@@ -180,6 +180,21 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------ own arm
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Step time of the job = the slowest rank's (every rank runs an independent replica)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(flops_per_rank: float, ms: float, world: int) -> float:
+    """Whole-job executed TFLOP/s: all ranks' work over the slowest rank's time."""
+    return world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 def run_own(args):
     import torch
     import paper_2312_14227_b200 as et
@@ -251,11 +266,7 @@ def run_own(args):
             fn()
         e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1) / steps
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1) / steps, dist, dev)
         return ms, et.et_launch_count() - n0
 
     sampler = ClockSampler(local)
@@ -270,7 +281,7 @@ def run_own(args):
     flops = rep.flops_executed
     st = et.et_device_status(stack, stream=stream)
     assert st == et.ET_OK, et.et_status_string(st)
-    value = world * flops / (ms * 1e-3) / 1e12
+    value = aggregate_value(flops, ms, world)
 
     # end to end through the host-buffer entry point: dY comes from pinned host memory and the
     # importances go back to it, inside the timed region
@@ -278,7 +289,7 @@ def run_own(args):
         et.et_backward_elastic_host(stack, dY_host, w.mask, None, delta, imp_host, flags, w.lr, rep, stream=stream)
 
     e2e_ms, _ = timed(step_host, args.steps, args.warmup)
-    e2e_value = world * flops / (e2e_ms * 1e-3) / 1e12
+    e2e_value = aggregate_value(flops, e2e_ms, world)
     clocks = sampler.stop()     # sampled from the full-backprop run to the end of the end-to-end run
 
     # per-kernel-class device time over the same steps (event pair around every launch; while

@@ -271,7 +271,9 @@ et_status et_timing_read(et_stack* s, double* ms, int64_t* launches);
 /* ---- status ------------------------------------------------------------------------ */
 
 /* Synchronises `stream` and reports ET_ERR_TIMEOUT if a kernel's bounded wait gave up,
- * ET_ERR_CUDA if the stream is in error, else ET_OK. */
+ * ET_ERR_CUDA if the stream is in error, else ET_OK.  (The kernels record the first such event
+ * as a non-zero code in the first 32-bit word of the workspace; it stays set until the
+ * workspace is re-bound.) */
 et_status et_device_status(et_stack* s, void* stream);
 const char* et_status_string(et_status st);
 /* cudaError_t of the last failing CUDA call seen by this thread (0 if none). */

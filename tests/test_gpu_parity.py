@@ -180,3 +180,17 @@ def test_bf16_vit_b_full_size_config():
     stats = {}
     h.check_step(w, w.mask, TOL_BF16, stats=stats)
     print("vit_b worst gradient error", stats)
+
+
+def test_device_status_reports_a_recorded_timeout():
+    # every bounded device-side wait that gives up leaves a code in the status word at the start
+    # of the workspace; the host turns it into ET_ERR_TIMEOUT.  The word is planted from the host
+    # here: nothing on the GPU is made to wait.
+    h = _h()
+    w = wl.tiny_mlp()
+    run = h.GpuRun(w)
+    assert et.et_device_status(run.stack) == et.ET_OK
+    run.ws[:4] = torch.tensor([2, 0, 0, 0], dtype=torch.uint8, device=h.DEV)
+    assert et.et_device_status(run.stack) == et.ET_ERR_TIMEOUT
+    run.ws[:4] = 0
+    assert et.et_device_status(run.stack) == et.ET_OK
