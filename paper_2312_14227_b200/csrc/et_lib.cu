@@ -132,6 +132,8 @@ struct LayerRT {
   size_t off_Z = 0;         // Z_l               (act != none)
   size_t off_G_out = 0;     // G_{l+1}           (unused for the last layer: that is the caller's dY)
   size_t off_dZ = 0;        // dZ_l              (act != none)
+  size_t off_biaspart = 0;  // column partials of dZ_l for the bias gradient (own buffer per layer, so
+                            // that finishing a bias never has to be ordered against later GEMMs)
   int split = 1;            // wgrad contraction splits
   int bn_fwd = 256, bn_dgrad = 256, bn_wgrad = 256;   // tile widths chosen per GEMM
   bool pair_fwd = false, pair_dgrad = false, pair_wgrad = false;   // CTA-pair (cta_group::2) tiles
@@ -152,7 +154,7 @@ struct et_stack {
   std::vector<LayerRT> ly;
   std::vector<int> imp_offs, imp_counts;
   size_t ws_bytes = 0;
-  size_t off_status = 0, off_partial = 0, off_biaspart = 0, off_imp_parts = 0, off_imp_offs = 0,
+  size_t off_status = 0, off_partial = 0, off_imp_parts = 0, off_imp_offs = 0,
          off_imp_counts = 0, off_loss_parts = 0, off_dy_stage = 0, off_imp_stage = 0;
   int imp_total = 0;
   char* ws = nullptr;
@@ -162,6 +164,7 @@ struct et_stack {
   const void* map_dy_ptr = nullptr;
   const void* map_y_ptr = nullptr;
   bool delta_is_snapshot = false;      // per call: the delta tensors hold a weight snapshot
+  bool wgrad_one_unit = false;         // per call: weight-gradient CTAs take one unit each and leave
   // second stream: the error-gradient chain runs here while weight gradients run on the caller's
   cudaStream_t chain_stream = nullptr;
   std::vector<cudaEvent_t> chain_ev;   // [l] = dgrad(l) finished; [L] = top-layer dZ ready; [L+1] = join
@@ -260,7 +263,7 @@ const TMaps& dz_map(const et_stack* s, int l) {                                 
 // ---- GEMM launches ---------------------------------------------------------------------------
 template <int BN, bool A_MN, bool B_MN, bool PAIR, class Epi>
 et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em, et::tc::Params p,
-                       const Epi& epi, int sms, cudaStream_t st) {
+                       const Epi& epi, int sms, cudaStream_t st, bool one_unit) {
   auto kern = et::tc::gemm_tc_kernel<BN, A_MN, B_MN, Epi, PAIR>;
   using C = et::tc::Cfg<BN, Epi::kSlots, PAIR>;
   static bool attr_done = false;
@@ -289,31 +292,34 @@ et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::t
   p.tiles_m = ceil_div(p.rows, PAIR ? 2 * et::tc::BM : et::tc::BM);
   p.tiles_n = ceil_div(p.cols, BN);
   const int units = p.tiles_m * p.tiles_n * p.split;
-  cfg.gridDim = PAIR ? dim3(2 * std::min(units, max_clusters)) : dim3(std::min(units, sms));
+  // Persistent by default; one_unit: one work unit per CTA (pair), so that its SMs go back to
+  // the scheduler after every unit instead of after a whole persistent loop.
+  const int workers = one_unit ? units : std::min(units, PAIR ? max_clusters : sms);
+  cfg.gridDim = PAIR ? dim3(2 * workers) : dim3(workers);
   CU_TRY(cudaLaunchKernelEx(&cfg, kern, ma, mb, em, p, epi));
   return after_launch();
 }
 template <bool A_MN, bool B_MN, class Epi>
 et_status launch_tc(int bn, bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em,
-                    const et::tc::Params& p, const Epi& epi, int sms, cudaStream_t st) {
+                    const et::tc::Params& p, const Epi& epi, int sms, cudaStream_t st, bool one_unit = false) {
   if (pair) {
-    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st);
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit);
     if constexpr (!B_MN) {
-      if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st);
+      if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit);
     }
-    return launch_tc_bn<256, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st);
+    return launch_tc_bn<256, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit);
   }
   // staged epilogues take 64 KB of shared memory per slot: a single CTA keeps a deep enough
   // operand ring only with narrower tiles
   if constexpr (Epi::kSlots == 2) {
-    return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+    return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
   } else if constexpr (Epi::kSlots == 1) {
-    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
-    return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
+    return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
   } else {
-    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
-    if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
-    return launch_tc_bn<256, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st);
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
+    if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
+    return launch_tc_bn<256, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
   }
 }
 template <typename T, class Epi>
@@ -411,7 +417,7 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
       et::DgradEpiS<1> epi;
       epi.has_in[0] = need_skip; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = false; epi.act_prev = P.act;
-      epi.colsum = want_colsum ? (float*)s->at(s->off_biaspart) : nullptr; epi.ld = L.K;
+      epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = skip; em.out[0] = gout; em.in[1] = gout; em.out[1] = gout;
       return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
     }
@@ -419,14 +425,14 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
       et::DgradEpiS<1> epi;
       epi.has_in[0] = true; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = true; epi.act_prev = P.act;
-      epi.colsum = want_colsum ? (float*)s->at(s->off_biaspart) : nullptr; epi.ld = L.K;
+      epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = zmap; em.out[0] = dzout; em.in[1] = zmap; em.out[1] = dzout;
       return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
     }
     et::DgradEpiS<2> epi;                                     // both G_l and dZ_{l-1}
     epi.has_in[0] = need_skip; epi.has_in[1] = true; epi.has_out[0] = need_G; epi.has_out[1] = true;
     epi.mul_act = false; epi.act_prev = P.act;
-    epi.colsum = want_colsum ? (float*)s->at(s->off_biaspart) : nullptr; epi.ld = L.K;
+    epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
     em.in[0] = skip; em.out[0] = gout; em.in[1] = zmap; em.out[1] = dzout;
     return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
   } else {
@@ -472,7 +478,7 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
       const int bnh = L.pair_wgrad ? L.bn_wgrad / 2 : L.bn_wgrad;
       const CUtensorMap& amap = mn_map(a_map(s, l), 2, &p.a_3d);
       const CUtensorMap& bmap = mn_map(dz_map(s, l), bnh / 64, &p.b_3d);
-      ET_TRY((launch_tc<true, true>(L.bn_wgrad, L.pair_wgrad, amap, bmap, em, p, epi, s->sms, st)));
+      ET_TRY((launch_tc<true, true>(L.bn_wgrad, L.pair_wgrad, amap, bmap, em, p, epi, s->sms, st, s->wgrad_one_unit)));
     } else {
       et::simt::Params p;
       p.rows = L.K; p.cols = L.N; p.kc = (int)s->M; p.segs = 1;
@@ -500,7 +506,7 @@ et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
                           int* launches, cudaStream_t st, int fused_chunks = 0) {
   TimedLaunch tl(s, ET_K_BGRAD, st);
   const LayerRT& L = s->ly[l];
-  float* part = (float*)s->at(s->off_biaspart);
+  float* part = (float*)s->at(L.off_biaspart);
   int chunks = fused_chunks;
   if (fused_chunks == 0) {
     chunks = ceil_div(s->M, et::kColsumRows);
@@ -597,6 +603,12 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
       }
     }
     const bool two = !s->timing && setup_two_streams(s);   // per-kernel timing wants kernels one at a time
+    // Sharing the GPU with the higher-priority error-gradient chain: when few kernels are selected
+    // the weight gradients are filler work and should hand their SMs back after every unit; when
+    // they are as much work as the chain itself, persistent CTAs (epilogue overlap) pay more.
+    int n_w = 0;
+    for (int l = d; l < L; ++l) n_w += mask[2 * l] ? 1 : 0;
+    s->wgrad_one_unit = two && 2 * n_w <= L - d;
     cudaStream_t cs = two ? s->chain_stream : st;          // stream of the error-gradient chain
     if (two) {
       CU_TRY(cudaEventRecord(s->fork_ev, st));
@@ -616,11 +628,15 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
       const LayerRT& Y = s->ly[l];
       const double gemm = 2.0 * (double)s->M * Y.K * Y.N;
       if (mask[2 * l + 1]) {
-        // On the tensor-core path the column partials of dZ_l were left by dgrad(l+1) one
-        // iteration ago; they must be consumed before dgrad(l) reuses the buffer for dZ_{l-1}.
+        // On the tensor-core path the column partials of dZ_l were left by dgrad(l+1) in this
+        // layer's own buffer; finishing them need not sit on the chain's critical path.
         const int fused = (is_bf16<T>::value && l < L - 1) ? dgrad_row_blocks(s, l + 1) : 0;
+        // Which stream: with few selected kernels the caller's stream is nearly idle and takes
+        // the finishers off the chain; with many it is the busier one and the chain keeps them.
+        cudaStream_t bs = s->wgrad_one_unit ? st : cs;
+        if (two && bs == st) CU_TRY(cudaStreamWaitEvent(st, s->chain_ev[l + 1], 0));
         ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
-                                  delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, cs, fused));
+                                  delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, bs, fused));
       }
       if (l > d) {
         ET_TRY(run_dgrad_layer<T>(s, l, dY, cs, mask[2 * (l - 1) + 1] != 0));
@@ -744,7 +760,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
   s->off_status = take(256);
-  size_t max_partial = 0, max_biaspart = 0;
+  size_t max_partial = 0;
   const int chunks = ceil_div(M, et::kColsumRows);
   s->imp_offs.resize(2 * L); s->imp_counts.resize(2 * L);
   int imp_total = 0;
@@ -773,8 +789,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
       }
     }
     max_partial = std::max(max_partial, (size_t)y.split * y.K * y.N * sizeof(float));
-    max_biaspart = std::max(max_biaspart, (size_t)chunks * y.Nw * sizeof(float));
-    max_biaspart = std::max(max_biaspart, (size_t)(ceil_div(M, 256) * 8 + 8) * std::max(y.Nw, y.K) * sizeof(float));
+    y.off_biaspart = take((size_t)std::max(chunks, ceil_div(M, 256) * 8 + 8) * y.Nw * sizeof(float));
     y.imp_count_w = ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
     y.imp_count_b = ceil_div(y.N, et::kBiasCols);
     s->imp_offs[2 * l] = imp_total; s->imp_counts[2 * l] = y.imp_count_w; imp_total += y.imp_count_w;
@@ -782,7 +797,6 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
   }
   s->imp_total = imp_total;
   s->off_partial = take(max_partial);
-  s->off_biaspart = take(max_biaspart);
   s->off_imp_parts = take((size_t)imp_total * sizeof(float));
   s->off_imp_offs = take((size_t)2 * L * sizeof(int));
   s->off_imp_counts = take((size_t)2 * L * sizeof(int));
