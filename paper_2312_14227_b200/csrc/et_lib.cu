@@ -266,8 +266,14 @@ et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::t
                        const Epi& epi, int sms, cudaStream_t st, bool one_unit) {
   auto kern = et::tc::gemm_tc_kernel<BN, A_MN, B_MN, Epi, PAIR>;
   using C = et::tc::Cfg<BN, Epi::kSlots, PAIR>;
-  static bool attr_done = false;
-  static int max_clusters = 0;
+  // function attributes and occupancy are per device
+  static bool attr_done_dev[64] = {};
+  static int max_clusters_dev[64] = {};
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
+  bool& attr_done = attr_done_dev[dev];
+  int& max_clusters = max_clusters_dev[dev];
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   cfg.blockDim = dim3(et::tc::THREADS);

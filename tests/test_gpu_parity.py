@@ -147,6 +147,14 @@ def test_bf16_ragged_widths_and_bias_only_selection():
     h.check_step(w, w.mask, TOL_BF16)
 
 
+def test_bf16_fewer_rows_than_one_tile():
+    # 40 rows: every TMA box is taller than the tensors, half of each CTA pair works on padding
+    h = _h()
+    layers = [wl.Layer(64, 128, act=wl.ACT_GELU_TANH), wl.Layer(128, 64, residual_src=0), wl.Layer(64, 256, fold=1)]
+    w = wl.small_stack(layers, 40, wl.DT_BF16, 8, mask=np.ones(6, dtype=np.uint8), w_std=0.1, bias_std=0.05)
+    h.check_step(w, w.mask, TOL_BF16)
+
+
 def test_bf16_resnet_1x1_config():
     h = _h()
     w = wl.resnet_1x1()
