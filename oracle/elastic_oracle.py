@@ -358,3 +358,47 @@ def train_schedule(layers, W, b, x, target, lr: float, steps: int, period: int, 
         if new_mask is not None:
             mask = new_mask
     return dict(losses=np.array(losses), masks=masks, importances=evaluations, W=W, b=b)
+
+
+# --------------------------------------------------------------------------- the paper's optimisers, masked
+# Section 8: SGDW (momentum 0.9, decoupled weight decay 5e-4, cosine-scheduled learning rate) for the
+# convolutional models and Adam (learning rate 1e-4) for ViT.  Only selected tensors (and their
+# optimiser state) are touched.  The schedule lives with the caller: `lr` and `wd` are the values
+# of the current step.
+OPT_SGD, OPT_SGDW, OPT_ADAM = 0, 1, 2
+
+
+def optimizer_state(params):
+    """Zero-initialised state: first and second moment per tensor."""
+    return [np.zeros_like(p, dtype=np.float64) for p in params], [np.zeros_like(p, dtype=np.float64) for p in params]
+
+
+def optimizer_step_masked(params, grads, mask, kind, lr, state, step=1, momentum=0.9, wd=0.0,
+                          beta1=0.9, beta2=0.999, eps=1e-8):
+    """One masked update.  state = (m, v) lists as from optimizer_state, updated in place for
+    selected tensors; returns the new parameter list (unselected entries are the same objects).
+    SGDW (decoupled weight decay, Loshchilov & Hutter): m <- momentum*m + lr*g ;
+        w <- w - m - wd*w  (decay applied to the old weight, not through the gradient).
+    Adam (Kingma & Ba): m <- b1 m + (1-b1) g ; v <- b2 v + (1-b2) g^2 ;
+        w <- w - lr * (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps),  t = step (1-based)."""
+    m, v = state
+    out = []
+    for k, p in enumerate(params):
+        if not mask[k]:
+            out.append(p)
+            continue
+        g = grads[k]
+        if kind == OPT_SGD:
+            out.append(p - lr * g)
+        elif kind == OPT_SGDW:
+            m[k] = momentum * m[k] + lr * g
+            out.append(p - m[k] - wd * p)
+        elif kind == OPT_ADAM:
+            m[k] = beta1 * m[k] + (1.0 - beta1) * g
+            v[k] = beta2 * v[k] + (1.0 - beta2) * g * g
+            mhat = m[k] / (1.0 - beta1 ** step)
+            vhat = v[k] / (1.0 - beta2 ** step)
+            out.append(p - lr * mhat / (np.sqrt(vhat) + eps))
+        else:
+            raise ValueError(kind)
+    return out
