@@ -237,6 +237,16 @@ def run_own(args):
     et.et_forward_stack(stack, x, y, stream=stream)
     et.et_loss_mse_grad(stack, y, target, dY, None, stream=stream)
     torch.cuda.synchronize()
+    if args.optimizer != "sgd":                     # the paper's optimisers, with fp32 master weights
+        W32, b32 = [t.float() for t in W], [t.float() for t in b]
+        et.et_stack_bind_master(stack, W32, b32)
+        params = [t for pair in zip(W, b) for t in pair]
+        st1 = [torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in params]
+        st2 = [torch.zeros(p.shape, dtype=torch.float32, device=dev) for p in params]
+        if args.optimizer == "sgdw":
+            et.et_stack_set_optimizer(stack, et.ET_OPT_SGDW, st1, None, momentum=0.9, weight_decay=5e-4)
+        else:
+            et.et_stack_set_optimizer(stack, et.ET_OPT_ADAM, st1, st2)
     dY_host = dY.cpu().pin_memory()
     imp_host = torch.zeros(2 * w.L, dtype=torch.float32).pin_memory()
     ones = np.ones(2 * w.L, dtype=np.uint8)
@@ -352,7 +362,7 @@ def run_own(args):
         "config": {"workload": w.name, "blocks": 12, "tokens": w.M, "d": 768, "ffn": 3072,
                    "mask": "Bernoulli(0.3) per kernel tensor, seed 1, bias follows kernel",
                    "selected_tensors": int(w.mask.sum()), "deepest_selected_layer": first,
-                   "step": "et_backward_elastic with fused importance and SGD",
+                   "step": "et_backward_elastic with fused importance and " + {"sgd": "SGD", "sgdw": "SGDW (fp32 master weights)", "adam": "Adam (fp32 master weights)"}[args.optimizer],
                    "l2": "inputs larger than L2 (a step streams > 1 GB of activations and gradients)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "executed_flops_per_step": flops,
@@ -495,6 +505,8 @@ def main():
     ap.add_argument("--blocks", type=int, default=12, help="transformer blocks of the stack (12 = the benchmark workload)")
     ap.add_argument("--profile", action="store_true",
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
+    ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
+                    help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
     ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "schedule"],
                     help="vit_b = the benchmark line; resnet / schedule = side reports for the other shapes")
     args = ap.parse_args()

@@ -71,7 +71,8 @@ typedef enum {
 } et_cost_variant;
 
 enum {
-  ET_FLAG_FUSE_SGD = 1u,   /* et_backward_elastic also applies w <- w - lr*g to selected tensors */
+  ET_FLAG_FUSE_SGD = 1u,   /* et_backward_elastic also updates the selected tensors (w <- w - lr*g, or the
+                              optimiser set with et_stack_set_optimizer) */
   ET_FLAG_DELTA_IS_SNAPSHOT = 2u  /* delta[k] is a copy of tensor k taken earlier; the update of Eq. 2 is
                                      dw = (current tensor) - delta[k], formed on the fly (Section 3.1: the
                                      weight update accumulated since the start of the evaluation period) */
@@ -124,6 +125,34 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
  * masters in `delta`.  Unselected tensors and their masters are never written.  Call after
  * et_stack_bind (which detaches). */
 et_status et_stack_bind_master(et_stack* s, float* const* W32, float* const* b32);
+
+/* The optimisers the paper trains with (Section 8): SGDW -- momentum 0.9, decoupled weight decay
+ * 5e-4, cosine-scheduled learning rate -- for the convolutional models, Adam for ViT.  Masked like
+ * everything else: only selected tensors and their state are read or written.
+ *   ET_OPT_SGD :  w <- w - lr g
+ *   ET_OPT_SGDW:  m <- momentum m + lr g ;  w <- w - m - wd w
+ *   ET_OPT_ADAM:  m <- b1 m + (1-b1) g ;  v <- b2 v + (1-b2) g^2 ;
+ *                 w <- w - lr (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps)
+ * Schedules stay with the caller: `lr` is the argument of the updating call, the step number t
+ * and this step's weight decay wd are set with et_stack_set_optimizer_step. */
+typedef enum { ET_OPT_SGD = 0, ET_OPT_SGDW = 1, ET_OPT_ADAM = 2 } et_optimizer;
+typedef struct {
+  int32_t kind;         /* et_optimizer */
+  float momentum;       /* SGDW */
+  float weight_decay;   /* SGDW: initial wd (et_stack_set_optimizer_step overrides it per step) */
+  float beta1, beta2;   /* Adam */
+  float eps;            /* Adam */
+} et_optimizer_config;
+
+/* Selects the optimiser used by ET_FLAG_FUSE_SGD and et_update_masked.  state1 / state2: host
+ * arrays of 2L device float* in tensor order, shaped like the tensors, caller-owned and
+ * zero-initialised (state1 = momentum / first moment, needed for SGDW and Adam; state2 = second
+ * moment, Adam only).  cfg == NULL or kind ET_OPT_SGD restores plain SGD.  Resets t to 1.
+ * Call after et_stack_bind (which restores plain SGD). */
+et_status et_stack_set_optimizer(et_stack* s, const et_optimizer_config* cfg, float* const* state1,
+                                 float* const* state2);
+/* Step number t >= 1 (Adam's bias correction) and weight decay of the next updating call. */
+et_status et_stack_set_optimizer_step(et_stack* s, int32_t step, float weight_decay);
 
 /* ---- forward and loss (precede the hot path; Eq. 3's T_forward) -------------------- */
 
@@ -183,9 +212,13 @@ et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
                         const void* const* delta, float* importance_dev, void* stream);
 
 /* Stand-alone masked SGD: w_k <- w_k - lr * grads[k] for selected k (fp32 arithmetic,
- * rounded once to the storage dtype).  Unselected tensors are never written. */
+ * rounded once to the storage dtype), whatever optimiser is configured.  Unselected tensors
+ * are never written. */
 et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads,
                         float lr, void* stream);
+/* Stand-alone masked update with the configured optimiser (et_stack_set_optimizer). */
+et_status et_update_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads,
+                           float lr, void* stream);
 
 /* Bias gradient without any allocation.  (The paper has no counterpart for this call; it
  * exists for how this library gets embedded.)

@@ -33,6 +33,14 @@ class et_layer_desc(C.Structure):
                 ("fold", C.c_int32), ("residual_src", C.c_int32)]
 
 
+class et_optimizer_config(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("momentum", C.c_float), ("weight_decay", C.c_float),
+                ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+
+
+ET_OPT_SGD, ET_OPT_SGDW, ET_OPT_ADAM = 0, 1, 2
+
+
 class et_exec_report(C.Structure):
     _fields_ = [("dgrad", C.c_void_p), ("wgrad", C.c_void_p), ("bgrad", C.c_void_p), ("updated", C.c_void_p),
                 ("deepest", C.c_int32), ("launches", C.c_int32), ("flops_executed", C.c_double)]
@@ -51,6 +59,9 @@ _SIGS = {
     "et_backward_elastic_host": [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _u32, _f32, _vp, _vp],
     "et_importance": [_vp, _vp, _i32, _vp, _vp, _vp, _vp],
     "et_sgd_masked": [_vp, _vp, _i32, _vp, _f32, _vp],
+    "et_update_masked": [_vp, _vp, _i32, _vp, _f32, _vp],
+    "et_stack_set_optimizer": [_vp, _vp, _vp, _vp],
+    "et_stack_set_optimizer_step": [_vp, _i32, _f32],
     "et_profile_costs": [_vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp],
     "et_time_selective": [_vp, _vp, _vp, _i32, _i32, _vp],
     "et_select_dp": [_vp, _vp, _vp, _i32, _f64, _f64, _i32, _i32, _vp, _vp, _vp],
@@ -270,6 +281,26 @@ def et_sgd_masked(s: Stack, mask, grads, lr: float, stream=None):
     m = _mask_arr(mask)
     _check(_lib.et_sgd_masked(s.handle, _ptr(m), len(m), _ptr_array(grads, len(m)), lr, _stream_ptr(stream)),
            "et_sgd_masked")
+
+
+def et_update_masked(s: Stack, mask, grads, lr: float, stream=None):
+    m = _mask_arr(mask)
+    _check(_lib.et_update_masked(s.handle, _ptr(m), len(m), _ptr_array(grads, len(m)), lr, _stream_ptr(stream)),
+           "et_update_masked")
+
+
+def et_stack_set_optimizer(s: Stack, kind: int, state1=None, state2=None, momentum=0.9, weight_decay=0.0,
+                           beta1=0.9, beta2=0.999, eps=1e-8):
+    cfg = et_optimizer_config(kind, momentum, weight_decay, beta1, beta2, eps)
+    s._keep_opt = [state1, state2]
+    n = 2 * s.L
+    _check(_lib.et_stack_set_optimizer(s.handle, C.addressof(cfg),
+                                       _ptr_array(state1, n) if state1 is not None else None,
+                                       _ptr_array(state2, n) if state2 is not None else None), "et_stack_set_optimizer")
+
+
+def et_stack_set_optimizer_step(s: Stack, step: int, weight_decay: float = 0.0):
+    _check(_lib.et_stack_set_optimizer_step(s.handle, int(step), float(weight_decay)), "et_stack_set_optimizer_step")
 
 
 def et_profile_costs(s: Stack, x, y, dY, iters: int = 20, stream=None):

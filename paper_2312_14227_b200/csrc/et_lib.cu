@@ -4,6 +4,7 @@
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <new>
 #include <type_traits>
@@ -128,6 +129,8 @@ struct LayerRT {
   void* b = nullptr;
   float* W32 = nullptr;     // optional fp32 master copies (et_stack_bind_master)
   float* b32 = nullptr;
+  float* st1[2] = {nullptr, nullptr};   // optimiser state of kernel / bias: first moment (momentum)
+  float* st2[2] = {nullptr, nullptr};   // second moment (Adam)
   size_t off_a_out = 0;     // a_{l+1}           (unused for the last layer: that is the caller's y)
   size_t off_Z = 0;         // Z_l               (act != none)
   size_t off_G_out = 0;     // G_{l+1}           (unused for the last layer: that is the caller's dY)
@@ -163,6 +166,9 @@ struct et_stack {
   TMaps map_x, map_y, map_dy;
   const void* map_dy_ptr = nullptr;
   const void* map_y_ptr = nullptr;
+  et_optimizer_config opt_cfg = {ET_OPT_SGD, 0.f, 0.f, 0.f, 0.f, 0.f};
+  int opt_step = 1;                    // Adam's t (1-based)
+  float opt_wd_now = 0.f;              // this step's (scheduled) decoupled weight decay
   bool delta_is_snapshot = false;      // per call: the delta tensors hold a weight snapshot
   bool wgrad_one_unit = false;         // per call: weight-gradient CTAs take one unit each and leave
   // second stream: the error-gradient chain runs here while weight gradients run on the caller's
@@ -463,6 +469,20 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
   }
 }
 
+// Optimiser parameters of this step.  plain = true forces plain SGD (et_sgd_masked).
+et::OptParams opt_params(const et_stack* s, float lr, bool plain = false) {
+  et::OptParams o{};
+  o.kind = plain ? et::kOptSgd : s->opt_cfg.kind;
+  o.lr = lr;
+  if (o.kind == et::kOptSgdw) { o.a = s->opt_cfg.momentum; o.b = s->opt_wd_now; }
+  if (o.kind == et::kOptAdam) {
+    o.a = s->opt_cfg.beta1; o.b = s->opt_cfg.beta2; o.eps = s->opt_cfg.eps;
+    o.c1 = (float)(1.0 / (1.0 - std::pow((double)o.a, (double)s->opt_step)));
+    o.c2 = (float)(1.0 / (1.0 - std::pow((double)o.b, (double)s->opt_step)));
+  }
+  return o;
+}
+
 // dW_l = a_l^T dZ_l as split partials, then the reducer with grad / importance / SGD.
 template <typename T>
 et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
@@ -499,8 +519,9 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   TimedLaunch tl(s, ET_K_WGRAD_REDUCE, st);
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
   et::wgrad_reduce_kernel<T><<<L.imp_count_w, et::kEltThreads, 0, st>>>(partial, split, count, count, grad, delta, imp,
-                                                                        (T*)L.W, lr, sgd ? 1 : 0,
-                                                                        s->delta_is_snapshot ? 1 : 0, L.W32);
+                                                                        (T*)L.W, opt_params(s, lr), sgd ? 1 : 0,
+                                                                        s->delta_is_snapshot ? 1 : 0, L.W32, L.st1[0],
+                                                                        L.st2[0]);
   ++*launches;
   return after_launch();
 }
@@ -523,7 +544,8 @@ et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   }
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l + 1];
   et::bias_finish_kernel<T><<<L.imp_count_b, dim3(32, 8), 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
-                                                                       (T*)L.b, lr, sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0, L.b32);
+                                                                       (T*)L.b, opt_params(s, lr), sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0, L.b32,
+                                                                       L.st1[1], L.st2[1]);
   ++*launches;
   return after_launch();
 }
@@ -838,7 +860,9 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   cudaStream_t st = (cudaStream_t)stream;
   s->bound = false;
   s->ws = (char*)workspace;
-  for (int l = 0; l < s->L; ++l) { s->ly[l].W = W[l]; s->ly[l].b = b[l]; s->ly[l].W32 = nullptr; s->ly[l].b32 = nullptr; }
+  for (int l = 0; l < s->L; ++l) { s->ly[l].W = W[l]; s->ly[l].b = b[l]; s->ly[l].W32 = nullptr; s->ly[l].b32 = nullptr;
+    for (int k = 0; k < 2; ++k) { s->ly[l].st1[k] = nullptr; s->ly[l].st2[k] = nullptr; } }
+  s->opt_cfg = {ET_OPT_SGD, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (s->dtype == ET_BF16) {
     for (int l = 0; l < s->L; ++l) {
       LayerRT& y = s->ly[l];
@@ -971,13 +995,15 @@ et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
   return after_launch();
 }
 
-et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads, float lr,
-                        void* stream) {
+namespace {
+et_status update_masked_impl(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads, float lr,
+                             void* stream, bool plain) {
   ET_TRY(check_ready(s, mask, n_tensors));
   if (grads == nullptr) return ET_ERR_INVALID_ARG;
   for (int t = 0; t < n_tensors; ++t)
     if (mask[t] && grads[t] == nullptr) return ET_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
+  const et::OptParams o = opt_params(s, lr, plain);
   for (int t = 0; t < n_tensors; ++t) {
     if (!mask[t]) continue;
     const LayerRT& y = s->ly[t / 2];
@@ -985,11 +1011,57 @@ et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
     const size_t count = is_w ? (size_t)y.K * y.N : (size_t)y.N;
     void* w = is_w ? y.W : y.b;
     float* m = is_w ? y.W32 : y.b32;
+    float* s1 = y.st1[t & 1];
+    float* s2 = y.st2[t & 1];
     const int blocks = ceil_div(count, et::kEltThreads * et::kVec);
-    if (s->dtype == ET_BF16) et::sgd_kernel<bf16><<<blocks, et::kEltThreads, 0, st>>>((bf16*)w, grads[t], count, lr, m);
-    else                     et::sgd_kernel<float><<<blocks, et::kEltThreads, 0, st>>>((float*)w, grads[t], count, lr, m);
+    if (s->dtype == ET_BF16) et::sgd_kernel<bf16><<<blocks, et::kEltThreads, 0, st>>>((bf16*)w, grads[t], count, o, m, s1, s2);
+    else                     et::sgd_kernel<float><<<blocks, et::kEltThreads, 0, st>>>((float*)w, grads[t], count, o, m, s1, s2);
     ET_TRY(after_launch());
   }
+  return ET_OK;
+}
+}  // namespace
+
+et_status et_sgd_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads, float lr,
+                        void* stream) {
+  return update_masked_impl(s, mask, n_tensors, grads, lr, stream, true);
+}
+
+et_status et_update_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads, float lr,
+                           void* stream) {
+  return update_masked_impl(s, mask, n_tensors, grads, lr, stream, false);
+}
+
+et_status et_stack_set_optimizer(et_stack* s, const et_optimizer_config* cfg, float* const* state1,
+                                 float* const* state2) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  et_optimizer_config c = {ET_OPT_SGD, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (cfg != nullptr) c = *cfg;
+  if (c.kind != ET_OPT_SGD && c.kind != ET_OPT_SGDW && c.kind != ET_OPT_ADAM) return ET_ERR_INVALID_ARG;
+  if (c.kind != ET_OPT_SGD && state1 == nullptr) return ET_ERR_INVALID_ARG;
+  if (c.kind == ET_OPT_ADAM && state2 == nullptr) return ET_ERR_INVALID_ARG;
+  if (c.kind == ET_OPT_ADAM && !(c.beta1 >= 0.f && c.beta1 < 1.f && c.beta2 >= 0.f && c.beta2 < 1.f && c.eps > 0.f))
+    return ET_ERR_INVALID_ARG;
+  const int n = 2 * s->L;
+  for (int t = 0; t < n; ++t) {
+    if (c.kind != ET_OPT_SGD && (state1[t] == nullptr || ((uintptr_t)state1[t] & 15))) return ET_ERR_INVALID_ARG;
+    if (c.kind == ET_OPT_ADAM && (state2[t] == nullptr || ((uintptr_t)state2[t] & 15))) return ET_ERR_INVALID_ARG;
+  }
+  for (int t = 0; t < n; ++t) {
+    s->ly[t / 2].st1[t & 1] = c.kind != ET_OPT_SGD ? state1[t] : nullptr;
+    s->ly[t / 2].st2[t & 1] = c.kind == ET_OPT_ADAM ? state2[t] : nullptr;
+  }
+  s->opt_cfg = c;
+  s->opt_step = 1;
+  s->opt_wd_now = c.weight_decay;
+  return ET_OK;
+}
+
+et_status et_stack_set_optimizer_step(et_stack* s, int32_t step, float weight_decay) {
+  if (s == nullptr || step < 1 || !(weight_decay >= 0.f)) return ET_ERR_INVALID_ARG;
+  s->opt_step = step;
+  s->opt_wd_now = weight_decay;
   return ET_OK;
 }
 

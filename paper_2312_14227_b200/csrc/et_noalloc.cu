@@ -45,7 +45,7 @@ et_status run(const void* dZ, int64_t M, int32_t width, float* db, float* scratc
   et::colsum_partial_kernel<T><<<grid, block, 0, st>>>((const T*)dZ, (int)M, width, scratch);
   if (cudaGetLastError() != cudaSuccess) return ET_ERR_CUDA;
   et::bias_finish_kernel<T><<<(width + et::kBiasCols - 1) / et::kBiasCols, dim3(32, 8), 0, st>>>(
-      scratch, chunks, width, width, db, (const T*)nullptr, nullptr, (T*)nullptr, 0.f, 0, 0, nullptr);
+      scratch, chunks, width, width, db, (const T*)nullptr, nullptr, (T*)nullptr, et::OptParams{}, 0, 0, nullptr, nullptr, nullptr);
   if (cudaGetLastError() != cudaSuccess) return ET_ERR_CUDA;
   return ET_OK;
 }

@@ -12,19 +12,62 @@ constexpr int kEltThreads = 256;
 constexpr int kVec = 8;                         // elements per thread per step
 constexpr int kColsumRows = 128;                // rows per column-sum chunk
 
+// Optimiser of the masked update (Section 8 of the paper: SGDW for the convolutional models,
+// Adam for ViT; plain SGD otherwise).  Schedules live with the caller: lr and wd are this
+// step's values.
+//   SGD : w <- w - lr g
+//   SGDW: m <- momentum m + lr g ;  w <- w - m - wd w            (decoupled weight decay)
+//   Adam: m <- b1 m + (1-b1) g ;  v <- b2 v + (1-b2) g^2 ;  w <- w - lr (m c1) / (sqrt(v c2) + eps),
+//         c1 = 1 / (1 - b1^t), c2 = 1 / (1 - b2^t)
+constexpr int kOptSgd = 0, kOptSgdw = 1, kOptAdam = 2;
+struct OptParams {
+  int kind;
+  float lr;
+  float a;       // SGDW: momentum      Adam: beta1
+  float b;       // SGDW: weight decay  Adam: beta2
+  float eps;     // Adam
+  float c1, c2;  // Adam bias corrections
+};
+__device__ __forceinline__ float opt_update(float w, float g, const OptParams& o, float& m, float& v) {
+  if (o.kind == kOptSgdw) {
+    m = fmaf(o.a, m, o.lr * g);
+    return w - m - o.b * w;
+  }
+  if (o.kind == kOptAdam) {
+    m = fmaf(o.a, m, (1.0f - o.a) * g);
+    v = fmaf(o.b, v, (1.0f - o.b) * g * g);
+    return w - o.lr * (m * o.c1) / (sqrtf(v * o.c2) + o.eps);
+  }
+  return fmaf(-o.lr, g, w);
+}
+// Update of kVec consecutive weights with their state (state pointers may be null for SGD).
+__device__ __forceinline__ void opt_update_seg(float (&w)[8], const float (&g)[8], const OptParams& o,
+                                               float* m_state, float* v_state, size_t i0, int n) {
+  float m[8], v[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { m[i] = 0.0f; v[i] = 0.0f; }
+  if (o.kind != kOptSgd) load_seg<8>(m_state + i0, n, m);
+  if (o.kind == kOptAdam) load_seg<8>(v_state + i0, n, v);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w[i] = opt_update(w[i], g[i], o, m[i], v[i]);
+  if (o.kind != kOptSgd) store_seg<8>(m_state + i0, n, m);
+  if (o.kind == kOptAdam) store_seg<8>(v_state + i0, n, v);
+}
+
 // ---- weight gradient: sum the K-split partials, then everything that consumes g ----------
 //   g = sum_s partial[s]                       (fixed order s = 0, 1, ...)
 //   grad        <- g                           if grad != nullptr
 //   imp_part[b] <- sum over this block of g * dw        if delta != nullptr   (Eq. 2);
 //                  dw = delta, or W - delta when delta holds a snapshot of W
-//   W           <- W - lr * g                  if do_sgd   (fp32 arithmetic, one rounding)
+//   W           <- optimiser update of W with g if do_sgd   (fp32 arithmetic, one rounding)
 //   master != nullptr: the weight lives in fp32 there (W is its rounded copy): the update and
 //                  the snapshot difference use it, and a snapshot `delta` is fp32 as well
 template <typename T>
 __global__ void __launch_bounds__(kEltThreads)
 wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_t count,
                     float* grad /* may alias partial: each thread reads its elements before writing them */, const T* __restrict__ delta, float* __restrict__ imp_part,
-                    T* __restrict__ W, float lr, int do_sgd, int delta_is_snapshot, float* __restrict__ master) {
+                    T* __restrict__ W, OptParams opt, int do_sgd, int delta_is_snapshot, float* __restrict__ master,
+                    float* __restrict__ m_state, float* __restrict__ v_state) {
   const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
   float dot = 0.0f;
   if (i0 < count) {
@@ -54,8 +97,7 @@ wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_
       for (int i = 0; i < kVec; ++i) dot = fmaf(g[i], t[i], dot);
     }
     if (do_sgd) {
-#pragma unroll
-      for (int i = 0; i < kVec; ++i) w[i] = fmaf(-lr, g[i], w[i]);
+      opt_update_seg(w, g, opt, m_state, v_state, i0, n);
       if (master != nullptr) store_seg<kVec>(master + i0, n, w);
       store_seg<kVec>(W + i0, n, w);
     }
@@ -121,7 +163,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
                    float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
-                   T* __restrict__ b, float lr, int do_sgd, int delta_is_snapshot, float* __restrict__ master) {
+                   T* __restrict__ b, OptParams opt, int do_sgd, int delta_is_snapshot, float* __restrict__ master,
+                   float* __restrict__ m_state, float* __restrict__ v_state) {
   __shared__ float sm[8][kBiasCols + 1];
   const int j = blockIdx.x * kBiasCols + threadIdx.x;
   float g = 0.0f;
@@ -149,7 +192,11 @@ bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int co
         dot = g * dw;
       }
       if (do_sgd) {
-        w = fmaf(-lr, g, w);
+        float m = opt.kind != kOptSgd ? m_state[j] : 0.0f;
+        float v = opt.kind == kOptAdam ? v_state[j] : 0.0f;
+        w = opt_update(w, g, opt, m, v);
+        if (opt.kind != kOptSgd) m_state[j] = m;
+        if (opt.kind == kOptAdam) v_state[j] = v;
         if (master != nullptr) master[j] = w;
         b[j] = from_f32<T>(w);
       }
@@ -198,7 +245,8 @@ importance_kernel(const float* __restrict__ grad, const T* __restrict__ delta, s
 // ---- stand-alone masked SGD on one selected tensor -----------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(kEltThreads)
-sgd_kernel(T* __restrict__ w, const float* __restrict__ grad, size_t count, float lr, float* __restrict__ master) {
+sgd_kernel(T* __restrict__ w, const float* __restrict__ grad, size_t count, OptParams opt, float* __restrict__ master,
+           float* __restrict__ m_state, float* __restrict__ v_state) {
   const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
   if (i0 >= count) return;
   const int n = (int)min((size_t)kVec, count - i0);
@@ -206,8 +254,7 @@ sgd_kernel(T* __restrict__ w, const float* __restrict__ grad, size_t count, floa
   load_seg<kVec>(grad + i0, n, g);
   if (master != nullptr) load_seg<kVec>(master + i0, n, t);
   else load_seg<kVec>(w + i0, n, t);
-#pragma unroll
-  for (int i = 0; i < kVec; ++i) t[i] = fmaf(-lr, g[i], t[i]);
+  opt_update_seg(t, g, opt, m_state, v_state, i0, n);
   if (master != nullptr) store_seg<kVec>(master + i0, n, t);
   store_seg<kVec>(w + i0, n, t);
 }
