@@ -543,7 +543,7 @@ et_status run_bgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
     ++*launches;
   }
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l + 1];
-  et::bias_finish_kernel<T><<<L.imp_count_b, dim3(32, 8), 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
+  et::bias_finish_kernel<T><<<L.imp_count_b, dim3(et::kBiasCols, et::kBiasLanes), 0, st>>>(part, chunks, L.Nw, L.N, grad, delta, imp,
                                                                        (T*)L.b, opt_params(s, lr), sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0, L.b32,
                                                                        L.st1[1], L.st2[1]);
   ++*launches;

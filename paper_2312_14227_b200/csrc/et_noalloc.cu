@@ -44,7 +44,7 @@ et_status run(const void* dZ, int64_t M, int32_t width, float* db, float* scratc
   // call is ever consumed and nothing has to be cleared first
   et::colsum_partial_kernel<T><<<grid, block, 0, st>>>((const T*)dZ, (int)M, width, scratch);
   if (cudaGetLastError() != cudaSuccess) return ET_ERR_CUDA;
-  et::bias_finish_kernel<T><<<(width + et::kBiasCols - 1) / et::kBiasCols, dim3(32, 8), 0, st>>>(
+  et::bias_finish_kernel<T><<<(width + et::kBiasCols - 1) / et::kBiasCols, dim3(et::kBiasCols, et::kBiasLanes), 0, st>>>(
       scratch, chunks, width, width, db, (const T*)nullptr, nullptr, (T*)nullptr, et::OptParams{}, 0, 0, nullptr, nullptr, nullptr);
   if (cudaGetLastError() != cudaSuccess) return ET_ERR_CUDA;
   return ET_OK;

@@ -155,22 +155,24 @@ colsum_partial_kernel(const T* __restrict__ dZ, int M, int width, float* __restr
 }
 
 // ---- bias gradient, stage 2: sum the chunks, then grad / importance / SGD -----------------
-// Block (32, 8) handles kBiasCols bias elements j in [0, fold*width): x -> element, y -> which
-// chunks (y, y+8, ...) this thread adds; a fixed-order shared-memory sum joins the eight.
+// Block (32, 32) handles kBiasCols bias elements j in [0, fold*width): x -> element, y -> which
+// chunks (y, y+32, ...) this thread adds (a few independent loads each: the kernel is latency-
+// bound); a fixed-order shared-memory sum joins the 32.
 // column = j mod width (a folded layer's dZ is the same gradient repeated for each slice).
 constexpr int kBiasCols = 32;
+constexpr int kBiasLanes = 32;
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kBiasCols * kBiasLanes)
 bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
                    float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
                    T* __restrict__ b, OptParams opt, int do_sgd, int delta_is_snapshot, float* __restrict__ master,
                    float* __restrict__ m_state, float* __restrict__ v_state) {
-  __shared__ float sm[8][kBiasCols + 1];
+  __shared__ float sm[kBiasLanes][kBiasCols + 1];
   const int j = blockIdx.x * kBiasCols + threadIdx.x;
   float g = 0.0f;
   if (j < count) {
     const int col = j % width;
-    for (int c = threadIdx.y; c < chunks; c += 8) g += part[(size_t)c * width + col];
+    for (int c = threadIdx.y; c < chunks; c += kBiasLanes) g += part[(size_t)c * width + col];
   }
   sm[threadIdx.y][threadIdx.x] = g;
   __syncthreads();
@@ -179,7 +181,7 @@ bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int co
     if (j < count) {
       g = 0.0f;
 #pragma unroll
-      for (int y = 0; y < 8; ++y) g += sm[y][threadIdx.x];
+      for (int y = 0; y < kBiasLanes; ++y) g += sm[y][threadIdx.x];
       if (grad != nullptr) grad[j] = g;
       float w = 0.0f;
       if (do_sgd || (delta != nullptr && delta_is_snapshot)) w = master != nullptr ? master[j] : to_f32(b[j]);
