@@ -171,6 +171,8 @@ struct et_stack {
   float opt_wd_now = 0.f;              // this step's (scheduled) decoupled weight decay
   bool delta_is_snapshot = false;      // per call: the delta tensors hold a weight snapshot
   bool wgrad_one_unit = false;         // per call: weight-gradient CTAs take one unit each and leave
+  bool overlap_launch = true;          // forward / dgrad kernels start their prologue under the previous kernel's tail
+  bool chain_shares_gpu = false;       // per call: weight gradients run beside the error-gradient chain
   // second stream: the error-gradient chain runs here while weight gradients run on the caller's
   cudaStream_t chain_stream = nullptr;
   std::vector<cudaEvent_t> chain_ev;   // [l] = dgrad(l) finished; [L] = top-layer dZ ready; [L+1] = join
@@ -269,7 +271,7 @@ const TMaps& dz_map(const et_stack* s, int l) {                                 
 // ---- GEMM launches ---------------------------------------------------------------------------
 template <int BN, bool A_MN, bool B_MN, bool PAIR, class Epi>
 et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em, et::tc::Params p,
-                       const Epi& epi, int sms, cudaStream_t st, bool one_unit) {
+                       const Epi& epi, int sms, cudaStream_t st, bool one_unit, bool overlap_prev) {
   auto kern = et::tc::gemm_tc_kernel<BN, A_MN, B_MN, Epi, PAIR>;
   using C = et::tc::Cfg<BN, Epi::kSlots, PAIR>;
   // function attributes and occupancy are per device
@@ -281,20 +283,32 @@ et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::t
   bool& attr_done = attr_done_dev[dev];
   int& max_clusters = max_clusters_dev[dev];
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   cfg.blockDim = dim3(et::tc::THREADS);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = st;
+  cfg.attrs = attr;
   if (PAIR) {
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
+    attr[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
+    attr[cfg.numAttrs].val.clusterDim.x = 2; attr[cfg.numAttrs].val.clusterDim.y = 1;
+    attr[cfg.numAttrs].val.clusterDim.z = 1;
+    ++cfg.numAttrs;
+  }
+  const unsigned n_plain_attrs = cfg.numAttrs;
+  if (overlap_prev) {
+    // the kernel's prologue may start while the stream's previous kernel drains; the kernel itself
+    // waits (griddepcontrol.wait) before it touches global memory
+    attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+    ++cfg.numAttrs;
   }
   if (!attr_done) {
     CU_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES));
     if (PAIR) {
       cfg.gridDim = dim3(sms & ~1);
-      if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) != cudaSuccess || max_clusters < 1) {
+      cudaLaunchConfig_t occ = cfg;
+      occ.numAttrs = n_plain_attrs;
+      if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &occ) != cudaSuccess || max_clusters < 1) {
         (void)cudaGetLastError();
         max_clusters = sms / 2;
       }
@@ -313,25 +327,26 @@ et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::t
 }
 template <bool A_MN, bool B_MN, class Epi>
 et_status launch_tc(int bn, bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const et::tc::EpiMaps& em,
-                    const et::tc::Params& p, const Epi& epi, int sms, cudaStream_t st, bool one_unit = false) {
+                    const et::tc::Params& p, const Epi& epi, int sms, cudaStream_t st, bool one_unit = false,
+                    bool overlap_prev = false) {
   if (pair) {
-    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit);
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
     if constexpr (!B_MN) {
-      if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit);
+      if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
     }
-    return launch_tc_bn<256, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit);
+    return launch_tc_bn<256, A_MN, B_MN, true>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
   }
   // staged epilogues take 64 KB of shared memory per slot: a single CTA keeps a deep enough
   // operand ring only with narrower tiles
   if constexpr (Epi::kSlots == 2) {
-    return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
+    return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
   } else if constexpr (Epi::kSlots == 1) {
-    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
-    return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
+    return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
   } else {
-    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
-    if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
-    return launch_tc_bn<256, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit);
+    if (bn == 128) return launch_tc_bn<128, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
+    if (bn == 192) return launch_tc_bn<192, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
+    return launch_tc_bn<256, A_MN, B_MN, false>(ma, mb, em, p, epi, sms, st, one_unit, overlap_prev);
   }
 }
 template <typename T, class Epi>
@@ -378,10 +393,10 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
     };
     if (L.act != ET_ACT_NONE) {
       et::FwdEpiS<2> epi; fill(epi);
-      return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st);
+      return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch);
     }
     et::FwdEpiS<1> epi; fill(epi);
-    return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st);
+    return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch);
   } else {
     et::FwdEpi<T> epi;
     epi.bias = (const T*)L.b;
@@ -431,7 +446,7 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
       epi.mul_act = false; epi.act_prev = P.act;
       epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = skip; em.out[0] = gout; em.in[1] = gout; em.out[1] = gout;
-      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
+      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
     }
     if (!need_skip && !need_G) {                              // dZ_{l-1} = acc * act'(Z_{l-1})
       et::DgradEpiS<1> epi;
@@ -439,14 +454,14 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
       epi.mul_act = true; epi.act_prev = P.act;
       epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = zmap; em.out[0] = dzout; em.in[1] = zmap; em.out[1] = dzout;
-      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
+      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
     }
     et::DgradEpiS<2> epi;                                     // both G_l and dZ_{l-1}
     epi.has_in[0] = need_skip; epi.has_in[1] = true; epi.has_out[0] = need_G; epi.has_out[1] = true;
     epi.mul_act = false; epi.act_prev = P.act;
     epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
     em.in[0] = skip; em.out[0] = gout; em.in[1] = zmap; em.out[1] = dzout;
-    return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st);
+    return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
   } else {
     et::DgradEpi<T> epi;
     epi.skip = need_skip ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
@@ -637,6 +652,10 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
     int n_w = 0;
     for (int l = d; l < L; ++l) n_w += mask[2 * l] ? 1 : 0;
     s->wgrad_one_unit = two && 2 * n_w <= L - d;
+    // With a second stream the weight-gradient CTAs get their SMs in the gaps between the chain's
+    // kernels; a chain kernel that took over each SM the moment its predecessor left would starve
+    // them until the chain ends (measured: 2.45 -> 2.62 ms per ViT-B step), so no launch overlap then.
+    s->chain_shares_gpu = two;
     cudaStream_t cs = two ? s->chain_stream : st;          // stream of the error-gradient chain
     if (two) {
       CU_TRY(cudaEventRecord(s->fork_ev, st));
@@ -747,6 +766,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
   if (s == nullptr) return ET_ERR_INVALID_ARG;
   s->L = L; s->M = M; s->dtype = dtype; s->elt = dtype == ET_BF16 ? 2 : 4;
   s->ly.resize(L);
+  s->overlap_launch = getenv("ET_NO_LAUNCH_OVERLAP") == nullptr;
   {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&

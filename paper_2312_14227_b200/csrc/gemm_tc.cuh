@@ -388,6 +388,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if constexpr (PAIR) cluster_sync_all();          // the peer's barriers exist before anything targets them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Programmatic dependent launch: everything above touched only this CTA's own shared and tensor
+  // memory, so it may run while the previous kernel of the stream drains.  From here on global memory
+  // is read and written: wait until that kernel has completed and its writes are visible (returns at
+  // once in an ordinary launch), then let the next kernel's CTAs take each SM as this grid leaves it.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int tiles = p.tiles_m * p.tiles_n;
   const int units = tiles * p.split;
