@@ -13,6 +13,11 @@ layer l, tensor 2*l+1 its bias.  Layer l computes
     H_l     = act_l(Z_l)
     a_{l+1} = sum of `fold` equal column slices of H_l  (+ a_j if residual_src = j)
 
+or, for a normalisation layer (Section 5.2; its Gamma and Beta are tensors 2*l and 2*l+1),
+
+    xhat    = (a_l - mean) / sqrt(var + eps)         mean, var over the features of each row
+    a_{l+1} = xhat * gamma_l + beta_l
+
 Pins (tests/test_oracle_*.py): central finite differences of the loss for every
 tensor and every layer kind; the closed form of the importance sum when the update
 is a gradient step; the first-order Taylor identity of Eq. (6); masked == full
@@ -29,7 +34,12 @@ from typing import Dict, List, Optional, Sequence
 import numpy as np
 
 ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
+KIND_DENSE, KIND_NORM = 0, 1
 STRICT, INCLUSIVE = 0, 1
+
+
+def _kind(ly) -> int:
+    return getattr(ly, "kind", KIND_DENSE)
 
 _C0 = np.sqrt(2.0 / np.pi)
 _C1 = 0.044715
@@ -73,6 +83,15 @@ def forward(layers, W: Sequence[np.ndarray], b: Sequence[np.ndarray], x: np.ndar
     a = [np.asarray(x, dtype=np.float64)]
     Z = []
     for l, ly in enumerate(layers):
+        if _kind(ly) == KIND_NORM:
+            # layer normalisation: per row, biased variance; Z keeps (xhat, 1/sqrt(var + eps))
+            mean = a[l].mean(axis=1, keepdims=True)
+            var = ((a[l] - mean) ** 2).mean(axis=1, keepdims=True)
+            rstd = 1.0 / np.sqrt(var + ly.eps)
+            xhat = (a[l] - mean) * rstd
+            Z.append((xhat, rstd))
+            a.append(xhat * np.asarray(W[l], dtype=np.float64) + np.asarray(b[l], dtype=np.float64))
+            continue
         z = a[l] @ np.asarray(W[l], dtype=np.float64) + np.asarray(b[l], dtype=np.float64)
         h = act_forward(z, ly.act)
         w = ly.out_features // ly.fold
@@ -124,9 +143,12 @@ def exec_plan(L: int, mask: Sequence[int]) -> Plan:
 
 
 def executed_flops(layers, M: int, plan: Plan) -> float:
-    """2*M*K*N per executed GEMM (dgrad and wgrad of one layer cost the same)."""
+    """2*M*K*N per executed GEMM (dgrad and wgrad of one layer cost the same);
+    normalisation layers are not GEMMs and count nothing."""
     fl = 0.0
     for l, ly in enumerate(layers):
+        if _kind(ly) == KIND_NORM:
+            continue
         g = 2.0 * M * ly.in_features * ly.out_features
         fl += g * (int(plan.dgrad[l]) + int(plan.wgrad[l]))
     return fl
@@ -143,6 +165,21 @@ def _backward_sweep(layers, W, saved: Saved, dY: np.ndarray, stop: int,
     for l in range(L - 1, stop - 1, -1):
         ly = layers[l]
         g_out = G[l + 1]
+        if _kind(ly) == KIND_NORM:
+            xhat, rstd = saved.Z[l]
+            if want_w[l]:
+                grads[2 * l] = (g_out * xhat).sum(axis=0)           # d gamma
+            if want_b[l]:
+                grads[2 * l + 1] = g_out.sum(axis=0)                # d beta
+            if l > stop:
+                # y = xhat*gamma + beta with xhat = (x - mean(x)) * rstd(x): differentiating through
+                # the row mean and the row variance leaves the part of gy = g*gamma that is
+                # orthogonal to the all-ones vector and to xhat, scaled by rstd
+                gy = g_out * np.asarray(W[l], dtype=np.float64)
+                dX = rstd * (gy - gy.mean(axis=1, keepdims=True)
+                             - xhat * (gy * xhat).mean(axis=1, keepdims=True))
+                G[l] = dX if G[l] is None else G[l] + dX
+            continue
         if ly.residual_src >= 0:
             j = ly.residual_src
             G[j] = g_out.copy() if G[j] is None else G[j] + g_out

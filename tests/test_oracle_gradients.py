@@ -179,3 +179,88 @@ def test_mse_gradient_normalisation():
     t = np.zeros((2, 2))
     loss, g = orc.mse_loss_grad(y, t)
     assert loss == (1 + 4 + 9 + 25) / 4 and np.array_equal(g, y / 2)
+
+
+# ------------------------------------------------------------------ normalisation layers (Section 5.2)
+def _norm_stack():
+    # normalisation first, between dense layers, before an activation layer, under a residual, last
+    return [
+        wl.norm_layer(6),                                        # 0: acts on the stack input
+        wl.Layer(6, 8, act=wl.ACT_GELU_TANH),                    # 1
+        wl.Layer(8, 6, residual_src=0),                          # 2: residual from the stack input
+        wl.norm_layer(6, eps=1e-3),                              # 3: its input a_3 also feeds layer 5's residual
+        wl.Layer(6, 9, fold=3),                                  # 4
+        wl.Layer(3, 6, act=wl.ACT_RELU, residual_src=3),         # 5
+        wl.norm_layer(6),                                        # 6: last layer
+    ]
+
+
+def test_finite_differences_through_normalisation_layers():
+    _fd_check(_norm_stack(), M=5, seed=21, tol=5e-6)
+    _fd_check(wl.vit_blocks_prenorm(2, 6, 10), M=4, seed=22, tol=5e-6)
+
+
+def test_normalisation_forward_closed_forms():
+    # two features: xhat = +-(|a-b|/2) / sqrt((a-b)^2/4 + eps), whatever the row's mean
+    ly = [wl.norm_layer(2, eps=0.25)]
+    x = np.array([[3.0, 1.0], [-2.0, 6.0], [5.0, 5.0]])
+    gamma, beta = np.array([2.0, -1.0]), np.array([0.5, 0.25])
+    y = orc.forward(ly, [gamma], [beta], x).a[-1]
+    half = np.array([1.0, 4.0, 0.0])
+    xh = half / np.sqrt(half ** 2 + 0.25)
+    want = np.stack([np.array([s, -s]) * gamma + beta for s in (xh[0], -xh[1], 0.0)])
+    assert np.allclose(y, want, atol=1e-15)
+    # any width: rows of xhat have mean 0 and second moment var/(var+eps); shifting or scaling a row
+    # (eps = 0) does not change the output
+    rng = np.random.default_rng(3)
+    x = rng.normal(size=(9, 11)) * 3.0 + 2.0
+    ly = [wl.norm_layer(11, eps=0.0)]
+    one, zero = np.ones(11), np.zeros(11)
+    xh = orc.forward(ly, [one], [zero], x).a[-1]
+    assert np.allclose(xh.mean(axis=1), 0.0, atol=1e-14) and np.allclose((xh ** 2).mean(axis=1), 1.0, atol=1e-13)
+    assert np.allclose(orc.forward(ly, [one], [zero], 7.5 * x - 4.0).a[-1], xh, atol=1e-12)
+
+
+def test_normalisation_gradients_match_the_library_layer_norm():
+    # the same stack written with torch's own linear / layer_norm / gelu and differentiated by autograd
+    torch = pytest.importorskip("torch")
+    F = torch.nn.functional
+    layers = [wl.Layer(5, 8), wl.norm_layer(8, eps=1e-5), wl.Layer(8, 8, act=wl.ACT_GELU_TANH), wl.norm_layer(8, eps=1e-2)]
+    w = wl.small_stack(layers, 6, wl.DT_F32, 31, w_std=0.5, bias_std=0.2)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    grads = orc.backward_full(w.layers, w.W, saved, dY)
+    tW = [torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in w.W]
+    tb = [torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in w.b]
+    h = torch.tensor(w.x, dtype=torch.float64)
+    for l, ly in enumerate(layers):
+        if ly.kind == wl.KIND_NORM:
+            h = F.layer_norm(h, (ly.out_features,), tW[l], tb[l], ly.eps)
+        else:
+            h = h @ tW[l] + tb[l]
+            if ly.act == wl.ACT_GELU_TANH:
+                h = F.gelu(h, approximate="tanh")
+    loss = ((h - torch.tensor(w.target, dtype=torch.float64)) ** 2).mean()
+    loss.backward()
+    assert abs(loss.item() - orc.mse_loss(saved.a[-1], w.target)) < 1e-13
+    for l in range(len(layers)):
+        assert np.allclose(grads[2 * l], tW[l].grad.numpy(), rtol=1e-9, atol=1e-13), l
+        assert np.allclose(grads[2 * l + 1], tb[l].grad.numpy(), rtol=1e-9, atol=1e-13), l
+
+
+def test_masked_backward_with_normalisation_layers():
+    # selected tensors get the full-backprop gradients; nothing below the deepest selected layer runs;
+    # a normalisation layer that is itself the deepest passes no gradient on
+    layers = _norm_stack()
+    w = wl.small_stack(layers, 5, wl.DT_F32, 23, w_std=0.4, bias_std=0.3)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    full = orc.backward_full(w.layers, w.W, saved, dY)
+    mask = np.zeros(14, dtype=np.uint8)
+    mask[[6, 7, 10, 13]] = 1                     # gamma_3, beta_3, W_5, beta_6
+    grads, plan = orc.backward_masked(w.layers, w.W, saved, dY, mask)
+    assert plan.deepest == 3 and list(plan.dgrad) == [False] * 4 + [True] * 3
+    assert sorted(grads) == [6, 7, 10, 13]
+    for t in grads:
+        assert np.array_equal(grads[t], full[t])
+    assert orc.executed_flops(layers, 5, plan) == 2.0 * 5 * (6 * 9 + 2 * 3 * 6)

@@ -7,7 +7,8 @@ selection): both sides receive the same arrays from here and compute on their ow
 Layer / tensor indexing is forward execution order, 0 = nearest the input
 (the paper lists trainable tensors in execution order, Section 5).  Tensor
 ``2*l`` is the kernel of layer ``l`` and tensor ``2*l + 1`` its bias
-(Section 5.1: a dense layer carries a Kernel and a Bias tensor).
+(Section 5.1: a dense layer carries a Kernel and a Bias tensor); for a
+normalisation layer they are its Gamma and Beta (Section 5.2).
 
 The stacks stand in for the models the paper trains (ViT, ResNet50; Section 8)
 with every non-dense operator replaced by the identity, so that the whole
@@ -24,6 +25,9 @@ import numpy as np
 # activation / post-op codes (mirrored by include/et.h)
 ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
 DT_F32, DT_BF16 = 0, 1
+# layer kinds: a dense layer (kernel, bias) or a layer normalisation over the feature axis, whose two
+# trainable tensors gamma and beta take the kernel and bias slots (Section 5.2: Gamma and Beta)
+KIND_DENSE, KIND_NORM = 0, 1
 
 
 @dataclass(frozen=True)
@@ -34,6 +38,8 @@ class Layer:
     fold: int = 1              # output = sum of `fold` equal column slices of act(Z)
     residual_src: int = -1     # -1, or j: add activation a_j (a_0 = stack input,
                                # a_{j+1} = output of layer j) to this layer's output
+    kind: int = KIND_DENSE     # KIND_NORM: in_features == out_features, no act / fold / residual
+    eps: float = 1e-5          # KIND_NORM: added to the variance
 
     @property
     def out_width(self) -> int:
@@ -113,10 +119,34 @@ def vit_blocks(n_blocks: int, d: int, ffn: int) -> List[Layer]:
     return layers
 
 
+def norm_layer(d: int, eps: float = 1e-5) -> Layer:
+    return Layer(d, d, kind=KIND_NORM, eps=eps)
+
+
+def vit_blocks_prenorm(n_blocks: int, d: int, ffn: int) -> List[Layer]:
+    """Pre-norm transformer block, attention core still the identity:
+    LN, QKV d->3d (three slices summed), out-proj d->d + block input,
+    LN, fc1 d->ffn with tanh-GELU, fc2 ffn->d + the second LN's input."""
+    layers: List[Layer] = []
+    for blk in range(n_blocks):
+        base = 6 * blk
+        layers.append(norm_layer(d))
+        layers.append(Layer(d, 3 * d, fold=3))
+        layers.append(Layer(d, d, residual_src=base))
+        layers.append(norm_layer(d))
+        layers.append(Layer(d, ffn, act=ACT_GELU_TANH))
+        layers.append(Layer(ffn, d, residual_src=base + 3))
+    return layers
+
+
 # --------------------------------------------------------------------------- draws
 def _draw_params(rng, layers, dtype, w_std=None, he_init=False):
     W, b = [], []
     for ly in layers:
+        if ly.kind == KIND_NORM:
+            W.append(_store(1.0 + rng.normal(0.0, 0.1, size=ly.out_features), dtype))     # gamma
+            b.append(_store(rng.normal(0.0, 0.1, size=ly.out_features), dtype))           # beta
+            continue
         std = np.sqrt(2.0 / ly.in_features) if he_init else w_std
         W.append(_store(rng.normal(0.0, std, size=(ly.in_features, ly.out_features)), dtype))
         b.append(np.zeros(ly.out_features, dtype=np.float64))
@@ -155,6 +185,16 @@ def vit_b(seed: int = 1, p_select: float = 0.3, n_blocks: int = 12, tokens: int 
     layers = vit_blocks(n_blocks, d, ffn)
     mask = bernoulli_weight_mask(rng, len(layers), p_select)
     return _finish(name, layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
+
+
+def vit_b_prenorm(seed: int = 4, p_select: float = 0.3, n_blocks: int = 12, tokens: int = 64 * 197,
+                  d: int = 768, ffn: int = 3072, params: bool = True) -> Workload:
+    """The ViT-B/16-shaped stack with its two layer normalisations per block (gamma and beta are
+    selectable tensors); Bernoulli(p_select) over layers, both tensors of a layer follow the draw."""
+    rng = np.random.default_rng(seed)
+    layers = vit_blocks_prenorm(n_blocks, d, ffn)
+    mask = bernoulli_weight_mask(rng, len(layers), p_select)
+    return _finish("vit_b_prenorm_bf16", layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
 
 
 def vit_l(seed: int = 3, params: bool = True, n_blocks: int = 24, tokens: int = 32 * 197,
@@ -212,6 +252,7 @@ def draw_delta(w: Workload, seed: int, std: float = 1e-3):
     rng = np.random.default_rng(seed)
     out = []
     for ly in w.layers:
-        out.append(_store(rng.normal(0.0, std, size=(ly.in_features, ly.out_features)), w.dtype))
+        shape = (ly.out_features,) if ly.kind == KIND_NORM else (ly.in_features, ly.out_features)
+        out.append(_store(rng.normal(0.0, std, size=shape), w.dtype))
         out.append(_store(rng.normal(0.0, std, size=ly.out_features), w.dtype))
     return out
