@@ -22,6 +22,16 @@
  *       a_{l+1} = sum of the `fold` equal column slices of H_l  (+ a_j if residual_src = j)
  *   a_0 is the stack input; the width of a_{l+1} is out_features / fold.
  *
+ *   A layer of kind ET_LAYER_NORM is a layer normalisation over the features of each row
+ *   (Section 5.2 treats normalisation layers as two trainable tensors, Gamma and Beta;
+ *   Section 5.4 says LayerNorm behaves like batch normalisation in this respect):
+ *       xhat    = (a_l - mean) / sqrt(var + eps)        mean, biased var over the row
+ *       a_{l+1} = xhat * gamma_l + beta_l
+ *   Tensor 2l is gamma_l [features], tensor 2l+1 is beta_l [features]; they are passed
+ *   where a dense layer passes W_l and b_l.  Its backward pass has the same three parts:
+ *   the error gradient through the normalisation (only above the deepest selected layer),
+ *   d gamma = column sums of g * xhat and d beta = column sums of g for selected tensors.
+ *
  *   Storage type (et_dtype) applies to weights, biases, activations, error gradients
  *   and delta-W; accumulation is always fp32.  Exported gradients and importances are
  *   fp32.  ET_BF16 stacks run on tcgen05 tensor cores and need every feature count to
@@ -63,6 +73,7 @@ typedef enum {
 
 typedef enum { ET_F32 = 0, ET_BF16 = 1 } et_dtype;
 typedef enum { ET_ACT_NONE = 0, ET_ACT_GELU_TANH = 1, ET_ACT_RELU = 2 } et_act;
+typedef enum { ET_LAYER_DENSE = 0, ET_LAYER_NORM = 1 } et_layer_kind;
 
 /* Cost-model reading for the selector (Section 2.2 / Eq. 7 versus the example after Eq. 3). */
 typedef enum {
@@ -84,6 +95,9 @@ typedef struct {
   int32_t act;            /* et_act; must be ET_ACT_NONE when fold > 1 */
   int32_t fold;           /* >= 1, divides out_features */
   int32_t residual_src;   /* -1, or j in [0, l]: add a_j to this layer's output */
+  int32_t kind;           /* et_layer_kind.  ET_LAYER_NORM: in_features == out_features (a multiple of 8,
+                             at most 2048), act = ET_ACT_NONE, fold = 1, residual_src = -1 */
+  float eps;              /* ET_LAYER_NORM: added to the variance, > 0 or 0 */
 } et_layer_desc;
 
 /* What one et_backward_elastic call executed.  The four arrays are caller-owned host
@@ -255,7 +269,10 @@ et_status et_bias_grad_noalloc(const void* dZ, int64_t M, int32_t width, et_dtyp
  * and fills per-TENSOR cost vectors of length 2L following Section 5.1: kernel tensor:
  * t_dw = weight-gradient time, t_dy = error-gradient time (with the fused backward of the
  * non-trainable work below it, Section 5.3); bias tensor: t_dw = bias-gradient time,
- * t_dy = 0.  t_fwd receives the forward time.  Milliseconds.  Synchronous.  Runs a forward
+ * t_dy = 0.  A normalisation layer is one black box (Section 5.2): the time of its whole
+ * backward kernel (error gradient and d gamma together) plus its two finishing kernels goes
+ * to t_dy of beta; t_dw of gamma and beta and t_dy of gamma are 0.
+ * t_fwd receives the forward time.  Milliseconds.  Synchronous.  Runs a forward
  * pass from x (writing y) and a full backward from dY first; weights are not changed. */
 et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, int32_t iters,
                            double* t_dw, double* t_dy, double* t_fwd, void* stream);
@@ -288,7 +305,8 @@ typedef enum {
   ET_K_WGRAD_REDUCE = 3,   /* split reduction + gradient export + importance + SGD      */
   ET_K_BGRAD = 4,          /* bias gradient: column sums + finish (T2)                  */
   ET_K_OTHER = 5,          /* loss gradient, top-layer activation backward, importance finalise */
-  ET_K_CLASSES = 6
+  ET_K_NORM = 6,           /* normalisation layers: forward, backward (error gradient + d gamma), gamma finish */
+  ET_K_CLASSES = 7
 } et_kernel_class;
 
 /* on != 0: every kernel this stack launches from now on is bracketed by a pair of CUDA

@@ -17,6 +17,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
+#include "norm.cuh"
 
 namespace {
 
@@ -124,6 +125,11 @@ const CUtensorMap& mn_map(const TMaps& t, int chunks, int* use3d) {
 
 struct LayerRT {
   int K = 0, N = 0, Nw = 0, fold = 1, act = 0, residual_src = -1;
+  int kind = ET_LAYER_DENSE;     // ET_LAYER_NORM: K = N = Nw = features, W = gamma, b = beta
+  float eps = 0.f;
+  size_t off_stats = 0;     // norm: (mean, rstd) per row
+  size_t off_gpart = 0;     // norm: per-block partial column sums of g * xhat
+  int norm_blocks = 0;      // norm: blocks of the backward kernel = rows of off_gpart
   int consumer = -1;        // layer whose residual reads a_l (its output gradient joins G_l), or -1
   void* W = nullptr;
   void* b = nullptr;
@@ -141,6 +147,7 @@ struct LayerRT {
   int bn_fwd = 256, bn_dgrad = 256, bn_wgrad = 256;   // tile widths chosen per GEMM
   bool pair_fwd = false, pair_dgrad = false, pair_wgrad = false;   // CTA-pair (cta_group::2) tiles
   int imp_count_w = 0, imp_count_b = 0;
+  size_t w_count() const { return kind == ET_LAYER_NORM ? (size_t)N : (size_t)K * N; }   // elements of tensor 2l
   // bf16 stacks: one TMA descriptor per tensor (the caller's x, y and dY get theirs per call)
   TMaps map_W, map_aout, map_Gout, map_Z, map_dZ;
   CUtensorMap map_Wd;       // W as the K-major B of the dgrad GEMM: one box = the CTA's whole B tile
@@ -498,6 +505,78 @@ et::OptParams opt_params(const et_stack* s, float lr, bool plain = false) {
   return o;
 }
 
+// ---- normalisation layers ------------------------------------------------------------------
+// Register chunks per lane for a row of `d` features: 1..4, 6 or 8 (d <= 2048).
+template <typename F>
+et_status norm_dispatch(int d, F&& f) {
+  const int need = ceil_div(d, 256);
+  if (need <= 1) return f(std::integral_constant<int, 1>());
+  if (need == 2) return f(std::integral_constant<int, 2>());
+  if (need == 3) return f(std::integral_constant<int, 3>());
+  if (need == 4) return f(std::integral_constant<int, 4>());
+  if (need <= 6) return f(std::integral_constant<int, 6>());
+  if (need <= 8) return f(std::integral_constant<int, 8>());
+  return ET_ERR_UNSUPPORTED;
+}
+
+template <typename T>
+et_status run_norm_forward(et_stack* s, int l, void* y, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_NORM, st);
+  const LayerRT& L = s->ly[l];
+  T* out = l == s->L - 1 ? (T*)y : (T*)s->at(L.off_a_out);
+  const int blocks = std::min(ceil_div(s->M, et::kNormWarps), s->sms * 8);
+  return norm_dispatch(L.N, [&](auto vpl) -> et_status {
+    et::norm_forward_kernel<T, decltype(vpl)::value><<<blocks, et::kNormThreads, 0, st>>>(
+        act_in<T>(s, l), (const T*)L.W, (const T*)L.b, out, (float2*)s->at(L.off_stats), (int)s->M, L.N, L.eps);
+    return after_launch();
+  });
+}
+
+// Backward of normalisation layer l.  want_dx: G_l (with the skip gradient) and dZ_{l-1} for the layer
+// below (l >= 1); want_dgamma: the partial column sums of g * xhat, finished into the gradient of
+// gamma with importance and update like a bias.
+template <typename T>
+et_status run_norm_backward(et_stack* s, int l, const void* dY, bool want_dx, bool want_dgamma, float* grad,
+                            const T* delta, bool sgd, float lr, int* launches, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_NORM, st);
+  const LayerRT& L = s->ly[l];
+  if (!want_dx && !want_dgamma) return ET_OK;
+  const T* skip = nullptr;
+  T* G_in = nullptr;
+  const T* z_prev = nullptr;
+  T* dz_prev = nullptr;
+  int act_prev = ET_ACT_NONE;
+  if (want_dx) {
+    const LayerRT& P = s->ly[l - 1];
+    const bool need_act = P.act != ET_ACT_NONE;
+    const bool need_G = !need_act || P.residual_src >= 0;
+    if (L.consumer >= 0) skip = grad_act<T>(s, L.consumer + 1, dY);
+    if (need_G) G_in = (T*)s->at(P.off_G_out);
+    if (need_act) { z_prev = (const T*)s->at(P.off_Z); dz_prev = (T*)s->at(P.off_dZ); act_prev = P.act; }
+  }
+  float* gpart = (float*)s->at(L.off_gpart);
+  ET_TRY(norm_dispatch(L.N, [&](auto vpl) -> et_status {
+    constexpr int V = decltype(vpl)::value;
+    auto go = [&](auto kern) -> et_status {
+      kern<<<L.norm_blocks, et::kNormThreads, 0, st>>>(dz_src<T>(s, l, dY), act_in<T>(s, l),
+                                                        (const float2*)s->at(L.off_stats), (const T*)L.W, skip, G_in,
+                                                        z_prev, dz_prev, act_prev, gpart, (int)s->M, L.N);
+      return after_launch();
+    };
+    if (want_dx && want_dgamma) return go(et::norm_backward_kernel<T, V, true, true>);
+    if (want_dx) return go(et::norm_backward_kernel<T, V, true, false>);
+    return go(et::norm_backward_kernel<T, V, false, true>);
+  }));
+  ++*launches;
+  if (!want_dgamma || (grad == nullptr && delta == nullptr && !sgd)) return ET_OK;
+  float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
+  et::bias_finish_kernel<T><<<L.imp_count_w, dim3(et::kBiasCols, et::kBiasLanes), 0, st>>>(
+      gpart, L.norm_blocks, L.N, L.N, grad, delta, imp, (T*)L.W, opt_params(s, lr), sgd ? 1 : 0,
+      s->delta_is_snapshot ? 1 : 0, L.W32, L.st1[0], L.st2[0]);
+  ++*launches;
+  return after_launch();
+}
+
 // dW_l = a_l^T dZ_l as split partials, then the reducer with grad / importance / SGD.
 template <typename T>
 et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
@@ -673,17 +752,31 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
     if (two) CU_TRY(cudaEventRecord(s->chain_ev[L], cs));  // dZ_{L-1} is ready
     for (int l = L - 1; l >= d; --l) {
       const LayerRT& Y = s->ly[l];
-      const double gemm = 2.0 * (double)s->M * Y.K * Y.N;
+      const bool norm = Y.kind == ET_LAYER_NORM;
+      const double gemm = norm ? 0.0 : 2.0 * (double)s->M * Y.K * Y.N;
       if (mask[2 * l + 1]) {
         // On the tensor-core path the column partials of dZ_l were left by dgrad(l+1) in this
         // layer's own buffer; finishing them need not sit on the chain's critical path.
-        const int fused = (is_bf16<T>::value && l < L - 1) ? dgrad_row_blocks(s, l + 1) : 0;
+        // (A normalisation layer above leaves none: the column-sum kernel runs instead.)
+        const int fused = (is_bf16<T>::value && l < L - 1 && s->ly[l + 1].kind == ET_LAYER_DENSE)
+                              ? dgrad_row_blocks(s, l + 1) : 0;
         // Which stream: with few selected kernels the caller's stream is nearly idle and takes
         // the finishers off the chain; with many it is the busier one and the chain keeps them.
         cudaStream_t bs = s->wgrad_one_unit ? st : cs;
         if (two && bs == st) CU_TRY(cudaStreamWaitEvent(st, s->chain_ev[l + 1], 0));
         ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
                                   delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, bs, fused));
+      }
+      if (norm) {
+        // one kernel passes the error gradient on (above the deepest selected layer) and leaves the
+        // partials of d gamma (if selected); it reads gamma, so the finisher that may update gamma
+        // follows it on the same stream
+        if (l > d || mask[2 * l]) {
+          ET_TRY(run_norm_backward<T>(s, l, dY, l > d, mask[2 * l] != 0, grads ? grads[2 * l] : nullptr,
+                                      delta ? (const T*)delta[2 * l] : nullptr, sgd, lr, &launches, cs));
+        }
+        if (two && l > d) CU_TRY(cudaEventRecord(s->chain_ev[l], cs));
+        continue;
       }
       if (l > d) {
         ET_TRY(run_dgrad_layer<T>(s, l, dY, cs, mask[2 * (l - 1) + 1] != 0));
@@ -744,7 +837,10 @@ et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
     }
   }
   s->x = x;
-  for (int l = 0; l < s->L; ++l) ET_TRY(run_forward_layer<T>(s, l, y, st));
+  for (int l = 0; l < s->L; ++l) {
+    if (s->ly[l].kind == ET_LAYER_NORM) ET_TRY(run_norm_forward<T>(s, l, y, st));
+    else ET_TRY(run_forward_layer<T>(s, l, y, st));
+  }
   s->forwarded = true;
   return ET_OK;
 }
@@ -786,6 +882,14 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (d.fold > 1 && d.act != ET_ACT_NONE) { err = ET_ERR_UNSUPPORTED; break; }
     y.K = d.in_features; y.N = d.out_features; y.fold = d.fold; y.Nw = d.out_features / d.fold;
     y.act = d.act; y.residual_src = d.residual_src;
+    if (d.kind != ET_LAYER_DENSE && d.kind != ET_LAYER_NORM) { err = ET_ERR_INVALID_ARG; break; }
+    y.kind = d.kind; y.eps = d.eps;
+    if (y.kind == ET_LAYER_NORM) {
+      if (y.K != y.N || y.fold != 1 || y.act != ET_ACT_NONE || y.residual_src != -1 || !(y.eps >= 0.f)) {
+        err = ET_ERR_INVALID_ARG; break;
+      }
+      if (y.N % 8 || y.N > et::kNormMaxWidth) { err = ET_ERR_UNSUPPORTED; break; }
+    }
     if (y.K != width[l]) { err = ET_ERR_SHAPE; break; }
     width[l + 1] = y.Nw;
     if (d.residual_src < -1 || d.residual_src > l) { err = ET_ERR_INVALID_ARG; break; }
@@ -817,7 +921,11 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     const size_t act_bytes = (size_t)M * y.Nw * s->elt;
     if (l < L - 1) { y.off_a_out = take(act_bytes); y.off_G_out = take(act_bytes); }
     if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
-    if (dtype == ET_BF16) {
+    if (y.kind == ET_LAYER_NORM) {
+      y.off_stats = take((size_t)M * sizeof(float2));
+      y.norm_blocks = std::min(ceil_div(M, et::kNormWarps), s->sms * 4);
+      y.off_gpart = take((size_t)y.norm_blocks * y.N * sizeof(float));
+    } else if (dtype == ET_BF16) {
       const int kb_n = ceil_div(y.Nw, et::tc::BK) * y.fold;
       const TilePlan f = choose_tiles((int)M, y.Nw, ceil_div(y.K, et::tc::BK) * y.fold, s->sms, false, false, 0);
       const TilePlan d = choose_tiles((int)M, y.K, kb_n, s->sms, false, true, 0);
@@ -836,9 +944,11 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
         }
       }
     }
-    max_partial = std::max(max_partial, (size_t)y.split * y.K * y.N * sizeof(float));
+    max_partial = std::max(max_partial, y.kind == ET_LAYER_NORM ? (size_t)y.N * sizeof(float)
+                                                                : (size_t)y.split * y.K * y.N * sizeof(float));
     y.off_biaspart = take((size_t)std::max(chunks, ceil_div(M, 256) * 8 + 8) * y.Nw * sizeof(float));
-    y.imp_count_w = ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
+    y.imp_count_w = y.kind == ET_LAYER_NORM ? ceil_div(y.N, et::kBiasCols)
+                                            : ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
     y.imp_count_b = ceil_div(y.N, et::kBiasCols);
     s->imp_offs[2 * l] = imp_total; s->imp_counts[2 * l] = y.imp_count_w; imp_total += y.imp_count_w;
     s->imp_offs[2 * l + 1] = imp_total; s->imp_counts[2 * l + 1] = y.imp_count_b; imp_total += y.imp_count_b;
@@ -886,8 +996,10 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   if (s->dtype == ET_BF16) {
     for (int l = 0; l < s->L; ++l) {
       LayerRT& y = s->ly[l];
-      ET_TRY(make_tmaps(&y.map_W, y.W, y.N, y.K));
-      ET_TRY(make_map(&y.map_Wd, y.W, y.N, y.K, y.pair_dgrad ? y.bn_dgrad / 2 : y.bn_dgrad));
+      if (y.kind != ET_LAYER_NORM) {
+        ET_TRY(make_tmaps(&y.map_W, y.W, y.N, y.K));
+        ET_TRY(make_map(&y.map_Wd, y.W, y.N, y.K, y.pair_dgrad ? y.bn_dgrad / 2 : y.bn_dgrad));
+      }
       if (l < s->L - 1) {
         ET_TRY(make_tmaps(&y.map_aout, s->at(y.off_a_out), y.Nw, s->M));
         ET_TRY(make_tmaps(&y.map_Gout, s->at(y.off_G_out), y.Nw, s->M));
@@ -997,14 +1109,15 @@ et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
     if (!mask[t]) continue;
     const LayerRT& y = s->ly[t / 2];
     const bool is_w = (t & 1) == 0;
-    const size_t count = is_w ? (size_t)y.K * y.N : (size_t)y.N;
+    const size_t count = is_w ? y.w_count() : (size_t)y.N;
     const int blocks = s->imp_counts[t];
     float* out = parts + s->imp_offs[t];
+    const bool wide = is_w && y.kind != ET_LAYER_NORM;       // 8 elements per thread; gamma goes like a bias
     if (s->dtype == ET_BF16) {
-      if (is_w) et::importance_kernel<bf16, 8><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const bf16*)delta[t], count, out);
+      if (wide) et::importance_kernel<bf16, 8><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const bf16*)delta[t], count, out);
       else      et::importance_kernel<bf16, 1><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const bf16*)delta[t], count, out);
     } else {
-      if (is_w) et::importance_kernel<float, 8><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const float*)delta[t], count, out);
+      if (wide) et::importance_kernel<float, 8><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const float*)delta[t], count, out);
       else      et::importance_kernel<float, 1><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const float*)delta[t], count, out);
     }
     ET_TRY(after_launch());
@@ -1028,7 +1141,7 @@ et_status update_masked_impl(et_stack* s, const uint8_t* mask, int32_t n_tensors
     if (!mask[t]) continue;
     const LayerRT& y = s->ly[t / 2];
     const bool is_w = (t & 1) == 0;
-    const size_t count = is_w ? (size_t)y.K * y.N : (size_t)y.N;
+    const size_t count = is_w ? y.w_count() : (size_t)y.N;
     void* w = is_w ? y.W : y.b;
     float* m = is_w ? y.W32 : y.b32;
     float* s1 = y.st1[t & 1];
@@ -1122,6 +1235,20 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
     for (int l = L - 1; l >= 0; --l) {
       int dummy = 0;
       t_dy[2 * l] = 0.0; t_dy[2 * l + 1] = 0.0;
+      if (s->ly[l].kind == ET_LAYER_NORM) {
+        // Section 5.2: the layer is one black box whose whole backward time belongs to t_dy of beta
+        t_dw[2 * l] = 0.0; t_dw[2 * l + 1] = 0.0;
+        double t_box = 0.0, t_beta = 0.0;
+        if (s->dtype == ET_BF16) {
+          ET_TRY(timed([&]() { return run_norm_backward<bf16>(s, l, dY, l >= 1, true, scratch_grad, nullptr, false, 0.f, &dummy, st); }, &t_box));
+          ET_TRY(timed([&]() { return run_bgrad_layer<bf16>(s, l, dY, nullptr, nullptr, false, 0.f, &dummy, st); }, &t_beta));
+        } else {
+          ET_TRY(timed([&]() { return run_norm_backward<float>(s, l, dY, l >= 1, true, scratch_grad, nullptr, false, 0.f, &dummy, st); }, &t_box));
+          ET_TRY(timed([&]() { return run_bgrad_layer<float>(s, l, dY, nullptr, nullptr, false, 0.f, &dummy, st); }, &t_beta));
+        }
+        t_dy[2 * l + 1] = t_box + t_beta;
+        continue;
+      }
       if (s->dtype == ET_BF16) {
         if (l >= 1) ET_TRY(timed([&]() { return run_dgrad_layer<bf16>(s, l, dY, st); }, &t_dy[2 * l]));
         ET_TRY(timed([&]() { return run_wgrad_layer<bf16>(s, l, dY, scratch_grad, nullptr, false, 0.f, &dummy, st); }, &t_dw[2 * l]));
