@@ -404,7 +404,7 @@ def run_side(args):
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
-    w = wl.resnet_1x1() if args.workload == "resnet" else wl.vit_l()
+    w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "schedule": wl.vit_l}[args.workload]()
     tdt = torch.bfloat16
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
     stack = et.et_stack_create(w.layers, w.M, w.dtype)
@@ -417,7 +417,7 @@ def run_side(args):
     et.et_forward_stack(stack, x, y)
     et.et_loss_mse_grad(stack, y, target, dY, None)
     torch.cuda.synchronize()
-    if args.workload == "resnet":
+    if args.workload in ("resnet", "prenorm"):
         rep = et.Report(w.L)
         delta = [to_dev(d) for d in wl.draw_delta(w, 5)]
         imp = torch.zeros(2 * w.L, dtype=torch.float32, device=dev)
@@ -463,7 +463,33 @@ def run_side(args):
         except Exception as exc:                      # report, do not hide
             gms = gfms = None
             print("graph capture failed:", exc, file=sys.stderr)
-        print(json.dumps({"report": "resnet50_conv4_1x1_bf16", "elastic_ms": ms, "elastic_tflops": fl / ms / 1e9,
+        extra = {}
+        if args.workload == "prenorm":
+            # normalisation kernels alone: CUDA-event time of their class over full-backprop steps against
+            # the bytes they must move (g, x, skip gradient in; error gradient out; bf16)
+            ones = np.ones(2 * w.L, dtype=np.uint8)
+            et.et_timing_enable(stack, True)
+            for _ in range(5):
+                et.et_backward_elastic(stack, dY, ones, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep)
+            t = et.et_timing_read(stack)
+            et.et_timing_enable(stack, False)
+            n_norm = sum(1 for l, ly in enumerate(w.layers) if ly.kind == wl.KIND_NORM and l > 0)
+            nbytes = n_norm * 4.0 * w.M * w.layers[0].out_features * 2
+            norm_ms = t["norm"][0] / 5
+            peaks = _peaks()
+            extra = {"norm_backward_ms_per_step": norm_ms, "norm_launches_per_step": t["norm"][1] / 5,
+                     "norm_backward_gbs": nbytes / norm_ms / 1e6,
+                     "norm_frac_of_hbm_peak": nbytes / norm_ms / 1e6 / peaks["hbm_gbs"],
+                     "norm_note": "class time includes the gamma finishing kernels; bytes count the row kernels only"}
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(args.steps):
+                et.et_forward_stack(stack, x, y)
+            e1.record()
+            torch.cuda.synchronize()
+            extra["forward_ms"] = e0.elapsed_time(e1) / args.steps
+        print(json.dumps({"report": w.name, **extra, "elastic_ms": ms, "elastic_tflops": fl / ms / 1e9,
                           "elastic_launches": n, "full_ms": fms, "full_tflops": ffl / fms / 1e9, "full_launches": fn,
                           "elastic_graph_ms": gms, "full_graph_ms": gfms,
                           "selected_tensors": int(w.mask.sum())}))
@@ -507,7 +533,7 @@ def main():
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
-    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "schedule"],
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "schedule"],
                     help="vit_b = the benchmark line; resnet / schedule = side reports for the other shapes")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup

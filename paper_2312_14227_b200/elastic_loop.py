@@ -85,6 +85,12 @@ def flop_costs(layers, M):
     for when measured times are not wanted."""
     t_dw, t_dy = [], []
     for ly in layers:
+        if getattr(ly, "kind", 0) == 1:
+            # normalisation layer: one pass over the rows, all of it charged to beta's error-gradient
+            # time (Section 5.2)
+            t_dw += [0.0, 0.0]
+            t_dy += [0.0, 8.0 * M * ly.out_features]
+            continue
         f = 2.0 * M * ly.in_features * ly.out_features
         t_dw += [f, float(M * ly.out_features)]
         t_dy += [f, 0.0]
