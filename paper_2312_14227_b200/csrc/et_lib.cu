@@ -519,14 +519,35 @@ et_status norm_dispatch(int d, F&& f) {
   return ET_ERR_UNSUPPORTED;
 }
 
+// Blocks of a row kernel that fit on one SM at a time (by registers and shared memory): grids are sized
+// to exactly one resident wave, so that no block starts late into a half-empty GPU.  The kernels differ
+// only in template arguments (one pointer type for all), so the answer is remembered per function address.
+template <class K>
+int norm_blocks_per_sm(K kern) {
+  struct Seen { const void* fn; int dev, per_sm; };
+  static std::vector<Seen> seen;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 1; }
+  for (const auto& e : seen)
+    if (e.fn == (const void*)kern && e.dev == dev) return e.per_sm;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, et::kNormThreads, 0) != cudaSuccess || per_sm < 1) {
+    (void)cudaGetLastError();
+    per_sm = 1;
+  }
+  seen.push_back({(const void*)kern, dev, per_sm});
+  return per_sm;
+}
+
 template <typename T>
 et_status run_norm_forward(et_stack* s, int l, void* y, cudaStream_t st) {
   TimedLaunch tl(s, ET_K_NORM, st);
   const LayerRT& L = s->ly[l];
   T* out = l == s->L - 1 ? (T*)y : (T*)s->at(L.off_a_out);
-  const int blocks = std::min(ceil_div(s->M, et::kNormWarps), s->sms * 8);
   return norm_dispatch(L.N, [&](auto vpl) -> et_status {
-    et::norm_forward_kernel<T, decltype(vpl)::value><<<blocks, et::kNormThreads, 0, st>>>(
+    auto kern = et::norm_forward_kernel<T, decltype(vpl)::value>;
+    const int grid = std::min(ceil_div(s->M, et::kNormWarps), s->sms * norm_blocks_per_sm(kern));
+    kern<<<grid, et::kNormThreads, 0, st>>>(
         act_in<T>(s, l), (const T*)L.W, (const T*)L.b, out, (float2*)s->at(L.off_stats), (int)s->M, L.N, L.eps);
     return after_launch();
   });
@@ -555,12 +576,13 @@ et_status run_norm_backward(et_stack* s, int l, const void* dY, bool want_dx, bo
     if (need_act) { z_prev = (const T*)s->at(P.off_Z); dz_prev = (T*)s->at(P.off_dZ); act_prev = P.act; }
   }
   float* gpart = (float*)s->at(L.off_gpart);
+  int grid = 0;                       // blocks launched = rows of gpart written (at most L.norm_blocks)
   ET_TRY(norm_dispatch(L.N, [&](auto vpl) -> et_status {
     constexpr int V = decltype(vpl)::value;
     auto go = [&](auto kern) -> et_status {
-      kern<<<L.norm_blocks, et::kNormThreads, 0, st>>>(dz_src<T>(s, l, dY), act_in<T>(s, l),
-                                                        (const float2*)s->at(L.off_stats), (const T*)L.W, skip, G_in,
-                                                        z_prev, dz_prev, act_prev, gpart, (int)s->M, L.N);
+      grid = std::min(L.norm_blocks, s->sms * norm_blocks_per_sm(kern));
+      kern<<<grid, et::kNormThreads, 0, st>>>(dz_src<T>(s, l, dY), act_in<T>(s, l), (const float2*)s->at(L.off_stats),
+                                              (const T*)L.W, skip, G_in, z_prev, dz_prev, act_prev, gpart, (int)s->M, L.N);
       return after_launch();
     };
     if (want_dx && want_dgamma) return go(et::norm_backward_kernel<T, V, true, true>);
@@ -571,7 +593,7 @@ et_status run_norm_backward(et_stack* s, int l, const void* dY, bool want_dx, bo
   if (!want_dgamma || (grad == nullptr && delta == nullptr && !sgd)) return ET_OK;
   float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
   et::bias_finish_kernel<T><<<L.imp_count_w, dim3(et::kBiasCols, et::kBiasLanes), 0, st>>>(
-      gpart, L.norm_blocks, L.N, L.N, grad, delta, imp, (T*)L.W, opt_params(s, lr), sgd ? 1 : 0,
+      gpart, grid, L.N, L.N, grad, delta, imp, (T*)L.W, opt_params(s, lr), sgd ? 1 : 0,
       s->delta_is_snapshot ? 1 : 0, L.W32, L.st1[0], L.st2[0]);
   ++*launches;
   return after_launch();
@@ -923,7 +945,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
     if (y.kind == ET_LAYER_NORM) {
       y.off_stats = take((size_t)M * sizeof(float2));
-      y.norm_blocks = std::min(ceil_div(M, et::kNormWarps), s->sms * 4);
+      y.norm_blocks = std::min(ceil_div(M, et::kNormWarps), s->sms * 8);
       y.off_gpart = take((size_t)y.norm_blocks * y.N * sizeof(float));
     } else if (dtype == ET_BF16) {
       const int kb_n = ceil_div(y.Nw, et::tc::BK) * y.fold;
