@@ -392,6 +392,65 @@ def run_own(args):
         dist.destroy_process_group()
 
 
+def run_selector(args):
+    """Host-side selector report (Section 6.3): how many subproblems the two prunings remove, how the
+    solution and the time of the dynamic program move with the resolution T_q (Eq. 8), and how the
+    time falls with threads when there are thousands of tensors.  No GPU work."""
+    import time
+    import paper_2312_14227_b200 as et
+    from paper_2312_14227_b200.elastic_loop import flop_costs
+
+    def timed(fn, reps=3):
+        best = None
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            out = fn()
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        return out, 1e3 * best
+
+    rng = np.random.default_rng(7)
+    out = {"report": "selector (host dynamic program)"}
+    # the ViT-L-shaped stack's 192 tensors with costs proportional to their work, rho = 0.5
+    w = wl.vit_l(params=False)
+    t_dw, t_dy = flop_costs(w.layers, w.M)
+    I = rng.random(2 * w.L)
+    t_fwd = 0.5 * float(t_dw.sum() + t_dy.sum()) / 2.0
+    sweep = []
+    ref_val = None
+    for Tq in (10, 100, 1000, 10000, 100000):
+        (mask, val, est, st), ms = timed(lambda: et.et_select_dp_ex(I, t_dw, t_dy, t_fwd, 0.5, Tq))
+        (_, val_full, _, st_full), ms_full = timed(lambda: et.et_select_dp_ex(I, t_dw, t_dy, t_fwd, 0.5, Tq, prune=False), 1) \
+            if Tq <= 10000 else ((None, val, None, None), None)
+        assert abs(val_full - val) < 1e-9
+        budget = 0.5 * (t_fwd + t_dw.sum() + t_dy.sum()) - t_fwd
+        sweep.append({"Tq": Tq, "value": val, "selected": int(mask.sum()), "time_over_budget": float(est / budget),
+                      "dp_ms": ms, "dp_ms_unpruned": ms_full, "subproblems_unpruned": st["table_full"],
+                      "without_invalid": st["table_budget"], "visited": st["visited"],
+                      "reduction": st["table_full"] / max(st["visited"], 1)})
+        ref_val = val
+    for e in sweep:
+        e["value_vs_finest"] = e["value"] / ref_val
+    out["vit_l_192_tensors_rho_0.5"] = sweep
+    # thousands of tensors
+    big = []
+    for n, Tq in ((2048, 2000), (4096, 4000)):
+        I2, w2, y2 = wl.selector_instance(rng, n, integer=False)
+        row = {"n": n, "Tq": Tq, "rho": 0.4}
+        base = None
+        for threads in (1, 4, 16):
+            (mask, val, est, st), ms = timed(lambda: et.et_select_dp_ex(I2, w2, y2, 10.0, 0.4, Tq, threads=threads), 2)
+            base = val if base is None else base
+            assert val == base
+            row[f"ms_{threads}_threads"] = ms
+            row["threads_used_%d" % threads] = st["threads"]
+        row["transitions"] = st["transitions"]
+        big.append(row)
+    out["large_instances"] = big
+    out["host_cores"] = os.cpu_count()
+    print(json.dumps(out))
+
+
 def run_side(args):
     """Side reports for the other workload shapes (not the benchmark line): one JSON line each.
     resnet: ResNet-50 conv4_x 1x1 stack, elastic vs full step time (launch-bound GEMMs).
@@ -533,11 +592,14 @@ def main():
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
-    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "schedule"],
-                    help="vit_b = the benchmark line; resnet / schedule = side reports for the other shapes")
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "schedule", "selector"],
+                    help="vit_b = the benchmark line; resnet / prenorm / schedule = side reports for the other shapes; "
+                         "selector = host-side report on the selection dynamic program")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup
-    if args.workload != "vit_b":
+    if args.workload == "selector":
+        run_selector(args)
+    elif args.workload != "vit_b":
         run_side(args)
     elif args.impl == "reference":
         run_reference(args)

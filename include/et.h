@@ -225,6 +225,16 @@ et_status et_backward_elastic_host(et_stack* s, const void* dY_host, const uint8
 et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads,
                         const void* const* delta, float* importance_dev, void* stream);
 
+/* The two importance metrics the paper compares Eq. 2 against in its ablation (Section 8, "Efficacy of
+ * Tensor Importance Evaluator"): weight magnitudes and gradient feedback.  The paper gives no formula
+ * for either; here they are the L1 norms  sum_i |w_i|  (of the tensors as bound, the fp32 masters
+ * when attached) and  sum_i |g_i|  (of materialised fp32 gradients, as et_backward_elastic exports
+ * them).  metric_dev receives n_tensors floats, 0 for unselected tensors.  Uses the importance
+ * scratch of the workspace: do not overlap with a backward call.  Asynchronous on `stream`. */
+typedef enum { ET_METRIC_WEIGHT_MAGNITUDE = 1, ET_METRIC_GRADIENT_MAGNITUDE = 2 } et_metric_kind;
+et_status et_tensor_metric(et_stack* s, const uint8_t* mask, int32_t n_tensors, int32_t kind,
+                           float* const* grads, float* metric_dev, void* stream);
+
 /* Stand-alone masked SGD: w_k <- w_k - lr * grads[k] for selected k (fp32 arithmetic,
  * rounded once to the storage dtype), whatever optimiser is configured.  Unselected tensors
  * are never written. */
@@ -289,6 +299,29 @@ et_status et_time_selective(const uint8_t* mask, const double* t_dw, const doubl
 et_status et_select_dp(const double* importance, const double* t_dw, const double* t_dy, int32_t n,
                        double t_fwd, double rho, int32_t Tq, int32_t variant,
                        uint8_t* mask_out, double* value_out, double* est_time_out);
+
+/* What a run of the selector's dynamic program did (Section 6.3 counts subproblems). */
+typedef struct {
+  int64_t table_full;     /* n * (T + 1): subproblems of the unpruned table, t up to the full (quantised) backward time T */
+  int64_t table_budget;   /* n * (budget + 1): without the invalid ones, whose t exceeds the time constraint */
+  int64_t visited;        /* (k, t) entries evaluated: also without the redundant ones, whose t cannot even pay
+                             the error-gradient path down to tensor k */
+  int64_t transitions;    /* (k, k_c, t) candidates compared (the O(N^2 T) work of Section 6.2) */
+  int32_t rows_reached;   /* tensors, from the output, that the budget reaches at all */
+  int32_t threads;        /* threads that took part */
+} et_dp_stats;
+
+/* et_select_dp with the choices of Sections 6.3 exposed: `prune` = 1 skips invalid and redundant
+ * subproblems (the default of et_select_dp), 0 evaluates the whole table, which must give a selection of
+ * the same value; `threads` >= 1 host threads share each row of the table (for N in the thousands,
+ * Section 6.3's last paragraph); `stats` may be NULL.  Host only, synchronous. */
+et_status et_select_dp_ex(const double* importance, const double* t_dw, const double* t_dy, int32_t n,
+                          double t_fwd, double rho, int32_t Tq, int32_t variant, int32_t threads,
+                          int32_t prune, uint8_t* mask_out, double* value_out, double* est_time_out,
+                          et_dp_stats* stats);
+et_status et_select_dp_int_ex(const double* importance, const int64_t* t_dw, const int64_t* t_dy,
+                              int32_t n, int64_t budget, int32_t variant, int32_t threads, int32_t prune,
+                              uint8_t* mask_out, double* value_out, et_dp_stats* stats);
 
 /* Same problem with integer costs given directly (no quantisation step). */
 et_status et_select_dp_int(const double* importance, const int64_t* t_dw, const int64_t* t_dy,

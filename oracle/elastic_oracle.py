@@ -224,6 +224,19 @@ def importance(grads: Dict[int, np.ndarray], delta: Sequence[np.ndarray], mask) 
     return out
 
 
+def magnitude_metric(tensors: Sequence[np.ndarray], mask) -> np.ndarray:
+    """The non-additive metrics of the paper's ablation (Section 8, importance evaluator): the paper
+    names them (weight magnitudes, gradient feedback) without a formula; read here as the L1 norm
+    sum_i |x_i| of each selected tensor -- its weights for the first, its gradient for the second;
+    0 for the others.  Unpinned against the paper (it prints no values); the tests pin it to the
+    definition on hand-written vectors."""
+    out = np.zeros(len(mask))
+    for k, m in enumerate(mask):
+        if m:
+            out[k] = float(np.sum(np.abs(np.asarray(tensors[k], dtype=np.float64))))
+    return out
+
+
 def sgd_masked(params: Sequence[np.ndarray], grads: Dict[int, np.ndarray], mask, lr: float):
     """w <- w - lr * g for selected tensors; the others are returned untouched
     (same object, so a caller can check they were not rewritten)."""

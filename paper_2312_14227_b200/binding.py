@@ -44,6 +44,14 @@ class et_optimizer_config(C.Structure):
 ET_OPT_SGD, ET_OPT_SGDW, ET_OPT_ADAM = 0, 1, 2
 
 
+class et_dp_stats(C.Structure):
+    _fields_ = [("table_full", C.c_int64), ("table_budget", C.c_int64), ("visited", C.c_int64),
+                ("transitions", C.c_int64), ("rows_reached", C.c_int32), ("threads", C.c_int32)]
+
+    def as_dict(self):
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
 class et_exec_report(C.Structure):
     _fields_ = [("dgrad", C.c_void_p), ("wgrad", C.c_void_p), ("bgrad", C.c_void_p), ("updated", C.c_void_p),
                 ("deepest", C.c_int32), ("launches", C.c_int32), ("flops_executed", C.c_double)]
@@ -61,6 +69,7 @@ _SIGS = {
     "et_backward_elastic": [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _u32, _f32, _vp, _vp],
     "et_backward_elastic_host": [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _u32, _f32, _vp, _vp],
     "et_importance": [_vp, _vp, _i32, _vp, _vp, _vp, _vp],
+    "et_tensor_metric": [_vp, _vp, _i32, _i32, _vp, _vp, _vp],
     "et_sgd_masked": [_vp, _vp, _i32, _vp, _f32, _vp],
     "et_update_masked": [_vp, _vp, _i32, _vp, _f32, _vp],
     "et_stack_set_optimizer": [_vp, _vp, _vp, _vp],
@@ -69,6 +78,8 @@ _SIGS = {
     "et_time_selective": [_vp, _vp, _vp, _i32, _i32, _vp],
     "et_select_dp": [_vp, _vp, _vp, _i32, _f64, _f64, _i32, _i32, _vp, _vp, _vp],
     "et_select_dp_int": [_vp, _vp, _vp, _i32, _i64, _i32, _vp, _vp],
+    "et_select_dp_ex": [_vp, _vp, _vp, _i32, _f64, _f64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp],
+    "et_select_dp_int_ex": [_vp, _vp, _vp, _i32, _i64, _i32, _i32, _i32, _vp, _vp, _vp],
     "et_device_status": [_vp, _vp],
     "et_bias_grad_noalloc": [_vp, _i64, _i32, _i32, _vp, _vp],
     "et_timing_enable": [_vp, _i32],
@@ -157,6 +168,35 @@ def et_select_dp(importance, t_dw, t_dy, t_fwd: float, rho: float, Tq: int = 100
     _check(_lib.et_select_dp(_ptr(I), _ptr(w), _ptr(y), n, t_fwd, rho, Tq, variant, _ptr(mask),
                              C.addressof(val), C.addressof(est)), "et_select_dp")
     return mask[:n], val.value, est.value
+
+
+def et_select_dp_ex(importance, t_dw, t_dy, t_fwd: float, rho: float, Tq: int = 1000, variant: int = ET_COST_STRICT,
+                    threads: int = 1, prune: bool = True):
+    """et_select_dp with the thread count and the pruning switch; also returns the run's et_dp_stats as a dict."""
+    I = np.ascontiguousarray(importance, dtype=np.float64)
+    w = np.ascontiguousarray(t_dw, dtype=np.float64)
+    y = np.ascontiguousarray(t_dy, dtype=np.float64)
+    n = len(I)
+    mask = np.zeros(max(n, 1), dtype=np.uint8)
+    val, est = C.c_double(), C.c_double()
+    st = et_dp_stats()
+    _check(_lib.et_select_dp_ex(_ptr(I), _ptr(w), _ptr(y), n, t_fwd, rho, Tq, variant, threads, 1 if prune else 0,
+                                _ptr(mask), C.addressof(val), C.addressof(est), C.addressof(st)), "et_select_dp_ex")
+    return mask[:n], val.value, est.value, st.as_dict()
+
+
+def et_select_dp_int_ex(importance, t_dw, t_dy, budget: int, variant: int = ET_COST_STRICT, threads: int = 1,
+                        prune: bool = True):
+    I = np.ascontiguousarray(importance, dtype=np.float64)
+    w = np.ascontiguousarray(t_dw, dtype=np.int64)
+    y = np.ascontiguousarray(t_dy, dtype=np.int64)
+    n = len(I)
+    mask = np.zeros(max(n, 1), dtype=np.uint8)
+    val = C.c_double()
+    st = et_dp_stats()
+    _check(_lib.et_select_dp_int_ex(_ptr(I), _ptr(w), _ptr(y), n, int(budget), variant, threads, 1 if prune else 0,
+                                    _ptr(mask), C.addressof(val), C.addressof(st)), "et_select_dp_int_ex")
+    return mask[:n], val.value, st.as_dict()
 
 
 def et_select_dp_int(importance, t_dw, t_dy, budget: int, variant: int = ET_COST_STRICT):
@@ -279,6 +319,16 @@ def et_importance(s: Stack, mask, grads, delta, importance_dev, stream=None):
     m = _mask_arr(mask)
     _check(_lib.et_importance(s.handle, _ptr(m), len(m), _ptr_array(grads, len(m)), _ptr_array(delta, len(m)),
                               _ptr(importance_dev), _stream_ptr(stream)), "et_importance")
+
+
+ET_METRIC_WEIGHT_MAGNITUDE, ET_METRIC_GRADIENT_MAGNITUDE = 1, 2
+
+
+def et_tensor_metric(s: Stack, mask, kind: int, grads, metric_dev, stream=None):
+    m = _mask_arr(mask)
+    g = _ptr_array(grads, len(m)) if grads is not None else None
+    _check(_lib.et_tensor_metric(s.handle, _ptr(m), len(m), kind, g, _ptr(metric_dev), _stream_ptr(stream)),
+           "et_tensor_metric")
 
 
 def et_sgd_masked(s: Stack, mask, grads, lr: float, stream=None):

@@ -29,7 +29,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         "-gencode", "arch=compute_100a,code=sm_100a",
         "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=default",
         "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-        "-cudart", "static",
+        "-cudart", "static", "-Xcompiler", "-pthread",
     ]
     if verbose:
         cmd += ["-Xptxas", "-v"]

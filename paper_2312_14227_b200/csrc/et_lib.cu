@@ -1150,6 +1150,44 @@ et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
   return after_launch();
 }
 
+et_status et_tensor_metric(et_stack* s, const uint8_t* mask, int32_t n_tensors, int32_t kind, float* const* grads,
+                           float* metric_dev, void* stream) {
+  ET_TRY(check_ready(s, mask, n_tensors));
+  if (metric_dev == nullptr) return ET_ERR_INVALID_ARG;
+  if (kind != ET_METRIC_WEIGHT_MAGNITUDE && kind != ET_METRIC_GRADIENT_MAGNITUDE) return ET_ERR_INVALID_ARG;
+  if (kind == ET_METRIC_GRADIENT_MAGNITUDE) {
+    if (grads == nullptr) return ET_ERR_INVALID_ARG;
+    for (int t = 0; t < n_tensors; ++t)
+      if (mask[t] && grads[t] == nullptr) return ET_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  float* parts = (float*)s->at(s->off_imp_parts);
+  for (int t = 0; t < n_tensors; ++t) {
+    if (!mask[t]) continue;
+    const LayerRT& y = s->ly[t / 2];
+    const bool is_w = (t & 1) == 0;
+    const size_t count = is_w ? y.w_count() : (size_t)y.N;
+    const int blocks = s->imp_counts[t];
+    float* out = parts + s->imp_offs[t];
+    const bool wide = is_w && y.kind != ET_LAYER_NORM;
+    const float* f32 = kind == ET_METRIC_GRADIENT_MAGNITUDE ? grads[t] : (is_w ? y.W32 : y.b32);   // masters if attached
+    const void* stored = is_w ? y.W : y.b;
+    if (f32 != nullptr || s->dtype == ET_F32) {
+      const float* p = f32 != nullptr ? f32 : (const float*)stored;
+      if (wide) et::abs_sum_kernel<float, 8><<<blocks, et::kEltThreads, 0, st>>>(p, count, out);
+      else      et::abs_sum_kernel<float, 1><<<blocks, et::kEltThreads, 0, st>>>(p, count, out);
+    } else {
+      if (wide) et::abs_sum_kernel<bf16, 8><<<blocks, et::kEltThreads, 0, st>>>((const bf16*)stored, count, out);
+      else      et::abs_sum_kernel<bf16, 1><<<blocks, et::kEltThreads, 0, st>>>((const bf16*)stored, count, out);
+    }
+    ET_TRY(after_launch());
+  }
+  et::importance_finalize_kernel<<<n_tensors, 128, 0, st>>>(parts, (const int*)s->at(s->off_imp_offs),
+                                                            (const int*)s->at(s->off_imp_counts),
+                                                            mask_bits(mask, n_tensors), metric_dev);
+  return after_launch();
+}
+
 namespace {
 et_status update_masked_impl(et_stack* s, const uint8_t* mask, int32_t n_tensors, float* const* grads, float lr,
                              void* stream, bool plain) {

@@ -244,6 +244,23 @@ importance_kernel(const float* __restrict__ grad, const T* __restrict__ delta, s
   if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
 }
 
+// ---- magnitude of one tensor: block partials of sum |x| (V elements per thread) -------------
+template <typename T, int V>
+__global__ void __launch_bounds__(kEltThreads)
+abs_sum_kernel(const T* __restrict__ x, size_t count, float* __restrict__ part) {
+  const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * V;
+  float acc = 0.0f;
+  if (i0 < count) {
+    const int n = (int)min((size_t)V, count - i0);
+    float t[V];
+    load_seg<V>(x + i0, n, t);
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc += fabsf(t[i]);
+  }
+  acc = block_sum(acc);
+  if (threadIdx.x == 0) part[blockIdx.x] = acc;
+}
+
 // ---- stand-alone masked SGD on one selected tensor -----------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(kEltThreads)

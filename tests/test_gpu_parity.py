@@ -202,3 +202,26 @@ def test_device_status_reports_a_recorded_timeout():
     assert et.et_device_status(run.stack) == et.ET_ERR_TIMEOUT
     run.ws[:4] = 0
     assert et.et_device_status(run.stack) == et.ET_OK
+
+
+@pytest.mark.parametrize("dtype,tol", [(wl.DT_F32, TOL_F32), (wl.DT_BF16, TOL_BF16)])
+def test_ablation_metrics_weight_and_gradient_magnitude(dtype, tol):
+    # the two non-additive metrics of the paper's ablation, as stand-alone reductions
+    h = _h()
+    layers = [wl.Layer(72, 200, act=wl.ACT_RELU), wl.norm_layer(200), wl.Layer(200, 136)]
+    mask = np.array([1, 1, 1, 0, 1, 1], dtype=np.uint8)
+    w = wl.small_stack(layers, 300, dtype, 71, mask=mask, w_std=0.1, bias_std=0.05)
+    run = h.GpuRun(w)
+    run.forward_loss()
+    grads = run.alloc_grads(mask)
+    run.backward(mask, grads, None)
+    out = torch.full((6,), float("nan"), dtype=torch.float32, device=h.DEV)
+    et.et_tensor_metric(run.stack, mask, et.ET_METRIC_WEIGHT_MAGNITUDE, None, out)
+    want = orc.magnitude_metric(orc.tensors_of(w.W, w.b), mask)
+    got = h.to_np(out)
+    assert got[3] == 0.0 and np.all(np.abs(got - want) <= 1e-5 * np.abs(want) + 1e-12)      # inputs are exact in both
+    et.et_tensor_metric(run.stack, mask, et.ET_METRIC_GRADIENT_MAGNITUDE, grads, out)
+    ref = h.oracle_step(w, mask)
+    want = orc.magnitude_metric([ref["grads"].get(t) if mask[t] else None for t in range(6)], mask)
+    got = h.to_np(out)
+    assert got[3] == 0.0 and np.all(np.abs(got - want) <= tol * np.abs(want) + 1e-12)

@@ -154,3 +154,72 @@ def test_select_dp_quantised():
     I, t_dw, t_dy = wl.selector_instance(rng, 40, integer=False)
     mask, val, est = et.et_select_dp(I + 0.01, t_dw, t_dy, 3.0, 1.0, 1000, et.ET_COST_INCLUSIVE)
     assert mask.all()
+
+
+# ------------------------------------------------------------------ Section 6.3: pruning, threads, resolution
+@pytest.mark.parametrize("variant", [et.ET_COST_STRICT, et.ET_COST_INCLUSIVE])
+def test_pruned_and_threaded_dp_keep_the_optimum(variant):
+    # skipping invalid and redundant subproblems, and sharing rows between threads, must not change the
+    # value (Section 6.3: "without affecting optimality"); brute force is the referee
+    rng = np.random.default_rng(300 + variant)
+    for trial in range(80):
+        n = int(rng.integers(1, 13))
+        I, qw, qy = wl.selector_instance(rng, n, t_max=15)
+        qw, qy = qw.astype(np.int64), qy.astype(np.int64)
+        budget = int(rng.integers(0, int(qw.sum() + qy.sum()) + 3))
+        _, want = orc.select_bruteforce(I, qw, qy, budget, variant)
+        for prune in (True, False):
+            for threads in (1, 3):
+                mask, val, st = et.et_select_dp_int_ex(I, qw, qy, budget, variant, threads=threads, prune=prune)
+                assert abs(val - want) < 1e-12, (trial, prune, threads)
+                assert orc.t_selective(mask, qw, qy, variant) <= budget
+                assert abs(I[mask.astype(bool)].sum() - val) < 1e-12
+
+
+def test_dp_statistics_count_the_subproblems():
+    # 4 tensors, unit weight-gradient times, error-gradient times 0, 3, 0, 5 (forward order), budget 6.
+    # Counted from the output, tensor k costs at least low(k) = 1 + (error-gradient times above it):
+    # 1, 6, 6, 9.  The budget reaches three of them, and of their rows 7-1, 7-6 and 7-6 entries can hold a
+    # selection at all; no second tensor ever fits (every transition would start beyond t = 6).
+    I = np.array([1.0, 1.0, 1.0, 1.0])
+    w = np.array([1, 1, 1, 1], dtype=np.int64)
+    y = np.array([0, 3, 0, 5], dtype=np.int64)
+    mask, val, st = et.et_select_dp_int_ex(I, w, y, 6, et.ET_COST_STRICT)
+    assert st["table_full"] == 4 * (12 + 1) and st["table_budget"] == 4 * 7
+    assert st["rows_reached"] == 3 and st["visited"] == 6 + 1 + 1 and st["transitions"] == 0
+    assert val == 1.0 and mask.sum() == 1
+    _, _, full = et.et_select_dp_int_ex(I, w, y, 6, et.ET_COST_STRICT, prune=False)
+    assert full["rows_reached"] == 4 and full["visited"] == 4 * 13
+    assert full["transitions"] > st["transitions"]
+
+
+def test_threaded_dp_on_a_large_instance():
+    # N in the thousands: same value with 1 and 8 threads, and the same as the exact-cost knapsack route
+    rng = np.random.default_rng(17)
+    n = 1536
+    I, t_dw, t_dy = wl.selector_instance(rng, n, integer=False)
+    m1, v1, e1, s1 = et.et_select_dp_ex(I, t_dw, t_dy, 5.0, 0.4, 2000, et.ET_COST_STRICT, threads=1)
+    m8, v8, e8, s8 = et.et_select_dp_ex(I, t_dw, t_dy, 5.0, 0.4, 2000, et.ET_COST_STRICT, threads=8)
+    assert v1 == v8 and np.array_equal(m1, m8)
+    assert s1["visited"] == s8["visited"] < s1["table_budget"] < s1["table_full"]
+    assert s8["threads"] > 1 or (os.cpu_count() or 1) == 1      # rows this heavy are shared between threads
+    qw, qy, budget = orc.quantise(t_dw, t_dy, 5.0, 0.4, 2000)
+    assert abs(v1 - orc.select_by_depth_knapsack(I, qw, qy, budget, orc.STRICT)) < 1e-9
+
+
+def test_resolution_sweep_converges():
+    # Eq. 8: coarse resolutions blur the times; as T_q grows the selected value approaches the optimum of
+    # the finest resolution and the over-run of the true budget (at most one quantum per tensor) vanishes
+    rng = np.random.default_rng(23)
+    I, t_dw, t_dy = wl.selector_instance(rng, 60, integer=False)
+    T = t_dw.sum() + t_dy.sum()
+    t_fwd, rho = 4.0, 0.5
+    budget = rho * (t_fwd + T) - t_fwd
+    overrun, value = [], []
+    for Tq in (10, 100, 1000, 10000, 100000):
+        mask, val, est, _ = et.et_select_dp_ex(I, t_dw, t_dy, t_fwd, rho, Tq)
+        assert est <= budget + 2 * 60 * T / Tq + 1e-9
+        overrun.append(max(0.0, est - budget) / budget)
+        value.append(val)
+    assert overrun[-1] < 1e-3 and overrun[-1] <= overrun[0] + 1e-12
+    assert abs(value[-1] - value[-2]) <= 0.02 * value[-1]

@@ -264,3 +264,10 @@ def test_masked_backward_with_normalisation_layers():
     for t in grads:
         assert np.array_equal(grads[t], full[t])
     assert orc.executed_flops(layers, 5, plan) == 2.0 * 5 * (6 * 9 + 2 * 3 * 6)
+
+
+def test_magnitude_metric_is_the_l1_norm():
+    tensors = [np.array([[1.0, -2.0], [0.5, 0.0]]), np.array([-3.0, 4.0]), np.array([7.0])]
+    assert orc.magnitude_metric(tensors, [1, 1, 0]).tolist() == [3.5, 7.0, 0.0]
+    # unlike Eq. 2 it is not additive over a split of the update, and it ignores the sign of the effect
+    assert orc.magnitude_metric([-tensors[0]], [1])[0] == 3.5
