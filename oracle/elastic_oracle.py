@@ -18,6 +18,13 @@ or, for a normalisation layer (Section 5.2; its Gamma and Beta are tensors 2*l a
     xhat    = (a_l - mean) / sqrt(var + eps)         mean, var over the features of each row
     a_{l+1} = xhat * gamma_l + beta_l
 
+or, for an attention layer (no trainable tensors; Sections 5.3 / 5.4 count attention operations as
+non-trainable layers), with a_l = [q | k | v] (three blocks of `heads * head_dim` columns) and the
+rows grouped into sequences of `seq` consecutive tokens,
+
+    P       = softmax_over_keys( q_h k_h^T / sqrt(head_dim) )      per sequence and head h
+    a_{l+1} = [ P v_h ]_h                                          heads side by side
+
 Pins (tests/test_oracle_*.py): central finite differences of the loss for every
 tensor and every layer kind; the closed form of the importance sum when the update
 is a gradient step; the first-order Taylor identity of Eq. (6); masked == full
@@ -34,7 +41,7 @@ from typing import Dict, List, Optional, Sequence
 import numpy as np
 
 ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
-KIND_DENSE, KIND_NORM = 0, 1
+KIND_DENSE, KIND_NORM, KIND_ATTENTION = 0, 1, 2
 STRICT, INCLUSIVE = 0, 1
 
 
@@ -83,6 +90,20 @@ def forward(layers, W: Sequence[np.ndarray], b: Sequence[np.ndarray], x: np.ndar
     a = [np.asarray(x, dtype=np.float64)]
     Z = []
     for l, ly in enumerate(layers):
+        if _kind(ly) == KIND_ATTENTION:
+            d = ly.out_features
+            H, S = ly.heads, ly.seq
+            dh = d // H
+            B = a[l].shape[0] // S
+            q, k, v = (a[l][:, i * d:(i + 1) * d].reshape(B, S, H, dh).transpose(0, 2, 1, 3) for i in range(3))
+            s_ = q @ k.transpose(0, 1, 3, 2) / np.sqrt(dh)                  # [B, H, S(query), S(key)]
+            s_ = s_ - s_.max(axis=-1, keepdims=True)
+            P = np.exp(s_)
+            P = P / P.sum(axis=-1, keepdims=True)
+            o = (P @ v).transpose(0, 2, 1, 3).reshape(B * S, d)
+            Z.append((P, q, k, v))
+            a.append(o)
+            continue
         if _kind(ly) == KIND_NORM:
             # layer normalisation: per row, biased variance; Z keeps (xhat, 1/sqrt(var + eps))
             mean = a[l].mean(axis=1, keepdims=True)
@@ -147,7 +168,7 @@ def executed_flops(layers, M: int, plan: Plan) -> float:
     normalisation layers are not GEMMs and count nothing."""
     fl = 0.0
     for l, ly in enumerate(layers):
-        if _kind(ly) == KIND_NORM:
+        if _kind(ly) != KIND_DENSE:
             continue
         g = 2.0 * M * ly.in_features * ly.out_features
         fl += g * (int(plan.dgrad[l]) + int(plan.wgrad[l]))
@@ -165,6 +186,25 @@ def _backward_sweep(layers, W, saved: Saved, dY: np.ndarray, stop: int,
     for l in range(L - 1, stop - 1, -1):
         ly = layers[l]
         g_out = G[l + 1]
+        if _kind(ly) == KIND_ATTENTION:
+            if want_w[l]:
+                grads[2 * l] = np.zeros(0)                                  # its tensor slots are empty
+            if want_b[l]:
+                grads[2 * l + 1] = np.zeros(0)
+            if l > stop:
+                P, q, k, v = saved.Z[l]
+                B, H, S, dh = q.shape
+                d = H * dh
+                go = g_out.reshape(B, S, H, dh).transpose(0, 2, 1, 3)       # gradient of o, per head
+                dv = P.transpose(0, 1, 3, 2) @ go
+                dP = go @ v.transpose(0, 1, 3, 2)
+                # softmax: dS_ij = P_ij (dP_ij - sum_j' P_ij' dP_ij')
+                dS = P * (dP - (P * dP).sum(axis=-1, keepdims=True)) / np.sqrt(dh)
+                dq = dS @ k
+                dk = dS.transpose(0, 1, 3, 2) @ q
+                dX = np.concatenate([t.transpose(0, 2, 1, 3).reshape(B * S, d) for t in (dq, dk, dv)], axis=1)
+                G[l] = dX if G[l] is None else G[l] + dX
+            continue
         if _kind(ly) == KIND_NORM:
             xhat, rstd = saved.Z[l]
             if want_w[l]:

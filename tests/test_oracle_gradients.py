@@ -36,6 +36,8 @@ def _fd_check(layers, M, seed, h=1e-6, tol=2e-6):
             p = arr_list[l]
             g = grads[t]
             assert g.shape == p.shape
+            if p.size == 0:                          # a layer without trainable tensors
+                continue
             idxs = [tuple(rng.integers(0, s) for s in p.shape) for _ in range(12)]
             for idx in idxs:
                 old = p[idx]
@@ -271,3 +273,52 @@ def test_magnitude_metric_is_the_l1_norm():
     assert orc.magnitude_metric(tensors, [1, 1, 0]).tolist() == [3.5, 7.0, 0.0]
     # unlike Eq. 2 it is not additive over a split of the update, and it ignores the sign of the effect
     assert orc.magnitude_metric([-tensors[0]], [1])[0] == 3.5
+
+
+# ------------------------------------------------------------------ attention core (non-trainable layer)
+def _attn_stack(d=8, heads=2, seq=5):
+    return [wl.Layer(6, d), wl.norm_layer(d), wl.Layer(d, 3 * d), wl.attention_layer(d, heads, seq),
+            wl.Layer(d, d, residual_src=1), wl.Layer(d, 4)]
+
+
+def test_finite_differences_through_the_attention_core():
+    _fd_check(_attn_stack(), M=15, seed=41, tol=5e-6)
+    _fd_check(wl.vit_blocks_full(1, 8, 12, heads=2, seq=4), M=12, seed=42, tol=5e-6)
+
+
+def test_attention_matches_the_library_scaled_dot_product_attention():
+    torch = pytest.importorskip("torch")
+    F = torch.nn.functional
+    d, H, S, B = 12, 3, 7, 4
+    layers = [wl.Layer(5, 3 * d), wl.attention_layer(d, H, S), wl.Layer(d, 6)]
+    w = wl.small_stack(layers, B * S, wl.DT_F32, 43, w_std=0.6, bias_std=0.2)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    grads = orc.backward_full(w.layers, w.W, saved, dY)
+    tW = [torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (w.W[0], w.W[2])]
+    tb = [torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (w.b[0], w.b[2])]
+    qkv = torch.tensor(w.x, dtype=torch.float64) @ tW[0] + tb[0]
+    q, k, v = (qkv[:, i * d:(i + 1) * d].reshape(B, S, H, d // H).transpose(1, 2) for i in range(3))
+    o = F.scaled_dot_product_attention(q, k, v).transpose(1, 2).reshape(B * S, d)
+    assert np.allclose(o.detach().numpy(), saved.a[2], rtol=1e-10, atol=1e-12)
+    loss = ((o @ tW[1] + tb[1] - torch.tensor(w.target, dtype=torch.float64)) ** 2).mean()
+    loss.backward()
+    for t, ref in ((0, tW[0]), (1, tb[0]), (4, tW[1]), (5, tb[1])):
+        assert np.allclose(grads[t], ref.grad.numpy(), rtol=1e-9, atol=1e-13), t
+    assert grads[2].size == 0 and grads[3].size == 0
+
+
+def test_attention_closed_forms():
+    # equal keys: the softmax is uniform and every query gets the mean of the values; one key far ahead:
+    # the output is that key's value; sequences do not mix
+    d, H, S = 4, 1, 3
+    ly = [wl.attention_layer(d, H, S)]
+    q = np.arange(24.0).reshape(6, 4) / 10
+    k = np.ones((6, 4))
+    v = np.array([[1.0, 0, 0, 0], [0, 1, 0, 0], [0, 0, 1, 0], [5, 5, 5, 5], [7, 7, 7, 7], [9, 9, 9, 9]])
+    o = orc.forward(ly, [np.zeros(0)], [np.zeros(0)], np.concatenate([q, k, v], axis=1)).a[-1]
+    assert np.allclose(o[:3], np.tile(v[:3].mean(0), (3, 1))) and np.allclose(o[3:], np.tile(v[3:].mean(0), (3, 1)))
+    k2 = k.copy(); k2[1] = 1000.0
+    q2 = np.ones((6, 4))
+    o = orc.forward(ly, [np.zeros(0)], [np.zeros(0)], np.concatenate([q2, k2, v], axis=1)).a[-1]
+    assert np.allclose(o[:3], np.tile(v[1], (3, 1))) and np.allclose(o[3:], np.tile(v[3:].mean(0), (3, 1)))

@@ -27,7 +27,9 @@ ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
 DT_F32, DT_BF16 = 0, 1
 # layer kinds: a dense layer (kernel, bias) or a layer normalisation over the feature axis, whose two
 # trainable tensors gamma and beta take the kernel and bias slots (Section 5.2: Gamma and Beta)
-KIND_DENSE, KIND_NORM = 0, 1
+KIND_DENSE, KIND_NORM, KIND_ATTENTION = 0, 1, 2
+# KIND_ATTENTION: the softmax attention core, a layer without trainable tensors (Section 5.3 / 5.4:
+# attention operations are non-trainable layers); its two tensor slots are empty
 
 
 @dataclass(frozen=True)
@@ -40,6 +42,8 @@ class Layer:
                                # a_{j+1} = output of layer j) to this layer's output
     kind: int = KIND_DENSE     # KIND_NORM: in_features == out_features, no act / fold / residual
     eps: float = 1e-5          # KIND_NORM: added to the variance
+    heads: int = 0             # KIND_ATTENTION: in_features = 3 * out_features = 3 * heads * head_dim,
+    seq: int = 0               #   rows come in sequences of `seq` consecutive tokens
 
     @property
     def out_width(self) -> int:
@@ -123,6 +127,27 @@ def norm_layer(d: int, eps: float = 1e-5) -> Layer:
     return Layer(d, d, kind=KIND_NORM, eps=eps)
 
 
+def attention_layer(d: int, heads: int, seq: int) -> Layer:
+    return Layer(3 * d, d, kind=KIND_ATTENTION, heads=heads, seq=seq)
+
+
+def vit_blocks_full(n_blocks: int, d: int, ffn: int, heads: int, seq: int) -> List[Layer]:
+    """The whole pre-norm transformer block: LN, QKV d->3d, softmax attention over sequences of `seq`
+    tokens with `heads` heads, out-proj d->d + block input, LN, fc1 with tanh-GELU, fc2 + the second
+    LN's input."""
+    layers: List[Layer] = []
+    for blk in range(n_blocks):
+        base = 7 * blk
+        layers.append(norm_layer(d))
+        layers.append(Layer(d, 3 * d))
+        layers.append(attention_layer(d, heads, seq))
+        layers.append(Layer(d, d, residual_src=base))
+        layers.append(norm_layer(d))
+        layers.append(Layer(d, ffn, act=ACT_GELU_TANH))
+        layers.append(Layer(ffn, d, residual_src=base + 4))
+    return layers
+
+
 def vit_blocks_prenorm(n_blocks: int, d: int, ffn: int) -> List[Layer]:
     """Pre-norm transformer block, attention core still the identity:
     LN, QKV d->3d (three slices summed), out-proj d->d + block input,
@@ -143,6 +168,9 @@ def vit_blocks_prenorm(n_blocks: int, d: int, ffn: int) -> List[Layer]:
 def _draw_params(rng, layers, dtype, w_std=None, he_init=False):
     W, b = [], []
     for ly in layers:
+        if ly.kind == KIND_ATTENTION:
+            W.append(np.zeros(0)); b.append(np.zeros(0))
+            continue
         if ly.kind == KIND_NORM:
             W.append(_store(1.0 + rng.normal(0.0, 0.1, size=ly.out_features), dtype))     # gamma
             b.append(_store(rng.normal(0.0, 0.1, size=ly.out_features), dtype))           # beta
@@ -197,6 +225,19 @@ def vit_b_prenorm(seed: int = 4, p_select: float = 0.3, n_blocks: int = 12, toke
     return _finish("vit_b_prenorm_bf16", layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
 
 
+def vit_b_full(seed: int = 5, p_select: float = 0.3, n_blocks: int = 12, batch: int = 64, seq: int = 197,
+               d: int = 768, ffn: int = 3072, heads: int = 12, params: bool = True) -> Workload:
+    """ViT-B/16 with its normalisation layers and attention core: `batch` sequences of `seq` tokens.
+    Bernoulli(p_select) over layers; the attention layers own no tensors and are never selected."""
+    rng = np.random.default_rng(seed)
+    layers = vit_blocks_full(n_blocks, d, ffn, heads, seq)
+    mask = bernoulli_weight_mask(rng, len(layers), p_select)
+    for l, ly in enumerate(layers):
+        if ly.kind == KIND_ATTENTION:
+            mask[2 * l] = mask[2 * l + 1] = 0
+    return _finish("vit_b_full_bf16", layers, batch * seq, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
+
+
 def vit_l(seed: int = 3, params: bool = True, n_blocks: int = 24, tokens: int = 32 * 197,
           d: int = 1024, ffn: int = 4096) -> Workload:
     """bf16 ViT-L-shaped linear-only stack; the mask starts all-selected and is
@@ -228,7 +269,8 @@ def small_stack(layers: List[Layer], M: int, dtype: int, seed: int, mask=None, w
         mask = (rng.random(2 * len(layers)) < 0.5).astype(np.uint8)
     wl = _finish("small", layers, M, dtype, lr, np.asarray(mask, dtype=np.uint8), rng, w_std=w_std)
     if bias_std > 0:
-        wl.b = [_store(rng.normal(0.0, bias_std, size=ly.out_features), dtype) for ly in layers]
+        wl.b = [np.zeros(0) if ly.kind == KIND_ATTENTION else _store(rng.normal(0.0, bias_std, size=ly.out_features), dtype)
+                for ly in layers]
     return wl
 
 
@@ -252,6 +294,9 @@ def draw_delta(w: Workload, seed: int, std: float = 1e-3):
     rng = np.random.default_rng(seed)
     out = []
     for ly in w.layers:
+        if ly.kind == KIND_ATTENTION:
+            out += [np.zeros(0), np.zeros(0)]
+            continue
         shape = (ly.out_features,) if ly.kind == KIND_NORM else (ly.in_features, ly.out_features)
         out.append(_store(rng.normal(0.0, std, size=shape), w.dtype))
         out.append(_store(rng.normal(0.0, std, size=ly.out_features), w.dtype))
