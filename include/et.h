@@ -22,6 +22,13 @@
  *       a_{l+1} = sum of the `fold` equal column slices of H_l  (+ a_j if residual_src = j)
  *   a_0 is the stack input; the width of a_{l+1} is out_features / fold.
  *
+ *   A layer of kind ET_LAYER_ATTENTION is the softmax attention core (the paper counts attention
+ *   operations among the non-trainable layers, Sections 5.3 and 5.4): a_l = [q | k | v], per sequence
+ *   and head  P = softmax(q k^T / 8),  a_{l+1} = [P v] with the heads side by side.  It has no
+ *   trainable tensors: its W and b pointers may be NULL, its two mask bits must be 0 and its two
+ *   slots in gradient / importance / state arrays are ignored.  Its backward (above the deepest
+ *   selected layer only) recomputes P from the saved per-row log-sum-exp.
+ *
  *   A layer of kind ET_LAYER_NORM is a layer normalisation over the features of each row
  *   (Section 5.2 treats normalisation layers as two trainable tensors, Gamma and Beta;
  *   Section 5.4 says LayerNorm behaves like batch normalisation in this respect):
@@ -73,7 +80,7 @@ typedef enum {
 
 typedef enum { ET_F32 = 0, ET_BF16 = 1 } et_dtype;
 typedef enum { ET_ACT_NONE = 0, ET_ACT_GELU_TANH = 1, ET_ACT_RELU = 2 } et_act;
-typedef enum { ET_LAYER_DENSE = 0, ET_LAYER_NORM = 1 } et_layer_kind;
+typedef enum { ET_LAYER_DENSE = 0, ET_LAYER_NORM = 1, ET_LAYER_ATTENTION = 2 } et_layer_kind;
 
 /* Cost-model reading for the selector (Section 2.2 / Eq. 7 versus the example after Eq. 3). */
 typedef enum {
@@ -98,6 +105,10 @@ typedef struct {
   int32_t kind;           /* et_layer_kind.  ET_LAYER_NORM: in_features == out_features (a multiple of 8,
                              at most 2048), act = ET_ACT_NONE, fold = 1, residual_src = -1 */
   float eps;              /* ET_LAYER_NORM: added to the variance, > 0 or 0 */
+  int32_t heads;          /* ET_LAYER_ATTENTION: in_features = 3 * out_features, out_features = 64 * heads;   */
+  int32_t seq_len;        /*   rows form sequences of seq_len (<= 208) consecutive rows, M a multiple of it;  */
+                          /*   ET_BF16 only; not the first or last layer; the layer below has no activation;   */
+                          /*   act = ET_ACT_NONE, fold = 1, residual_src = -1.  Both fields 0 for other kinds. */
 } et_layer_desc;
 
 /* What one et_backward_elastic call executed.  The four arrays are caller-owned host
@@ -281,7 +292,8 @@ et_status et_bias_grad_noalloc(const void* dZ, int64_t M, int32_t width, et_dtyp
  * non-trainable work below it, Section 5.3); bias tensor: t_dw = bias-gradient time,
  * t_dy = 0.  A normalisation layer is one black box (Section 5.2): the time of its whole
  * backward kernel (error gradient and d gamma together) plus its two finishing kernels goes
- * to t_dy of beta; t_dw of gamma and beta and t_dy of gamma are 0.
+ * to t_dy of beta; t_dw of gamma and beta and t_dy of gamma are 0.  An attention layer is a
+ * non-trainable layer (Section 5.3): its backward time is added to t_dy of the bias of the layer below.
  * t_fwd receives the forward time.  Milliseconds.  Synchronous.  Runs a forward
  * pass from x (writing y) and a full backward from dY first; weights are not changed. */
 et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, int32_t iters,
@@ -339,7 +351,8 @@ typedef enum {
   ET_K_BGRAD = 4,          /* bias gradient: column sums + finish (T2)                  */
   ET_K_OTHER = 5,          /* loss gradient, top-layer activation backward, importance finalise */
   ET_K_NORM = 6,           /* normalisation layers: forward, backward (error gradient + d gamma), gamma finish */
-  ET_K_CLASSES = 7
+  ET_K_ATTENTION = 7,      /* attention core: forward, backward */
+  ET_K_CLASSES = 8
 } et_kernel_class;
 
 /* on != 0: every kernel this stack launches from now on is bracketed by a pair of CUDA

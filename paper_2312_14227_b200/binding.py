@@ -30,10 +30,11 @@ ET_NOALLOC_SCRATCH_FLOATS = 1 << 20
 
 class et_layer_desc(C.Structure):
     _fields_ = [("in_features", C.c_int32), ("out_features", C.c_int32), ("act", C.c_int32),
-                ("fold", C.c_int32), ("residual_src", C.c_int32), ("kind", C.c_int32), ("eps", C.c_float)]
+                ("fold", C.c_int32), ("residual_src", C.c_int32), ("kind", C.c_int32), ("eps", C.c_float),
+                ("heads", C.c_int32), ("seq_len", C.c_int32)]
 
 
-ET_LAYER_DENSE, ET_LAYER_NORM = 0, 1
+ET_LAYER_DENSE, ET_LAYER_NORM, ET_LAYER_ATTENTION = 0, 1, 2
 
 
 class et_optimizer_config(C.Structure):
@@ -241,7 +242,8 @@ class Stack:
                 descs[i] = et_layer_desc(*ly)
             else:
                 descs[i] = et_layer_desc(ly.in_features, ly.out_features, ly.act, ly.fold, ly.residual_src,
-                                         getattr(ly, "kind", ET_LAYER_DENSE), getattr(ly, "eps", 0.0))
+                                         getattr(ly, "kind", ET_LAYER_DENSE), getattr(ly, "eps", 0.0),
+                                         getattr(ly, "heads", 0), getattr(ly, "seq", 0))
         self.out_width = (descs[self.L - 1].out_features // max(descs[self.L - 1].fold, 1)) if self.L else 0
         h = C.c_void_p()
         _check(_lib.et_stack_create(descs, self.L, self.M, dtype, C.byref(h)), "et_stack_create")
@@ -366,7 +368,7 @@ def et_profile_costs(s: Stack, x, y, dY, iters: int = 20, stream=None):
     return t_dw, t_dy, t_fwd.value
 
 
-KERNEL_CLASSES = ("forward", "dgrad", "wgrad", "wgrad_reduce", "bgrad", "other", "norm")
+KERNEL_CLASSES = ("forward", "dgrad", "wgrad", "wgrad_reduce", "bgrad", "other", "norm", "attention")
 
 
 def et_timing_enable(s: Stack, on: bool):

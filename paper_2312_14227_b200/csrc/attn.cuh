@@ -1,0 +1,287 @@
+// Softmax attention core as a member of the stack: a layer without trainable tensors (the paper
+// counts attention operations among the non-trainable layers, Sections 5.3 and 5.4).  Input rows
+// are [q | k | v] (3 * heads * 64 columns), grouped in sequences of S consecutive rows; output
+// rows are the heads' P v side by side.
+//
+//   forward   P = softmax_j( q_i . k_j / 8 ),  o_i = sum_j P_ij v_j ;  keeps logsumexp per (head, row)
+//   backward  dV = P^T dO ;  dP = dO V^T ;  D_i = dO_i . o_i ;  dS = P * (dP - D_i) / 8 ;
+//             dQ = dS K ;  dK = dS^T Q          (P is recomputed from q, k and the saved logsumexp)
+//
+// One CTA per (sequence, head); K and V of the head stay in shared memory, queries go through in
+// blocks of 64 rows.  The five small GEMMs per block (64 x S x 64 and S x 64 x 64) run on the tensor
+// cores through the warp-level matrix fragments (16 x 16 x 16, bf16 in, fp32 accumulate); with S
+// around 200 and a head width of 64 the tiles are too small for a TMEM accumulator pipeline to pay.
+// Limits: head width 64, S <= 208, bf16 storage.
+#pragma once
+
+#include <mma.h>
+
+#include "common.cuh"
+
+namespace et {
+namespace attn {
+
+constexpr int DH = 64;           // head width
+constexpr int S_MAX = 208;       // longest sequence (padded to a multiple of 16)
+constexpr int RB = 64;           // query rows per pass
+constexpr int THREADS = 256;
+constexpr int WARPS = THREADS / 32;
+constexpr int LDK = DH + 8;      // row stride (elements) of the 64-wide bf16 tiles: breaks bank conflicts
+constexpr int MAX_OWN = 7;       // (S_MAX / 16) * (DH / 16) = 52 output tiles of dK (or dV) over 8 warps
+constexpr float SCALE = 0.125f;  // 1 / sqrt(DH)
+
+__host__ __device__ inline int pad16(int s) { return (s + 15) & ~15; }
+// row stride (floats) of the fp32 score buffer; it also stages 64-column results, so never below 68
+__host__ __device__ inline int score_ld(int SP) { return SP + 4 > DH + 4 ? SP + 4 : DH + 4; }
+inline size_t forward_smem_bytes(int S) {
+  const int SP = pad16(S);
+  return (size_t)(2 * SP + RB) * LDK * 2 + (size_t)RB * score_ld(SP) * 4 + (size_t)RB * (SP + 8) * 2;
+}
+inline size_t backward_smem_bytes(int S) {
+  const int SP = pad16(S);
+  return (size_t)(2 * SP + 2 * RB) * LDK * 2 + (size_t)RB * score_ld(SP) * 4 + (size_t)2 * RB * (SP + 8) * 2;
+}
+
+using FragA = nvcuda::wmma::fragment<nvcuda::wmma::matrix_a, 16, 16, 16, bf16, nvcuda::wmma::row_major>;
+using FragAT = nvcuda::wmma::fragment<nvcuda::wmma::matrix_a, 16, 16, 16, bf16, nvcuda::wmma::col_major>;
+using FragB = nvcuda::wmma::fragment<nvcuda::wmma::matrix_b, 16, 16, 16, bf16, nvcuda::wmma::row_major>;
+using FragBT = nvcuda::wmma::fragment<nvcuda::wmma::matrix_b, 16, 16, 16, bf16, nvcuda::wmma::col_major>;
+using FragC = nvcuda::wmma::fragment<nvcuda::wmma::accumulator, 16, 16, 16, float>;
+
+// rows [row0, row0 + nrows) of one head's 64 columns -> tile[r][LDK]; rows at or past S read as zeros
+__device__ __forceinline__ void load_tile(bf16* tile, const bf16* src, size_t ld, int row0, int nrows, int S) {
+  for (int i = threadIdx.x; i < nrows * 8; i += THREADS) {
+    const int r = i >> 3, ch = i & 7;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row0 + r < S) v = *reinterpret_cast<const uint4*>(src + (size_t)(row0 + r) * ld + ch * 8);
+    *reinterpret_cast<uint4*>(tile + r * LDK + ch * 8) = v;
+  }
+}
+// 16 consecutive floats of a staged fp32 tile -> 16 bf16 in global memory
+__device__ __forceinline__ void store16(bf16* dst, const float* src) {
+  uint4 a, b;
+  a.x = pack_bf16x2(src[0], src[1]);   a.y = pack_bf16x2(src[2], src[3]);
+  a.z = pack_bf16x2(src[4], src[5]);   a.w = pack_bf16x2(src[6], src[7]);
+  b.x = pack_bf16x2(src[8], src[9]);   b.y = pack_bf16x2(src[10], src[11]);
+  b.z = pack_bf16x2(src[12], src[13]); b.w = pack_bf16x2(src[14], src[15]);
+  reinterpret_cast<uint4*>(dst)[0] = a;
+  reinterpret_cast<uint4*>(dst)[1] = b;
+}
+
+// Sf[64][ldsf] = Q_blk K^T (fp32), all warps
+__device__ __forceinline__ void scores(const bf16* Qs, const bf16* Ks, float* Sf, int ntn, int ldsf, int warp) {
+  for (int t = warp; t < (RB / 16) * ntn; t += WARPS) {
+    const int mi = t / ntn, nj = t - mi * ntn;
+    FragC acc;
+    nvcuda::wmma::fill_fragment(acc, 0.0f);
+#pragma unroll
+    for (int kk = 0; kk < DH / 16; ++kk) {
+      FragA a;
+      FragBT b;
+      nvcuda::wmma::load_matrix_sync(a, Qs + mi * 16 * LDK + kk * 16, LDK);
+      nvcuda::wmma::load_matrix_sync(b, Ks + nj * 16 * LDK + kk * 16, LDK);     // B[k][n] = K[n][k]
+      nvcuda::wmma::mma_sync(acc, a, b, acc);
+    }
+    nvcuda::wmma::store_matrix_sync(Sf + mi * 16 * ldsf + nj * 16, acc, ldsf, nvcuda::wmma::mem_row_major);
+  }
+}
+// Of[64][ldsf] (columns 0..63) = A[64][SP] * Bm[SP][64], A bf16 with stride lda, all warps (2 tiles each)
+__device__ __forceinline__ void rows_times_head(const bf16* A, int lda, const bf16* Bm, float* Of, int ntn, int ldsf,
+                                                int warp) {
+  for (int t = warp; t < (RB / 16) * (DH / 16); t += WARPS) {
+    const int mi = t >> 2, nj = t & 3;
+    FragC acc;
+    nvcuda::wmma::fill_fragment(acc, 0.0f);
+    for (int kk = 0; kk < ntn; ++kk) {
+      FragA a;
+      FragB b;
+      nvcuda::wmma::load_matrix_sync(a, A + mi * 16 * lda + kk * 16, lda);
+      nvcuda::wmma::load_matrix_sync(b, Bm + kk * 16 * LDK + nj * 16, LDK);
+      nvcuda::wmma::mma_sync(acc, a, b, acc);
+    }
+    nvcuda::wmma::store_matrix_sync(Of + mi * 16 * ldsf + nj * 16, acc, ldsf, nvcuda::wmma::mem_row_major);
+  }
+}
+
+// grid = sequences * heads.  qkv: [M][3d]; out: [M][d]; lse: [sequences * heads][S].
+static __global__ void __launch_bounds__(THREADS)
+attn_forward_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __restrict__ lse, int S, int H, int d) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int SP = pad16(S), ntn = SP / 16, ldsf = score_ld(SP), ldp = SP + 8;
+  bf16* Ks = reinterpret_cast<bf16*>(smem);
+  bf16* Vs = Ks + SP * LDK;
+  bf16* Qs = Vs + SP * LDK;
+  float* Sf = reinterpret_cast<float*>(Qs + RB * LDK);
+  bf16* Pb = reinterpret_cast<bf16*>(Sf + RB * ldsf);
+  const int b = blockIdx.x / H, h = blockIdx.x - b * H;
+  const int warp = threadIdx.x >> 5;
+  const size_t ld = (size_t)3 * d;
+  const bf16* base = qkv + (size_t)b * S * ld + h * DH;
+  load_tile(Ks, base + d, ld, 0, SP, S);
+  load_tile(Vs, base + 2 * d, ld, 0, SP, S);
+  for (int rb0 = 0; rb0 < S; rb0 += RB) {
+    load_tile(Qs, base, ld, rb0, RB, S);
+    __syncthreads();
+    scores(Qs, Ks, Sf, ntn, ldsf, warp);
+    __syncthreads();
+    {   // softmax of row r by 4 neighbouring lanes
+      const int r = threadIdx.x >> 2, sub = threadIdx.x & 3;
+      const bool valid = rb0 + r < S;
+      float* row = Sf + r * ldsf;
+      float m = -INFINITY;
+      for (int c = sub; c < S; c += 4) m = fmaxf(m, row[c]);
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+      float sum = 0.0f;
+      for (int c = sub; c < S; c += 4) {
+        const float e = __expf((row[c] - m) * SCALE);
+        row[c] = e;
+        sum += e;
+      }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      const float inv = 1.0f / sum;
+      for (int c = sub; c < SP; c += 4) Pb[r * ldp + c] = __float2bfloat16_rn((valid && c < S) ? row[c] * inv : 0.0f);
+      if (valid && sub == 0) lse[(size_t)blockIdx.x * S + rb0 + r] = m * SCALE + __logf(sum);
+    }
+    __syncthreads();
+    rows_times_head(Pb, ldp, Vs, Sf, ntn, ldsf, warp);
+    __syncthreads();
+    {
+      const int r = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * 16;
+      if (rb0 + r < S) store16(out + ((size_t)b * S + rb0 + r) * d + h * DH + c0, Sf + r * ldsf + c0);
+    }
+    __syncthreads();
+  }
+}
+
+// dqkv: [M][3d] gradient of the layer's input; every element of this head's columns is written.
+static __global__ void __launch_bounds__(THREADS)
+attn_backward_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out, const bf16* __restrict__ dout,
+                     const float* __restrict__ lse, bf16* __restrict__ dqkv, int S, int H, int d) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ float Dsm[RB];
+  const int SP = pad16(S), ntn = SP / 16, ldsf = score_ld(SP), ldp = SP + 8;
+  bf16* Ks = reinterpret_cast<bf16*>(smem);
+  bf16* Vs = Ks + SP * LDK;
+  bf16* Qs = Vs + SP * LDK;
+  bf16* dOs = Qs + RB * LDK;
+  float* Sf = reinterpret_cast<float*>(dOs + RB * LDK);
+  bf16* Pb = reinterpret_cast<bf16*>(Sf + RB * ldsf);
+  bf16* dSb = Pb + RB * ldp;
+  const int b = blockIdx.x / H, h = blockIdx.x - b * H;
+  const int warp = threadIdx.x >> 5;
+  const size_t ld = (size_t)3 * d;
+  const bf16* base = qkv + (size_t)b * S * ld + h * DH;
+  bf16* gbase = dqkv + (size_t)b * S * ld + h * DH;
+  const bf16* obase = out + (size_t)b * S * d + h * DH;
+  const bf16* dobase = dout + (size_t)b * S * d + h * DH;
+  load_tile(Ks, base + d, ld, 0, SP, S);
+  load_tile(Vs, base + 2 * d, ld, 0, SP, S);
+  const int own_tiles = ntn * (DH / 16);            // output tiles of dK (and of dV): [SP][64]
+  FragC accK[MAX_OWN], accV[MAX_OWN];
+#pragma unroll
+  for (int i = 0; i < MAX_OWN; ++i) {
+    nvcuda::wmma::fill_fragment(accK[i], 0.0f);
+    nvcuda::wmma::fill_fragment(accV[i], 0.0f);
+  }
+  for (int rb0 = 0; rb0 < S; rb0 += RB) {
+    load_tile(Qs, base, ld, rb0, RB, S);
+    load_tile(dOs, dobase, (size_t)d, rb0, RB, S);
+    __syncthreads();
+    scores(Qs, Ks, Sf, ntn, ldsf, warp);
+    {   // D_r = dO_r . o_r
+      const int r = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * 16;
+      float s = 0.0f;
+      if (rb0 + r < S) {
+        const bf16* o = obase + (size_t)(rb0 + r) * d + c0;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) s = fmaf(__bfloat162float(dOs[r * LDK + c0 + c]), __bfloat162float(o[c]), s);
+      }
+      s += __shfl_xor_sync(0xffffffffu, s, 1);
+      s += __shfl_xor_sync(0xffffffffu, s, 2);
+      if ((threadIdx.x & 3) == 0) Dsm[r] = s;
+    }
+    __syncthreads();
+    {   // P = exp(s / 8 - logsumexp), zero outside the sequence
+      const int r = threadIdx.x >> 2, sub = threadIdx.x & 3;
+      const bool valid = rb0 + r < S;
+      const float l = valid ? lse[(size_t)blockIdx.x * S + rb0 + r] : 0.0f;
+      const float* row = Sf + r * ldsf;
+      for (int c = sub; c < SP; c += 4)
+        Pb[r * ldp + c] = __float2bfloat16_rn((valid && c < S) ? __expf(row[c] * SCALE - l) : 0.0f);
+    }
+    __syncthreads();
+    // dP = dO V^T -> Sf
+    for (int t = warp; t < (RB / 16) * ntn; t += WARPS) {
+      const int mi = t / ntn, nj = t - mi * ntn;
+      FragC acc;
+      nvcuda::wmma::fill_fragment(acc, 0.0f);
+#pragma unroll
+      for (int kk = 0; kk < DH / 16; ++kk) {
+        FragA a;
+        FragBT bt;
+        nvcuda::wmma::load_matrix_sync(a, dOs + mi * 16 * LDK + kk * 16, LDK);
+        nvcuda::wmma::load_matrix_sync(bt, Vs + nj * 16 * LDK + kk * 16, LDK);   // B[k][n] = V[n][k]
+        nvcuda::wmma::mma_sync(acc, a, bt, acc);
+      }
+      nvcuda::wmma::store_matrix_sync(Sf + mi * 16 * ldsf + nj * 16, acc, ldsf, nvcuda::wmma::mem_row_major);
+    }
+    __syncthreads();
+    {   // dS = P * (dP - D) / 8
+      const int r = threadIdx.x >> 2, sub = threadIdx.x & 3;
+      const float Dr = Dsm[r];
+      const float* row = Sf + r * ldsf;
+      for (int c = sub; c < SP; c += 4)
+        dSb[r * ldp + c] = __float2bfloat16_rn(__bfloat162float(Pb[r * ldp + c]) * (row[c] - Dr) * SCALE);
+    }
+    __syncthreads();
+    // dQ_blk = dS K -> Sf (columns 0..63)
+    rows_times_head(dSb, ldp, Ks, Sf, ntn, ldsf, warp);
+    // dV += P^T dO ; dK += dS^T Q   (contraction over the 64 rows of this block)
+#pragma unroll
+    for (int i = 0; i < MAX_OWN; ++i) {
+      const int t = warp + WARPS * i;
+      if (t < own_tiles) {
+        const int mj = t >> 2, nj = t & 3;
+#pragma unroll
+        for (int kk = 0; kk < RB / 16; ++kk) {
+          FragAT pt, st;
+          FragB bo, bq;
+          nvcuda::wmma::load_matrix_sync(pt, Pb + kk * 16 * ldp + mj * 16, ldp);     // A[m][k] = P[k][m]
+          nvcuda::wmma::load_matrix_sync(bo, dOs + kk * 16 * LDK + nj * 16, LDK);
+          nvcuda::wmma::mma_sync(accV[i], pt, bo, accV[i]);
+          nvcuda::wmma::load_matrix_sync(st, dSb + kk * 16 * ldp + mj * 16, ldp);
+          nvcuda::wmma::load_matrix_sync(bq, Qs + kk * 16 * LDK + nj * 16, LDK);
+          nvcuda::wmma::mma_sync(accK[i], st, bq, accK[i]);
+        }
+      }
+    }
+    __syncthreads();
+    {
+      const int r = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * 16;
+      if (rb0 + r < S) store16(gbase + (size_t)(rb0 + r) * ld + c0, Sf + r * ldsf + c0);
+    }
+    __syncthreads();
+  }
+  // dK, then dV: accumulators -> fp32 staging [SP][64] (it fits the score buffer) -> bf16 rows
+  float* stage = Sf;
+  for (int which = 0; which < 2; ++which) {
+#pragma unroll
+    for (int i = 0; i < MAX_OWN; ++i) {
+      const int t = warp + WARPS * i;
+      if (t < own_tiles)
+        nvcuda::wmma::store_matrix_sync(stage + (t >> 2) * 16 * DH + (t & 3) * 16, which == 0 ? accK[i] : accV[i], DH,
+                                        nvcuda::wmma::mem_row_major);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < S * 4; i += THREADS) {
+      const int r = i >> 2, c0 = (i & 3) * 16;
+      store16(gbase + (size_t)r * ld + (which + 1) * d + c0, stage + r * DH + c0);
+    }
+    __syncthreads();
+  }
+}
+
+}  // namespace attn
+}  // namespace et

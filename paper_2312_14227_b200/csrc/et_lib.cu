@@ -18,6 +18,7 @@
 #include "gemm_tc.cuh"
 #include "kernels.cuh"
 #include "norm.cuh"
+#include "attn.cuh"
 
 namespace {
 
@@ -130,6 +131,8 @@ struct LayerRT {
   size_t off_stats = 0;     // norm: (mean, rstd) per row
   size_t off_gpart = 0;     // norm: per-block partial column sums of g * xhat
   int norm_blocks = 0;      // norm: blocks of the backward kernel = rows of off_gpart
+  int heads = 0, seq = 0;   // attention: K = 3N, N = 64 * heads, rows in sequences of `seq`
+  size_t off_lse = 0;       // attention: log-sum-exp per (sequence, head, row)
   int consumer = -1;        // layer whose residual reads a_l (its output gradient joins G_l), or -1
   void* W = nullptr;
   void* b = nullptr;
@@ -147,7 +150,8 @@ struct LayerRT {
   int bn_fwd = 256, bn_dgrad = 256, bn_wgrad = 256;   // tile widths chosen per GEMM
   bool pair_fwd = false, pair_dgrad = false, pair_wgrad = false;   // CTA-pair (cta_group::2) tiles
   int imp_count_w = 0, imp_count_b = 0;
-  size_t w_count() const { return kind == ET_LAYER_NORM ? (size_t)N : (size_t)K * N; }   // elements of tensor 2l
+  bool trainable() const { return kind != ET_LAYER_ATTENTION; }
+  size_t w_count() const { return kind == ET_LAYER_ATTENTION ? 0 : kind == ET_LAYER_NORM ? (size_t)N : (size_t)K * N; }   // elements of tensor 2l
   // bf16 stacks: one TMA descriptor per tensor (the caller's x, y and dY get theirs per call)
   TMaps map_W, map_aout, map_Gout, map_Z, map_dZ;
   CUtensorMap map_Wd;       // W as the K-major B of the dgrad GEMM: one box = the CTA's whole B tile
@@ -599,6 +603,54 @@ et_status run_norm_backward(et_stack* s, int l, const void* dY, bool want_dx, bo
   return after_launch();
 }
 
+// ---- attention core --------------------------------------------------------------------------
+// Dynamic shared memory above 48 KB has to be allowed per kernel and device.
+et_status attn_allow_forward(size_t bytes) {
+  static size_t allowed[64] = {};
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
+  if (bytes > allowed[dev]) {
+    CU_TRY(cudaFuncSetAttribute(et::attn::attn_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    allowed[dev] = bytes;
+  }
+  return ET_OK;
+}
+et_status attn_allow_backward(size_t bytes) {
+  static size_t allowed[64] = {};
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
+  if (bytes > allowed[dev]) {
+    CU_TRY(cudaFuncSetAttribute(et::attn::attn_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    allowed[dev] = bytes;
+  }
+  return ET_OK;
+}
+
+et_status run_attn_forward(et_stack* s, int l, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_ATTENTION, st);
+  const LayerRT& L = s->ly[l];
+  const size_t smem = et::attn::forward_smem_bytes(L.seq);
+  ET_TRY(attn_allow_forward(smem));
+  const int grid = (int)(s->M / L.seq) * L.heads;
+  et::attn::attn_forward_kernel<<<grid, et::attn::THREADS, smem, st>>>(
+      act_in<bf16>(s, l), (bf16*)s->at(L.off_a_out), (float*)s->at(L.off_lse), L.seq, L.heads, L.N);
+  return after_launch();
+}
+// G_l (gradient of [q | k | v]) from G_{l+1}; l >= 1 and the layer below has no activation, so G_l is its dZ.
+et_status run_attn_backward(et_stack* s, int l, const void* dY, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_ATTENTION, st);
+  const LayerRT& L = s->ly[l];
+  const size_t smem = et::attn::backward_smem_bytes(L.seq);
+  ET_TRY(attn_allow_backward(smem));
+  const int grid = (int)(s->M / L.seq) * L.heads;
+  et::attn::attn_backward_kernel<<<grid, et::attn::THREADS, smem, st>>>(
+      act_in<bf16>(s, l), (const bf16*)s->at(L.off_a_out), grad_act<bf16>(s, l + 1, dY), (const float*)s->at(L.off_lse),
+      (bf16*)s->at(s->ly[l - 1].off_G_out), L.seq, L.heads, L.N);
+  return after_launch();
+}
+
 // dW_l = a_l^T dZ_l as split partials, then the reducer with grad / importance / SGD.
 template <typename T>
 et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
@@ -677,6 +729,8 @@ et::MaskBits mask_bits(const uint8_t* mask, int n) {
 et_status check_ready(const et_stack* s, const uint8_t* mask, int n_tensors) {
   if (s == nullptr || mask == nullptr) return ET_ERR_INVALID_ARG;
   if (n_tensors != 2 * s->L) return ET_ERR_INVALID_ARG;
+  for (int t = 0; t < n_tensors; ++t)
+    if (mask[t] && !s->ly[t / 2].trainable()) return ET_ERR_INVALID_ARG;   // nothing there to select
   if (!s->bound) return ET_ERR_STATE;
   return ET_OK;
 }
@@ -775,7 +829,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
     for (int l = L - 1; l >= d; --l) {
       const LayerRT& Y = s->ly[l];
       const bool norm = Y.kind == ET_LAYER_NORM;
-      const double gemm = norm ? 0.0 : 2.0 * (double)s->M * Y.K * Y.N;
+      const double gemm = Y.kind != ET_LAYER_DENSE ? 0.0 : 2.0 * (double)s->M * Y.K * Y.N;
       if (mask[2 * l + 1]) {
         // On the tensor-core path the column partials of dZ_l were left by dgrad(l+1) in this
         // layer's own buffer; finishing them need not sit on the chain's critical path.
@@ -788,6 +842,15 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         if (two && bs == st) CU_TRY(cudaStreamWaitEvent(st, s->chain_ev[l + 1], 0));
         ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
                                   delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, bs, fused));
+      }
+      if (Y.kind == ET_LAYER_ATTENTION) {
+        // a non-trainable layer: only passes the error gradient on, above the deepest selected layer
+        if (l > d) {
+          ET_TRY(run_attn_backward(s, l, dY, cs));
+          ++launches;
+          if (two) CU_TRY(cudaEventRecord(s->chain_ev[l], cs));
+        }
+        continue;
       }
       if (norm) {
         // one kernel passes the error gradient on (above the deepest selected layer) and leaves the
@@ -861,6 +924,7 @@ et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
   s->x = x;
   for (int l = 0; l < s->L; ++l) {
     if (s->ly[l].kind == ET_LAYER_NORM) ET_TRY(run_norm_forward<T>(s, l, y, st));
+    else if (s->ly[l].kind == ET_LAYER_ATTENTION) ET_TRY(run_attn_forward(s, l, st));
     else ET_TRY(run_forward_layer<T>(s, l, y, st));
   }
   s->forwarded = true;
@@ -904,8 +968,19 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (d.fold > 1 && d.act != ET_ACT_NONE) { err = ET_ERR_UNSUPPORTED; break; }
     y.K = d.in_features; y.N = d.out_features; y.fold = d.fold; y.Nw = d.out_features / d.fold;
     y.act = d.act; y.residual_src = d.residual_src;
-    if (d.kind != ET_LAYER_DENSE && d.kind != ET_LAYER_NORM) { err = ET_ERR_INVALID_ARG; break; }
+    if (d.kind != ET_LAYER_DENSE && d.kind != ET_LAYER_NORM && d.kind != ET_LAYER_ATTENTION) { err = ET_ERR_INVALID_ARG; break; }
     y.kind = d.kind; y.eps = d.eps;
+    if (y.kind == ET_LAYER_ATTENTION) {
+      y.heads = d.heads; y.seq = d.seq_len;
+      if (y.fold != 1 || y.act != ET_ACT_NONE || y.residual_src != -1 || y.heads < 1 || y.seq < 1 || y.K != 3 * y.N) {
+        err = ET_ERR_INVALID_ARG; break;
+      }
+      if (M % y.seq != 0) { err = ET_ERR_SHAPE; break; }
+      if (dtype != ET_BF16 || y.N != et::attn::DH * y.heads || y.seq > et::attn::S_MAX || l == 0 || l == L - 1 ||
+          s->ly[l - 1].act != ET_ACT_NONE) {
+        err = ET_ERR_UNSUPPORTED; break;
+      }
+    }
     if (y.kind == ET_LAYER_NORM) {
       if (y.K != y.N || y.fold != 1 || y.act != ET_ACT_NONE || y.residual_src != -1 || !(y.eps >= 0.f)) {
         err = ET_ERR_INVALID_ARG; break;
@@ -928,6 +1003,8 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
       if (y.fold > 1 && y.Nw % 256) { err = ET_ERR_UNSUPPORTED; break; }
     }
   }
+  for (int l = 0; l < L && err == ET_OK; ++l)
+    if (s->ly[l].kind == ET_LAYER_ATTENTION && s->ly[l].consumer >= 0) err = ET_ERR_UNSUPPORTED;   // [q|k|v] feeds nothing else
   if (err != ET_OK) { delete s; return err; }
 
   // ---- workspace layout
@@ -943,7 +1020,9 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     const size_t act_bytes = (size_t)M * y.Nw * s->elt;
     if (l < L - 1) { y.off_a_out = take(act_bytes); y.off_G_out = take(act_bytes); }
     if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
-    if (y.kind == ET_LAYER_NORM) {
+    if (y.kind == ET_LAYER_ATTENTION) {
+      y.off_lse = take((size_t)M * y.heads * sizeof(float));
+    } else if (y.kind == ET_LAYER_NORM) {
       y.off_stats = take((size_t)M * sizeof(float2));
       y.norm_blocks = std::min(ceil_div(M, et::kNormWarps), s->sms * 8);
       y.off_gpart = take((size_t)y.norm_blocks * y.N * sizeof(float));
@@ -965,6 +1044,12 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
           if (fs > 0) y.split = std::min(fs, ceil_div(M, et::tc::BK));
         }
       }
+    }
+    if (y.kind == ET_LAYER_ATTENTION) {                    // no tensors: no partials, no importance slots
+      y.imp_count_w = y.imp_count_b = 0;
+      s->imp_offs[2 * l] = s->imp_offs[2 * l + 1] = imp_total;
+      s->imp_counts[2 * l] = s->imp_counts[2 * l + 1] = 0;
+      continue;
     }
     max_partial = std::max(max_partial, y.kind == ET_LAYER_NORM ? (size_t)y.N * sizeof(float)
                                                                 : (size_t)y.split * y.K * y.N * sizeof(float));
@@ -1007,8 +1092,10 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
                         void* stream) {
   if (s == nullptr || W == nullptr || b == nullptr || workspace == nullptr) return ET_ERR_INVALID_ARG;
   if (workspace_bytes < s->ws_bytes || ((uintptr_t)workspace & 255) != 0) return ET_ERR_WORKSPACE;
-  for (int l = 0; l < s->L; ++l)
+  for (int l = 0; l < s->L; ++l) {
+    if (!s->ly[l].trainable()) continue;                  // no tensors: its pointers are ignored
     if (W[l] == nullptr || b[l] == nullptr || ((uintptr_t)W[l] & 15) || ((uintptr_t)b[l] & 15)) return ET_ERR_INVALID_ARG;
+  }
   cudaStream_t st = (cudaStream_t)stream;
   s->bound = false;
   s->ws = (char*)workspace;
@@ -1018,7 +1105,7 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   if (s->dtype == ET_BF16) {
     for (int l = 0; l < s->L; ++l) {
       LayerRT& y = s->ly[l];
-      if (y.kind != ET_LAYER_NORM) {
+      if (y.kind == ET_LAYER_DENSE) {
         ET_TRY(make_tmaps(&y.map_W, y.W, y.N, y.K));
         ET_TRY(make_map(&y.map_Wd, y.W, y.N, y.K, y.pair_dgrad ? y.bn_dgrad / 2 : y.bn_dgrad));
       }
@@ -1051,7 +1138,8 @@ et_status et_stack_bind_master(et_stack* s, float* const* W32, float* const* b32
   if ((W32 == nullptr) != (b32 == nullptr)) return ET_ERR_INVALID_ARG;
   if (W32 != nullptr)
     for (int l = 0; l < s->L; ++l)
-      if (W32[l] == nullptr || b32[l] == nullptr || ((uintptr_t)W32[l] & 15) || ((uintptr_t)b32[l] & 15))
+      if (s->ly[l].trainable() &&
+          (W32[l] == nullptr || b32[l] == nullptr || ((uintptr_t)W32[l] & 15) || ((uintptr_t)b32[l] & 15)))
         return ET_ERR_INVALID_ARG;
   for (int l = 0; l < s->L; ++l) {
     s->ly[l].W32 = W32 ? W32[l] : nullptr;
@@ -1238,6 +1326,7 @@ et_status et_stack_set_optimizer(et_stack* s, const et_optimizer_config* cfg, fl
     return ET_ERR_INVALID_ARG;
   const int n = 2 * s->L;
   for (int t = 0; t < n; ++t) {
+    if (!s->ly[t / 2].trainable()) continue;
     if (c.kind != ET_OPT_SGD && (state1[t] == nullptr || ((uintptr_t)state1[t] & 15))) return ET_ERR_INVALID_ARG;
     if (c.kind == ET_OPT_ADAM && (state2[t] == nullptr || ((uintptr_t)state2[t] & 15))) return ET_ERR_INVALID_ARG;
   }
@@ -1292,9 +1381,25 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
     std::vector<uint8_t> ones(2 * L, 1);
     ET_TRY(et_backward_elastic(s, dY, ones.data(), 2 * L, nullptr, nullptr, nullptr, 0, 0.f, nullptr, stream));
     float* scratch_grad = (float*)s->at(s->off_partial);      // in-place: each element is read before it is written
+    double pending_nontrainable = 0.0;
     for (int l = L - 1; l >= 0; --l) {
       int dummy = 0;
       t_dy[2 * l] = 0.0; t_dy[2 * l + 1] = 0.0;
+      if (s->ly[l].kind == ET_LAYER_ATTENTION) {
+        // Section 5.3: a non-trainable layer's backward time joins t_dy of the closest tensor of the
+        // trainable layer below it (that layer's bias)
+        t_dw[2 * l] = 0.0; t_dw[2 * l + 1] = 0.0;
+        double t_attn = 0.0;
+        ET_TRY(timed([&]() { return run_attn_backward(s, l, dY, st); }, &t_attn));
+        pending_nontrainable += t_attn;
+        continue;
+      }
+      const double carried = pending_nontrainable;
+      pending_nontrainable = 0.0;
+      struct AddCarried {
+        double* slot; double v;
+        ~AddCarried() { *slot += v; }
+      } add_carried{&t_dy[2 * l + 1], carried};
       if (s->ly[l].kind == ET_LAYER_NORM) {
         // Section 5.2: the layer is one black box whose whole backward time belongs to t_dy of beta
         t_dw[2 * l] = 0.0; t_dw[2 * l + 1] = 0.0;
