@@ -463,7 +463,7 @@ def run_side(args):
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
-    w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "schedule": wl.vit_l}[args.workload]()
+    w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "full": wl.vit_b_full, "schedule": wl.vit_l}[args.workload]()
     tdt = torch.bfloat16
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
     stack = et.et_stack_create(w.layers, w.M, w.dtype)
@@ -476,8 +476,12 @@ def run_side(args):
     et.et_forward_stack(stack, x, y)
     et.et_loss_mse_grad(stack, y, target, dY, None)
     torch.cuda.synchronize()
-    if args.workload in ("resnet", "prenorm"):
+    if args.workload in ("resnet", "prenorm", "full"):
         rep = et.Report(w.L)
+        all_trainable = np.ones(2 * w.L, dtype=np.uint8)
+        for l, ly in enumerate(w.layers):
+            if ly.kind == wl.KIND_ATTENTION:             # a layer without tensors cannot be selected
+                all_trainable[2 * l] = all_trainable[2 * l + 1] = 0
         delta = [to_dev(d) for d in wl.draw_delta(w, 5)]
         imp = torch.zeros(2 * w.L, dtype=torch.float32, device=dev)
 
@@ -494,7 +498,7 @@ def run_side(args):
             return e0.elapsed_time(e1) / args.steps, rep.flops_executed, rep.launches
 
         ms, fl, n = timed(w.mask)
-        fms, ffl, fn = timed(np.ones(2 * w.L, dtype=np.uint8))
+        fms, ffl, fn = timed(all_trainable)
 
         # the same elastic step replayed from a CUDA graph (the caller captures the library call)
         def graph_ms(mask):
@@ -518,11 +522,35 @@ def run_side(args):
             return e0.elapsed_time(e1) / args.steps
 
         try:
-            gms, gfms = graph_ms(w.mask), graph_ms(np.ones(2 * w.L, dtype=np.uint8))
+            gms, gfms = graph_ms(w.mask), graph_ms(all_trainable)
         except Exception as exc:                      # report, do not hide
             gms = gfms = None
             print("graph capture failed:", exc, file=sys.stderr)
         extra = {}
+        if args.workload == "full":
+            # the attention kernels alone, over full-backprop steps: 4 S^2 64 flops per (sequence, head)
+            # forward, 2.5 times that backward (five GEMMs, one of them the recomputed scores)
+            ones = all_trainable
+            et.et_timing_enable(stack, True)
+            for _ in range(5):
+                et.et_forward_stack(stack, x, y)
+                et.et_backward_elastic(stack, dY, ones, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep)
+            t = et.et_timing_read(stack)
+            et.et_timing_enable(stack, False)
+            att = [ly for ly in w.layers if ly.kind == wl.KIND_ATTENTION]
+            fwd_flops = sum(4.0 * (w.M // ly.seq) * ly.heads * ly.seq * ly.seq * 64 for ly in att)
+            att_ms = t["attention"][0] / 5
+            extra = {"attention_ms_per_forward_plus_backward": att_ms, "attention_launches": t["attention"][1] / 5,
+                     "attention_tflops": 3.5 * fwd_flops / att_ms / 1e9, "norm_ms": t["norm"][0] / 5,
+                     "dgrad_ms": t["dgrad"][0] / 5, "wgrad_ms": t["wgrad"][0] / 5, "forward_gemm_ms": t["forward"][0] / 5}
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(args.steps):
+                et.et_forward_stack(stack, x, y)
+            e1.record()
+            torch.cuda.synchronize()
+            extra["forward_ms"] = e0.elapsed_time(e1) / args.steps
         if args.workload == "prenorm":
             # normalisation kernels alone: CUDA-event time of their class over full-backprop steps against
             # the bytes they must move (g, x, skip gradient in; error gradient out; bf16)
@@ -592,7 +620,7 @@ def main():
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
-    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "schedule", "selector"],
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "schedule", "selector"],
                     help="vit_b = the benchmark line; resnet / prenorm / schedule = side reports for the other shapes; "
                          "selector = host-side report on the selection dynamic program")
     args = ap.parse_args()

@@ -23,7 +23,8 @@ namespace attn {
 
 constexpr int DH = 64;           // head width
 constexpr int S_MAX = 208;       // longest sequence (padded to a multiple of 16)
-constexpr int RB = 64;           // query rows per pass
+constexpr int RB = 64;           // query rows per pass, backward
+constexpr int RB_FWD = 32;       // query rows per pass, forward: two CTAs fit on an SM
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
 constexpr int LDK = DH + 8;      // row stride (elements) of the 64-wide bf16 tiles: breaks bank conflicts
@@ -35,7 +36,7 @@ __host__ __device__ inline int pad16(int s) { return (s + 15) & ~15; }
 __host__ __device__ inline int score_ld(int SP) { return SP + 4 > DH + 4 ? SP + 4 : DH + 4; }
 inline size_t forward_smem_bytes(int S) {
   const int SP = pad16(S);
-  return (size_t)(2 * SP + RB) * LDK * 2 + (size_t)RB * score_ld(SP) * 4 + (size_t)RB * (SP + 8) * 2;
+  return (size_t)(2 * SP + RB_FWD) * LDK * 2 + (size_t)RB_FWD * score_ld(SP) * 4 + (size_t)RB_FWD * (SP + 8) * 2;
 }
 inline size_t backward_smem_bytes(int S) {
   const int SP = pad16(S);
@@ -68,88 +69,131 @@ __device__ __forceinline__ void store16(bf16* dst, const float* src) {
   reinterpret_cast<uint4*>(dst)[1] = b;
 }
 
-// Sf[64][ldsf] = Q_blk K^T (fp32), all warps
-__device__ __forceinline__ void scores(const bf16* Qs, const bf16* Ks, float* Sf, int ntn, int ldsf, int warp) {
-  for (int t = warp; t < (RB / 16) * ntn; t += WARPS) {
-    const int mi = t / ntn, nj = t - mi * ntn;
-    FragC acc;
-    nvcuda::wmma::fill_fragment(acc, 0.0f);
+// Sf[RBT][ldsf] = A[RBT][64] * Bt[SP][64]^T (fp32).  A warp keeps its row tile's four A fragments and
+// walks over column tiles two at a time (two independent accumulator chains).
+template <int RBT>
+__device__ __forceinline__ void abt_tiles(const bf16* A, const bf16* Bt, float* Sf, int ntn, int ldsf, int warp) {
+  constexpr int MT = RBT / 16, G = WARPS / MT;
+  const int mi = warp % MT, g = warp / MT;
+  FragA a[DH / 16];
+#pragma unroll
+  for (int kk = 0; kk < DH / 16; ++kk) nvcuda::wmma::load_matrix_sync(a[kk], A + mi * 16 * LDK + kk * 16, LDK);
+  for (int nj = g; nj < ntn; nj += 2 * G) {
+    const int nj2 = nj + G;
+    const bool two = nj2 < ntn;                    // the same for the whole warp
+    FragC acc0, acc1;
+    nvcuda::wmma::fill_fragment(acc0, 0.0f);
+    nvcuda::wmma::fill_fragment(acc1, 0.0f);
 #pragma unroll
     for (int kk = 0; kk < DH / 16; ++kk) {
-      FragA a;
-      FragBT b;
-      nvcuda::wmma::load_matrix_sync(a, Qs + mi * 16 * LDK + kk * 16, LDK);
-      nvcuda::wmma::load_matrix_sync(b, Ks + nj * 16 * LDK + kk * 16, LDK);     // B[k][n] = K[n][k]
-      nvcuda::wmma::mma_sync(acc, a, b, acc);
+      FragBT b0, b1;
+      nvcuda::wmma::load_matrix_sync(b0, Bt + nj * 16 * LDK + kk * 16, LDK);       // B[k][n] = Bt[n][k]
+      if (two) nvcuda::wmma::load_matrix_sync(b1, Bt + nj2 * 16 * LDK + kk * 16, LDK);
+      nvcuda::wmma::mma_sync(acc0, a[kk], b0, acc0);
+      if (two) nvcuda::wmma::mma_sync(acc1, a[kk], b1, acc1);
     }
-    nvcuda::wmma::store_matrix_sync(Sf + mi * 16 * ldsf + nj * 16, acc, ldsf, nvcuda::wmma::mem_row_major);
+    nvcuda::wmma::store_matrix_sync(Sf + mi * 16 * ldsf + nj * 16, acc0, ldsf, nvcuda::wmma::mem_row_major);
+    if (two) nvcuda::wmma::store_matrix_sync(Sf + mi * 16 * ldsf + nj2 * 16, acc1, ldsf, nvcuda::wmma::mem_row_major);
   }
 }
-// Of[64][ldsf] (columns 0..63) = A[64][SP] * Bm[SP][64], A bf16 with stride lda, all warps (2 tiles each)
+// Of[RBT][ldsf] (columns 0..63) = A[RBT][SP] * Bm[SP][64], A bf16 with stride lda.  64 rows: two column
+// tiles per warp sharing the A fragment; 32 rows: one tile per warp, even and odd k steps in two chains.
+template <int RBT>
 __device__ __forceinline__ void rows_times_head(const bf16* A, int lda, const bf16* Bm, float* Of, int ntn, int ldsf,
                                                 int warp) {
-  for (int t = warp; t < (RB / 16) * (DH / 16); t += WARPS) {
-    const int mi = t >> 2, nj = t & 3;
-    FragC acc;
-    nvcuda::wmma::fill_fragment(acc, 0.0f);
+  FragC acc0, acc1;
+  nvcuda::wmma::fill_fragment(acc0, 0.0f);
+  nvcuda::wmma::fill_fragment(acc1, 0.0f);
+  if constexpr (RBT == 64) {
+    const int mi = warp & 3, nj = (warp >> 2) * 2;
     for (int kk = 0; kk < ntn; ++kk) {
       FragA a;
-      FragB b;
+      FragB b0, b1;
       nvcuda::wmma::load_matrix_sync(a, A + mi * 16 * lda + kk * 16, lda);
-      nvcuda::wmma::load_matrix_sync(b, Bm + kk * 16 * LDK + nj * 16, LDK);
-      nvcuda::wmma::mma_sync(acc, a, b, acc);
+      nvcuda::wmma::load_matrix_sync(b0, Bm + kk * 16 * LDK + nj * 16, LDK);
+      nvcuda::wmma::load_matrix_sync(b1, Bm + kk * 16 * LDK + nj * 16 + 16, LDK);
+      nvcuda::wmma::mma_sync(acc0, a, b0, acc0);
+      nvcuda::wmma::mma_sync(acc1, a, b1, acc1);
     }
-    nvcuda::wmma::store_matrix_sync(Of + mi * 16 * ldsf + nj * 16, acc, ldsf, nvcuda::wmma::mem_row_major);
+    nvcuda::wmma::store_matrix_sync(Of + mi * 16 * ldsf + nj * 16, acc0, ldsf, nvcuda::wmma::mem_row_major);
+    nvcuda::wmma::store_matrix_sync(Of + mi * 16 * ldsf + nj * 16 + 16, acc1, ldsf, nvcuda::wmma::mem_row_major);
+  } else {
+    static_assert(RBT == 32, "row block");
+    const int mi = warp & 1, nj = warp >> 1;
+    for (int kk = 0; kk < ntn; kk += 2) {
+      FragA a0, a1;
+      FragB b0, b1;
+      nvcuda::wmma::load_matrix_sync(a0, A + mi * 16 * lda + kk * 16, lda);
+      nvcuda::wmma::load_matrix_sync(b0, Bm + kk * 16 * LDK + nj * 16, LDK);
+      nvcuda::wmma::mma_sync(acc0, a0, b0, acc0);
+      if (kk + 1 < ntn) {
+        nvcuda::wmma::load_matrix_sync(a1, A + mi * 16 * lda + (kk + 1) * 16, lda);
+        nvcuda::wmma::load_matrix_sync(b1, Bm + (kk + 1) * 16 * LDK + nj * 16, LDK);
+        nvcuda::wmma::mma_sync(acc1, a1, b1, acc1);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < acc0.num_elements; ++i) acc0.x[i] += acc1.x[i];
+    nvcuda::wmma::store_matrix_sync(Of + mi * 16 * ldsf + nj * 16, acc0, ldsf, nvcuda::wmma::mem_row_major);
   }
+}
+// 8 consecutive floats of a staged fp32 tile -> 8 bf16 in global memory
+__device__ __forceinline__ void store8(bf16* dst, const float* src) {
+  uint4 a;
+  a.x = pack_bf16x2(src[0], src[1]); a.y = pack_bf16x2(src[2], src[3]);
+  a.z = pack_bf16x2(src[4], src[5]); a.w = pack_bf16x2(src[6], src[7]);
+  *reinterpret_cast<uint4*>(dst) = a;
 }
 
 // grid = sequences * heads.  qkv: [M][3d]; out: [M][d]; lse: [sequences * heads][S].
-static __global__ void __launch_bounds__(THREADS)
+static __global__ void __launch_bounds__(THREADS, 2)
 attn_forward_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float* __restrict__ lse, int S, int H, int d) {
   extern __shared__ __align__(128) uint8_t smem[];
+  constexpr int RBT = RB_FWD;
+  constexpr int TPR = THREADS / RBT;               // threads per row in the row-wise parts: 8
   const int SP = pad16(S), ntn = SP / 16, ldsf = score_ld(SP), ldp = SP + 8;
   bf16* Ks = reinterpret_cast<bf16*>(smem);
   bf16* Vs = Ks + SP * LDK;
   bf16* Qs = Vs + SP * LDK;
-  float* Sf = reinterpret_cast<float*>(Qs + RB * LDK);
-  bf16* Pb = reinterpret_cast<bf16*>(Sf + RB * ldsf);
+  float* Sf = reinterpret_cast<float*>(Qs + RBT * LDK);
+  bf16* Pb = reinterpret_cast<bf16*>(Sf + RBT * ldsf);
   const int b = blockIdx.x / H, h = blockIdx.x - b * H;
   const int warp = threadIdx.x >> 5;
   const size_t ld = (size_t)3 * d;
   const bf16* base = qkv + (size_t)b * S * ld + h * DH;
   load_tile(Ks, base + d, ld, 0, SP, S);
   load_tile(Vs, base + 2 * d, ld, 0, SP, S);
-  for (int rb0 = 0; rb0 < S; rb0 += RB) {
-    load_tile(Qs, base, ld, rb0, RB, S);
+  for (int rb0 = 0; rb0 < S; rb0 += RBT) {
+    load_tile(Qs, base, ld, rb0, RBT, S);
     __syncthreads();
-    scores(Qs, Ks, Sf, ntn, ldsf, warp);
+    abt_tiles<RBT>(Qs, Ks, Sf, ntn, ldsf, warp);
     __syncthreads();
-    {   // softmax of row r by 4 neighbouring lanes
-      const int r = threadIdx.x >> 2, sub = threadIdx.x & 3;
+    {   // softmax of row r by TPR neighbouring lanes
+      const int r = threadIdx.x / TPR, sub = threadIdx.x % TPR;
       const bool valid = rb0 + r < S;
       float* row = Sf + r * ldsf;
       float m = -INFINITY;
-      for (int c = sub; c < S; c += 4) m = fmaxf(m, row[c]);
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+      for (int c = sub; c < S; c += TPR) m = fmaxf(m, row[c]);
+#pragma unroll
+      for (int o = 1; o < TPR; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
       float sum = 0.0f;
-      for (int c = sub; c < S; c += 4) {
+      for (int c = sub; c < S; c += TPR) {
         const float e = __expf((row[c] - m) * SCALE);
         row[c] = e;
         sum += e;
       }
-      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+#pragma unroll
+      for (int o = 1; o < TPR; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
       const float inv = 1.0f / sum;
-      for (int c = sub; c < SP; c += 4) Pb[r * ldp + c] = __float2bfloat16_rn((valid && c < S) ? row[c] * inv : 0.0f);
+      for (int c = sub; c < SP; c += TPR) Pb[r * ldp + c] = __float2bfloat16_rn((valid && c < S) ? row[c] * inv : 0.0f);
       if (valid && sub == 0) lse[(size_t)blockIdx.x * S + rb0 + r] = m * SCALE + __logf(sum);
     }
     __syncthreads();
-    rows_times_head(Pb, ldp, Vs, Sf, ntn, ldsf, warp);
+    rows_times_head<RBT>(Pb, ldp, Vs, Sf, ntn, ldsf, warp);
     __syncthreads();
     {
-      const int r = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * 16;
-      if (rb0 + r < S) store16(out + ((size_t)b * S + rb0 + r) * d + h * DH + c0, Sf + r * ldsf + c0);
+      const int r = threadIdx.x / TPR, c0 = (threadIdx.x % TPR) * (DH / TPR);
+      if (rb0 + r < S) store8(out + ((size_t)b * S + rb0 + r) * d + h * DH + c0, Sf + r * ldsf + c0);
     }
     __syncthreads();
   }
@@ -189,7 +233,7 @@ attn_backward_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out,
     load_tile(Qs, base, ld, rb0, RB, S);
     load_tile(dOs, dobase, (size_t)d, rb0, RB, S);
     __syncthreads();
-    scores(Qs, Ks, Sf, ntn, ldsf, warp);
+    abt_tiles<RB>(Qs, Ks, Sf, ntn, ldsf, warp);
     {   // D_r = dO_r . o_r
       const int r = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * 16;
       float s = 0.0f;
@@ -213,20 +257,7 @@ attn_backward_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out,
     }
     __syncthreads();
     // dP = dO V^T -> Sf
-    for (int t = warp; t < (RB / 16) * ntn; t += WARPS) {
-      const int mi = t / ntn, nj = t - mi * ntn;
-      FragC acc;
-      nvcuda::wmma::fill_fragment(acc, 0.0f);
-#pragma unroll
-      for (int kk = 0; kk < DH / 16; ++kk) {
-        FragA a;
-        FragBT bt;
-        nvcuda::wmma::load_matrix_sync(a, dOs + mi * 16 * LDK + kk * 16, LDK);
-        nvcuda::wmma::load_matrix_sync(bt, Vs + nj * 16 * LDK + kk * 16, LDK);   // B[k][n] = V[n][k]
-        nvcuda::wmma::mma_sync(acc, a, bt, acc);
-      }
-      nvcuda::wmma::store_matrix_sync(Sf + mi * 16 * ldsf + nj * 16, acc, ldsf, nvcuda::wmma::mem_row_major);
-    }
+    abt_tiles<RB>(dOs, Vs, Sf, ntn, ldsf, warp);
     __syncthreads();
     {   // dS = P * (dP - D) / 8
       const int r = threadIdx.x >> 2, sub = threadIdx.x & 3;
@@ -237,23 +268,27 @@ attn_backward_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out,
     }
     __syncthreads();
     // dQ_blk = dS K -> Sf (columns 0..63)
-    rows_times_head(dSb, ldp, Ks, Sf, ntn, ldsf, warp);
-    // dV += P^T dO ; dK += dS^T Q   (contraction over the 64 rows of this block)
+    rows_times_head<RB>(dSb, ldp, Ks, Sf, ntn, ldsf, warp);
+    // dV += P^T dO ; dK += dS^T Q   (contraction over the 64 rows of this block).  All of a warp's output
+    // tiles share their column tile nj, so the dO / Q fragments of a k step are loaded once.
+    {
+      const int nj = warp & 3;
 #pragma unroll
-    for (int i = 0; i < MAX_OWN; ++i) {
-      const int t = warp + WARPS * i;
-      if (t < own_tiles) {
-        const int mj = t >> 2, nj = t & 3;
+      for (int kk = 0; kk < RB / 16; ++kk) {
+        FragB bo, bq;
+        nvcuda::wmma::load_matrix_sync(bo, dOs + kk * 16 * LDK + nj * 16, LDK);
+        nvcuda::wmma::load_matrix_sync(bq, Qs + kk * 16 * LDK + nj * 16, LDK);
 #pragma unroll
-        for (int kk = 0; kk < RB / 16; ++kk) {
-          FragAT pt, st;
-          FragB bo, bq;
-          nvcuda::wmma::load_matrix_sync(pt, Pb + kk * 16 * ldp + mj * 16, ldp);     // A[m][k] = P[k][m]
-          nvcuda::wmma::load_matrix_sync(bo, dOs + kk * 16 * LDK + nj * 16, LDK);
-          nvcuda::wmma::mma_sync(accV[i], pt, bo, accV[i]);
-          nvcuda::wmma::load_matrix_sync(st, dSb + kk * 16 * ldp + mj * 16, ldp);
-          nvcuda::wmma::load_matrix_sync(bq, Qs + kk * 16 * LDK + nj * 16, LDK);
-          nvcuda::wmma::mma_sync(accK[i], st, bq, accK[i]);
+        for (int i = 0; i < MAX_OWN; ++i) {
+          const int t = warp + WARPS * i;
+          if (t < own_tiles) {
+            const int mj = t >> 2;
+            FragAT pt, st;
+            nvcuda::wmma::load_matrix_sync(pt, Pb + kk * 16 * ldp + mj * 16, ldp);     // A[m][k] = P[k][m]
+            nvcuda::wmma::load_matrix_sync(st, dSb + kk * 16 * ldp + mj * 16, ldp);
+            nvcuda::wmma::mma_sync(accV[i], pt, bo, accV[i]);
+            nvcuda::wmma::mma_sync(accK[i], st, bq, accK[i]);
+          }
         }
       }
     }

@@ -81,3 +81,29 @@ def test_unsupported_shapes_and_selections_are_refused():
     bad = w.mask.copy(); bad[6] = 1
     with pytest.raises(et.EtError):
         et.et_backward_elastic(run.stack, run.dY, bad, None, None, None, 0, 0.0, None)
+
+
+def test_profiled_costs_follow_the_papers_rules_for_non_dense_layers():
+    # Section 5.2: a normalisation layer's whole backward time sits in t_dy of beta; Section 5.3: the
+    # attention core's backward time joins t_dy of the bias of the trainable layer below it
+    import torch
+    h = _h()
+    layers = _stack(128, 2, 40)
+    w = wl.small_stack(layers, 8 * 40, wl.DT_BF16, 85, mask=_mask_all(layers), w_std=0.1)
+    run = h.GpuRun(w)
+    run.forward_loss()
+    t_dw, t_dy, t_fwd = et.et_profile_costs(run.stack, run.x, run.y, run.dY, iters=3)
+    assert t_fwd > 0
+    assert t_dw[2] == 0 and t_dw[3] == 0 and t_dy[2] == 0 and t_dy[3] > 0            # layer 1: normalisation
+    assert t_dw[6] == 0 and t_dw[7] == 0 and t_dy[6] == 0 and t_dy[7] == 0            # layer 3: attention core
+    assert t_dy[5] > 0                                                                # bias of the QKV layer below it
+    for l in (0, 2, 4, 5):                                                            # dense layers
+        assert t_dw[2 * l] > 0 and t_dw[2 * l + 1] > 0
+        assert (t_dy[2 * l] > 0) == (l > 0)
+    for l in (0, 4, 5):
+        assert t_dy[2 * l + 1] == 0                                                   # a plain bias passes nothing on
+    # the selector accepts these vectors as they are
+    imp = np.abs(np.random.default_rng(0).normal(size=12))
+    imp[6:8] = 0.0
+    mask, val, est = et.et_select_dp(imp, t_dw, t_dy, t_fwd, 0.6, 1000)
+    assert mask[6] == 0 and mask[7] == 0 and est <= 0.6 * (t_fwd + t_dw.sum() + t_dy.sum()) - t_fwd + 12 * (t_dw.sum() + t_dy.sum()) / 1000
