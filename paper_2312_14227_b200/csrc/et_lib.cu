@@ -1379,6 +1379,8 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
     ET_TRY(timed([&]() { return et_forward_stack(s, x, y, stream); }, &fwd));
     if (t_fwd != nullptr) *t_fwd = fwd;
     std::vector<uint8_t> ones(2 * L, 1);
+    for (int l = 0; l < L; ++l)
+      if (!s->ly[l].trainable()) ones[2 * l] = ones[2 * l + 1] = 0;
     ET_TRY(et_backward_elastic(s, dY, ones.data(), 2 * L, nullptr, nullptr, nullptr, 0, 0.f, nullptr, stream));
     float* scratch_grad = (float*)s->at(s->off_partial);      // in-place: each element is read before it is written
     double pending_nontrainable = 0.0;
