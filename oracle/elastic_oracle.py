@@ -18,6 +18,11 @@ or, for a normalisation layer (Section 5.2; its Gamma and Beta are tensors 2*l a
     xhat    = (a_l - mean) / sqrt(var + eps)         mean, var over the features of each row
     a_{l+1} = xhat * gamma_l + beta_l
 
+or, for a patch-gather layer (no trainable tensors; with the dense layer after it, it is a k x k
+convolution with stride 1 and zero padding k // 2 on NHWC rows, the convolutional layer of Section 5.1),
+
+    a_{l+1}[(n,h,w), (kh*k + kw)*C + c] = a_l[(n, h + kh - k//2, w + kw - k//2), c]     (0 outside the image)
+
 or, for an attention layer (no trainable tensors; Sections 5.3 / 5.4 count attention operations as
 non-trainable layers), with a_l = [q | k | v] (three blocks of `heads * head_dim` columns) and the
 rows grouped into sequences of `seq` consecutive tokens,
@@ -41,7 +46,7 @@ from typing import Dict, List, Optional, Sequence
 import numpy as np
 
 ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
-KIND_DENSE, KIND_NORM, KIND_ATTENTION = 0, 1, 2
+KIND_DENSE, KIND_NORM, KIND_ATTENTION, KIND_IM2COL = 0, 1, 2, 3
 STRICT, INCLUSIVE = 0, 1
 
 
@@ -90,6 +95,18 @@ def forward(layers, W: Sequence[np.ndarray], b: Sequence[np.ndarray], x: np.ndar
     a = [np.asarray(x, dtype=np.float64)]
     Z = []
     for l, ly in enumerate(layers):
+        if _kind(ly) == KIND_IM2COL:
+            # patch gather of a k x k convolution, stride 1, zero padding k // 2, on NHWC rows:
+            # col[(n,h,w), (kh*k + kw)*C + c] = x[n, h + kh - p, w + kw - p, c]  (0 outside the image)
+            C_, Hh, Ww, k = ly.in_features, ly.height, ly.width, ly.ksize
+            pd = k // 2
+            xi = a[l].reshape(-1, Hh, Ww, C_)
+            xp = np.zeros((xi.shape[0], Hh + 2 * pd, Ww + 2 * pd, C_))
+            xp[:, pd:pd + Hh, pd:pd + Ww, :] = xi
+            col = np.concatenate([xp[:, kh:kh + Hh, kw:kw + Ww, :] for kh in range(k) for kw in range(k)], axis=3)
+            Z.append(None)
+            a.append(col.reshape(a[l].shape[0], k * k * C_))
+            continue
         if _kind(ly) == KIND_ATTENTION:
             d = ly.out_features
             H, S = ly.heads, ly.seq
@@ -186,6 +203,23 @@ def _backward_sweep(layers, W, saved: Saved, dY: np.ndarray, stop: int,
     for l in range(L - 1, stop - 1, -1):
         ly = layers[l]
         g_out = G[l + 1]
+        if _kind(ly) == KIND_IM2COL:
+            if want_w[l]:
+                grads[2 * l] = np.zeros(0)
+            if want_b[l]:
+                grads[2 * l + 1] = np.zeros(0)
+            if l > stop:
+                # every input pixel collects the gradient of each patch position it was copied to
+                C_, Hh, Ww, k = ly.in_features, ly.height, ly.width, ly.ksize
+                pd = k // 2
+                gc = g_out.reshape(-1, Hh, Ww, k * k, C_)
+                gp = np.zeros((gc.shape[0], Hh + 2 * pd, Ww + 2 * pd, C_))
+                for kh in range(k):
+                    for kw in range(k):
+                        gp[:, kh:kh + Hh, kw:kw + Ww, :] += gc[:, :, :, kh * k + kw, :]
+                dX = gp[:, pd:pd + Hh, pd:pd + Ww, :].reshape(-1, C_)
+                G[l] = dX if G[l] is None else G[l] + dX
+            continue
         if _kind(ly) == KIND_ATTENTION:
             if want_w[l]:
                 grads[2 * l] = np.zeros(0)                                  # its tensor slots are empty

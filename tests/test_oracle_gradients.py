@@ -322,3 +322,52 @@ def test_attention_closed_forms():
     q2 = np.ones((6, 4))
     o = orc.forward(ly, [np.zeros(0)], [np.zeros(0)], np.concatenate([q2, k2, v], axis=1)).a[-1]
     assert np.allclose(o[:3], np.tile(v[1], (3, 1))) and np.allclose(o[3:], np.tile(v[3:].mean(0), (3, 1)))
+
+
+# ------------------------------------------------------------------ k x k convolution = patch gather + dense layer
+def test_convolution_matches_the_library_conv2d():
+    torch = pytest.importorskip("torch")
+    F = torch.nn.functional
+    n, H, W, cin, cmid, cout, k = 2, 5, 4, 3, 6, 4, 3
+    layers = [wl.Layer(cin, cmid, act=wl.ACT_RELU)] + wl.conv_layers(cmid, cout, H, W, k, act=wl.ACT_GELU_TANH) + \
+        wl.conv_layers(cout, 5, H, W, 5)
+    w = wl.small_stack(layers, n * H * W, wl.DT_F32, 61, w_std=0.5, bias_std=0.2)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    grads = orc.backward_full(w.layers, w.W, saved, dY)
+    tW = {l: torch.tensor(w.W[l], dtype=torch.float64, requires_grad=True) for l in (0, 2, 4)}
+    tb = {l: torch.tensor(w.b[l], dtype=torch.float64, requires_grad=True) for l in (0, 2, 4)}
+    h = torch.relu(torch.tensor(w.x, dtype=torch.float64) @ tW[0] + tb[0])
+    img = h.reshape(n, H, W, cmid).permute(0, 3, 1, 2)                            # NCHW for the library
+    k1 = tW[2].reshape(k, k, cmid, cout).permute(3, 2, 0, 1)                       # (kh, kw, cin, cout) -> OIHW
+    img = F.gelu(F.conv2d(img, k1, tb[2], padding=k // 2), approximate="tanh")
+    k2 = tW[4].reshape(5, 5, cout, 5).permute(3, 2, 0, 1)
+    img = F.conv2d(img, k2, tb[4], padding=2)
+    y = img.permute(0, 2, 3, 1).reshape(n * H * W, 5)
+    assert np.allclose(y.detach().numpy(), saved.a[-1], rtol=1e-10, atol=1e-12)
+    loss = ((y - torch.tensor(w.target, dtype=torch.float64)) ** 2).mean()
+    loss.backward()
+    for l in (0, 2, 4):
+        assert np.allclose(grads[2 * l], tW[l].grad.numpy(), rtol=1e-9, atol=1e-13), l
+        assert np.allclose(grads[2 * l + 1], tb[l].grad.numpy(), rtol=1e-9, atol=1e-13), l
+
+
+def test_finite_differences_through_convolutions():
+    layers = [wl.Layer(3, 4, act=wl.ACT_GELU_TANH)] + wl.conv_layers(4, 4, 3, 4, 3, act=wl.ACT_RELU) + \
+        [wl.Layer(4, 4, residual_src=1)] + wl.conv_layers(4, 2, 3, 4, 3)
+    _fd_check(layers, M=2 * 12, seed=62, tol=5e-6)
+
+
+def test_patch_gather_closed_forms():
+    # a 1 x 1 "convolution" gathers nothing but the pixel itself; a 3 x 3 gather of a one-hot image puts the
+    # hot pixel into tap (2 - dh, 2 - dw) of its neighbour at offset (dh - 1, dw - 1); borders see zeros
+    x = np.arange(2 * 3 * 3 * 2, dtype=np.float64).reshape(18, 2)
+    one = [wl.Layer(2, 2, kind=wl.KIND_IM2COL, height=3, width=3, ksize=1)]
+    assert np.array_equal(orc.forward(one, [np.zeros(0)], [np.zeros(0)], x).a[-1], x)
+    hot = np.zeros((9, 1)); hot[4] = 1.0                                           # centre of a 3 x 3 image
+    g = [wl.Layer(1, 9, kind=wl.KIND_IM2COL, height=3, width=3, ksize=3)]
+    col = orc.forward(g, [np.zeros(0)], [np.zeros(0)], hot).a[-1]
+    assert np.array_equal(col, np.eye(9)[::-1])                                   # pixel p sees the centre in tap 8 - p
+    corner = np.zeros((9, 1)); corner[0] = 1.0
+    col = orc.forward(g, [np.zeros(0)], [np.zeros(0)], corner).a[-1]
+    assert col.sum() == 4 and col[0, 4] == 1 and col[1, 3] == 1 and col[3, 1] == 1 and col[4, 0] == 1

@@ -27,7 +27,9 @@ ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
 DT_F32, DT_BF16 = 0, 1
 # layer kinds: a dense layer (kernel, bias) or a layer normalisation over the feature axis, whose two
 # trainable tensors gamma and beta take the kernel and bias slots (Section 5.2: Gamma and Beta)
-KIND_DENSE, KIND_NORM, KIND_ATTENTION = 0, 1, 2
+KIND_DENSE, KIND_NORM, KIND_ATTENTION, KIND_IM2COL = 0, 1, 2, 3
+# KIND_IM2COL: the patch-gathering half of a k x k convolution (stride 1, zero padding k // 2) on NHWC
+# rows; followed by a dense layer with in_features = k * k * channels it is that convolution.  No tensors.
 # KIND_ATTENTION: the softmax attention core, a layer without trainable tensors (Section 5.3 / 5.4:
 # attention operations are non-trainable layers); its two tensor slots are empty
 
@@ -44,6 +46,9 @@ class Layer:
     eps: float = 1e-5          # KIND_NORM: added to the variance
     heads: int = 0             # KIND_ATTENTION: in_features = 3 * out_features = 3 * heads * head_dim,
     seq: int = 0               #   rows come in sequences of `seq` consecutive tokens
+    height: int = 0            # KIND_IM2COL: rows are images of height x width pixels (row = (n, h, w)),
+    width: int = 0             #   in_features = channels, out_features = ksize * ksize * channels,
+    ksize: int = 0             #   column (kh * ksize + kw) * channels + c holds pixel (h + kh - k//2, w + kw - k//2)
 
     @property
     def out_width(self) -> int:
@@ -148,6 +153,25 @@ def vit_blocks_full(n_blocks: int, d: int, ffn: int, heads: int, seq: int) -> Li
     return layers
 
 
+def conv_layers(c_in: int, c_out: int, height: int, width: int, ksize: int = 3, act: int = ACT_NONE,
+                residual_src: int = -1) -> List[Layer]:
+    """A k x k convolution (stride 1, "same" zero padding) on NHWC rows as two stack layers: the patch
+    gather and a dense layer whose kernel is the convolution kernel in (kh, kw, c_in) x c_out layout."""
+    return [Layer(c_in, ksize * ksize * c_in, kind=KIND_IM2COL, height=height, width=width, ksize=ksize),
+            Layer(ksize * ksize * c_in, c_out, act=act, residual_src=residual_src)]
+
+
+def resnet_bottleneck_blocks(n_blocks: int, c: int, mid: int, height: int, width: int) -> List[Layer]:
+    """ResNet bottleneck: 1x1 c->mid ReLU, 3x3 mid->mid ReLU, 1x1 mid->c + block input (4 layers)."""
+    layers: List[Layer] = []
+    for blk in range(n_blocks):
+        base = 4 * blk
+        layers.append(Layer(c, mid, act=ACT_RELU))
+        layers += conv_layers(mid, mid, height, width, 3, act=ACT_RELU)
+        layers.append(Layer(mid, c, residual_src=base))
+    return layers
+
+
 def vit_blocks_prenorm(n_blocks: int, d: int, ffn: int) -> List[Layer]:
     """Pre-norm transformer block, attention core still the identity:
     LN, QKV d->3d (three slices summed), out-proj d->d + block input,
@@ -168,7 +192,7 @@ def vit_blocks_prenorm(n_blocks: int, d: int, ffn: int) -> List[Layer]:
 def _draw_params(rng, layers, dtype, w_std=None, he_init=False):
     W, b = [], []
     for ly in layers:
-        if ly.kind == KIND_ATTENTION:
+        if ly.kind in (KIND_ATTENTION, KIND_IM2COL):
             W.append(np.zeros(0)); b.append(np.zeros(0))
             continue
         if ly.kind == KIND_NORM:
@@ -261,6 +285,19 @@ def resnet_1x1(seed: int = 2, p_select: float = 0.5, n_blocks: int = 6, tokens: 
                    he_init=True, params=params)
 
 
+def resnet_bottleneck(seed: int = 6, p_select: float = 0.5, n_blocks: int = 6, images: int = 32, height: int = 14,
+                      width: int = 14, c: int = 1024, mid: int = 256, params: bool = True) -> Workload:
+    """bf16 ResNet-50 conv4_x bottlenecks with their 3x3 convolutions (NHWC rows)."""
+    rng = np.random.default_rng(seed)
+    layers = resnet_bottleneck_blocks(n_blocks, c, mid, height, width)
+    mask = bernoulli_weight_mask(rng, len(layers), p_select)
+    for l, ly in enumerate(layers):
+        if ly.kind == KIND_IM2COL:
+            mask[2 * l] = mask[2 * l + 1] = 0
+    return _finish("resnet50_conv4_bottleneck_bf16", layers, images * height * width, DT_BF16, 0.01, mask, rng,
+                   he_init=True, params=params)
+
+
 def small_stack(layers: List[Layer], M: int, dtype: int, seed: int, mask=None, w_std: float = 0.05,
                 bias_std: float = 0.0, lr: float = 0.01) -> Workload:
     """Arbitrary small stack for parity and oracle tests (ragged sizes, every act/fold/residual kind)."""
@@ -269,8 +306,8 @@ def small_stack(layers: List[Layer], M: int, dtype: int, seed: int, mask=None, w
         mask = (rng.random(2 * len(layers)) < 0.5).astype(np.uint8)
     wl = _finish("small", layers, M, dtype, lr, np.asarray(mask, dtype=np.uint8), rng, w_std=w_std)
     if bias_std > 0:
-        wl.b = [np.zeros(0) if ly.kind == KIND_ATTENTION else _store(rng.normal(0.0, bias_std, size=ly.out_features), dtype)
-                for ly in layers]
+        wl.b = [np.zeros(0) if ly.kind in (KIND_ATTENTION, KIND_IM2COL)
+                else _store(rng.normal(0.0, bias_std, size=ly.out_features), dtype) for ly in layers]
     return wl
 
 
@@ -294,7 +331,7 @@ def draw_delta(w: Workload, seed: int, std: float = 1e-3):
     rng = np.random.default_rng(seed)
     out = []
     for ly in w.layers:
-        if ly.kind == KIND_ATTENTION:
+        if ly.kind in (KIND_ATTENTION, KIND_IM2COL):
             out += [np.zeros(0), np.zeros(0)]
             continue
         shape = (ly.out_features,) if ly.kind == KIND_NORM else (ly.in_features, ly.out_features)
