@@ -29,6 +29,12 @@
  *   slots in gradient / importance / state arrays are ignored.  Its backward (above the deepest
  *   selected layer only) recomputes P from the saved per-row log-sum-exp.
  *
+ *   A layer of kind ET_LAYER_IM2COL gathers the k x k patches of a convolution (stride 1, zero
+ *   padding k / 2) from NHWC rows:  a_{l+1}[(n,h,w), (kh*k + kw)*C + c] = a_l[(n, h+kh-k/2, w+kw-k/2), c].
+ *   Followed by a dense layer with in_features = k*k*C it is the convolutional layer of Section 5.1
+ *   (that layer's kernel is the convolution kernel in (kh, kw, c_in) x c_out layout).  Like the
+ *   attention core it has no tensors: NULL pointers, mask bits 0.
+ *
  *   A layer of kind ET_LAYER_NORM is a layer normalisation over the features of each row
  *   (Section 5.2 treats normalisation layers as two trainable tensors, Gamma and Beta;
  *   Section 5.4 says LayerNorm behaves like batch normalisation in this respect):
@@ -80,7 +86,7 @@ typedef enum {
 
 typedef enum { ET_F32 = 0, ET_BF16 = 1 } et_dtype;
 typedef enum { ET_ACT_NONE = 0, ET_ACT_GELU_TANH = 1, ET_ACT_RELU = 2 } et_act;
-typedef enum { ET_LAYER_DENSE = 0, ET_LAYER_NORM = 1, ET_LAYER_ATTENTION = 2 } et_layer_kind;
+typedef enum { ET_LAYER_DENSE = 0, ET_LAYER_NORM = 1, ET_LAYER_ATTENTION = 2, ET_LAYER_IM2COL = 3 } et_layer_kind;
 
 /* Cost-model reading for the selector (Section 2.2 / Eq. 7 versus the example after Eq. 3). */
 typedef enum {
@@ -109,6 +115,9 @@ typedef struct {
   int32_t seq_len;        /*   rows form sequences of seq_len (<= 208) consecutive rows, M a multiple of it;  */
                           /*   ET_BF16 only; not the first or last layer; the layer below has no activation;   */
                           /*   act = ET_ACT_NONE, fold = 1, residual_src = -1.  Both fields 0 for other kinds. */
+  int32_t height;         /* ET_LAYER_IM2COL: rows are images of height x width pixels, NHWC (M a multiple of  */
+  int32_t width;          /*   height * width); in_features = channels (a multiple of 8), out_features =        */
+  int32_t ksize;          /*   ksize^2 * channels, ksize odd and <= 7; act, fold, residual_src as for attention. */
 } et_layer_desc;
 
 /* What one et_backward_elastic call executed.  The four arrays are caller-owned host
@@ -351,7 +360,7 @@ typedef enum {
   ET_K_BGRAD = 4,          /* bias gradient: column sums + finish (T2)                  */
   ET_K_OTHER = 5,          /* loss gradient, top-layer activation backward, importance finalise */
   ET_K_NORM = 6,           /* normalisation layers: forward, backward (error gradient + d gamma), gamma finish */
-  ET_K_ATTENTION = 7,      /* attention core: forward, backward */
+  ET_K_ATTENTION = 7,      /* layers without tensors: attention core, patch gather; forward, backward */
   ET_K_CLASSES = 8
 } et_kernel_class;
 

@@ -31,10 +31,11 @@ ET_NOALLOC_SCRATCH_FLOATS = 1 << 20
 class et_layer_desc(C.Structure):
     _fields_ = [("in_features", C.c_int32), ("out_features", C.c_int32), ("act", C.c_int32),
                 ("fold", C.c_int32), ("residual_src", C.c_int32), ("kind", C.c_int32), ("eps", C.c_float),
-                ("heads", C.c_int32), ("seq_len", C.c_int32)]
+                ("heads", C.c_int32), ("seq_len", C.c_int32), ("height", C.c_int32), ("width", C.c_int32),
+                ("ksize", C.c_int32)]
 
 
-ET_LAYER_DENSE, ET_LAYER_NORM, ET_LAYER_ATTENTION = 0, 1, 2
+ET_LAYER_DENSE, ET_LAYER_NORM, ET_LAYER_ATTENTION, ET_LAYER_IM2COL = 0, 1, 2, 3
 
 
 class et_optimizer_config(C.Structure):
@@ -243,7 +244,8 @@ class Stack:
             else:
                 descs[i] = et_layer_desc(ly.in_features, ly.out_features, ly.act, ly.fold, ly.residual_src,
                                          getattr(ly, "kind", ET_LAYER_DENSE), getattr(ly, "eps", 0.0),
-                                         getattr(ly, "heads", 0), getattr(ly, "seq", 0))
+                                         getattr(ly, "heads", 0), getattr(ly, "seq", 0), getattr(ly, "height", 0),
+                                         getattr(ly, "width", 0), getattr(ly, "ksize", 0))
         self.out_width = (descs[self.L - 1].out_features // max(descs[self.L - 1].fold, 1)) if self.L else 0
         h = C.c_void_p()
         _check(_lib.et_stack_create(descs, self.L, self.M, dtype, C.byref(h)), "et_stack_create")

@@ -19,6 +19,7 @@
 #include "kernels.cuh"
 #include "norm.cuh"
 #include "attn.cuh"
+#include "im2col.cuh"
 
 namespace {
 
@@ -150,8 +151,9 @@ struct LayerRT {
   int bn_fwd = 256, bn_dgrad = 256, bn_wgrad = 256;   // tile widths chosen per GEMM
   bool pair_fwd = false, pair_dgrad = false, pair_wgrad = false;   // CTA-pair (cta_group::2) tiles
   int imp_count_w = 0, imp_count_b = 0;
-  bool trainable() const { return kind != ET_LAYER_ATTENTION; }
-  size_t w_count() const { return kind == ET_LAYER_ATTENTION ? 0 : kind == ET_LAYER_NORM ? (size_t)N : (size_t)K * N; }   // elements of tensor 2l
+  int img_h = 0, img_w = 0, ksize = 0;   // patch gather: K = channels, N = ksize^2 * K
+  bool trainable() const { return kind == ET_LAYER_DENSE || kind == ET_LAYER_NORM; }
+  size_t w_count() const { return !trainable() ? 0 : kind == ET_LAYER_NORM ? (size_t)N : (size_t)K * N; }   // elements of tensor 2l
   // bf16 stacks: one TMA descriptor per tensor (the caller's x, y and dY get theirs per call)
   TMaps map_W, map_aout, map_Gout, map_Z, map_dZ;
   CUtensorMap map_Wd;       // W as the K-major B of the dgrad GEMM: one box = the CTA's whole B tile
@@ -651,6 +653,33 @@ et_status run_attn_backward(et_stack* s, int l, const void* dY, cudaStream_t st)
   return after_launch();
 }
 
+// ---- patch gather of a convolution --------------------------------------------------------------
+template <typename T>
+et_status run_im2col_forward(et_stack* s, int l, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_ATTENTION, st);
+  const LayerRT& L = s->ly[l];
+  const long long total = (long long)s->M * L.ksize * L.ksize * (L.K / 8);
+  et::im2col_kernel<T><<<ceil_div(total, et::kGatherThreads), et::kGatherThreads, 0, st>>>(
+      act_in<T>(s, l), (T*)s->at(L.off_a_out), s->M, L.img_h, L.img_w, L.K, L.ksize);
+  return after_launch();
+}
+// G_l (with the skip gradient) and dZ_{l-1} from the gradient of the gathered rows; l >= 1.
+template <typename T>
+et_status run_im2col_backward(et_stack* s, int l, const void* dY, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_ATTENTION, st);
+  const LayerRT& L = s->ly[l];
+  const LayerRT& P = s->ly[l - 1];
+  const bool need_act = P.act != ET_ACT_NONE;
+  const bool need_G = !need_act || P.residual_src >= 0;
+  const T* skip = L.consumer >= 0 ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
+  const long long total = (long long)s->M * (L.K / 8);
+  et::col2im_kernel<T><<<ceil_div(total, et::kGatherThreads), et::kGatherThreads, 0, st>>>(
+      grad_act<T>(s, l + 1, dY), skip, need_G ? (T*)s->at(P.off_G_out) : nullptr,
+      need_act ? (const T*)s->at(P.off_Z) : nullptr, need_act ? (T*)s->at(P.off_dZ) : nullptr, P.act, s->M, L.img_h,
+      L.img_w, L.K, L.ksize);
+  return after_launch();
+}
+
 // dW_l = a_l^T dZ_l as split partials, then the reducer with grad / importance / SGD.
 template <typename T>
 et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const T* delta, bool sgd, float lr,
@@ -843,10 +872,11 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         ET_TRY(run_bgrad_layer<T>(s, l, dY, grads ? grads[2 * l + 1] : nullptr,
                                   delta ? (const T*)delta[2 * l + 1] : nullptr, sgd, lr, &launches, bs, fused));
       }
-      if (Y.kind == ET_LAYER_ATTENTION) {
+      if (!Y.trainable()) {
         // a non-trainable layer: only passes the error gradient on, above the deepest selected layer
         if (l > d) {
-          ET_TRY(run_attn_backward(s, l, dY, cs));
+          if (Y.kind == ET_LAYER_ATTENTION) ET_TRY(run_attn_backward(s, l, dY, cs));
+          else ET_TRY(run_im2col_backward<T>(s, l, dY, cs));
           ++launches;
           if (two) CU_TRY(cudaEventRecord(s->chain_ev[l], cs));
         }
@@ -925,6 +955,7 @@ et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
   for (int l = 0; l < s->L; ++l) {
     if (s->ly[l].kind == ET_LAYER_NORM) ET_TRY(run_norm_forward<T>(s, l, y, st));
     else if (s->ly[l].kind == ET_LAYER_ATTENTION) ET_TRY(run_attn_forward(s, l, st));
+    else if (s->ly[l].kind == ET_LAYER_IM2COL) ET_TRY(run_im2col_forward<T>(s, l, st));
     else ET_TRY(run_forward_layer<T>(s, l, y, st));
   }
   s->forwarded = true;
@@ -968,8 +999,17 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (d.fold > 1 && d.act != ET_ACT_NONE) { err = ET_ERR_UNSUPPORTED; break; }
     y.K = d.in_features; y.N = d.out_features; y.fold = d.fold; y.Nw = d.out_features / d.fold;
     y.act = d.act; y.residual_src = d.residual_src;
-    if (d.kind != ET_LAYER_DENSE && d.kind != ET_LAYER_NORM && d.kind != ET_LAYER_ATTENTION) { err = ET_ERR_INVALID_ARG; break; }
+    if (d.kind < ET_LAYER_DENSE || d.kind > ET_LAYER_IM2COL) { err = ET_ERR_INVALID_ARG; break; }
     y.kind = d.kind; y.eps = d.eps;
+    if (y.kind == ET_LAYER_IM2COL) {
+      y.img_h = d.height; y.img_w = d.width; y.ksize = d.ksize;
+      if (y.fold != 1 || y.act != ET_ACT_NONE || y.residual_src != -1 || y.img_h < 1 || y.img_w < 1 || y.ksize < 1 ||
+          y.ksize % 2 == 0 || (long long)y.N != (long long)y.ksize * y.ksize * y.K) {
+        err = ET_ERR_INVALID_ARG; break;
+      }
+      if (M % ((long long)y.img_h * y.img_w) != 0) { err = ET_ERR_SHAPE; break; }
+      if (y.K % 8 || y.ksize > 7 || l == L - 1) { err = ET_ERR_UNSUPPORTED; break; }
+    }
     if (y.kind == ET_LAYER_ATTENTION) {
       y.heads = d.heads; y.seq = d.seq_len;
       if (y.fold != 1 || y.act != ET_ACT_NONE || y.residual_src != -1 || y.heads < 1 || y.seq < 1 || y.K != 3 * y.N) {
@@ -1045,7 +1085,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
         }
       }
     }
-    if (y.kind == ET_LAYER_ATTENTION) {                    // no tensors: no partials, no importance slots
+    if (!y.trainable()) {                                  // no tensors: no partials, no importance slots
       y.imp_count_w = y.imp_count_b = 0;
       s->imp_offs[2 * l] = s->imp_offs[2 * l + 1] = imp_total;
       s->imp_counts[2 * l] = s->imp_counts[2 * l + 1] = 0;
@@ -1387,12 +1427,16 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
     for (int l = L - 1; l >= 0; --l) {
       int dummy = 0;
       t_dy[2 * l] = 0.0; t_dy[2 * l + 1] = 0.0;
-      if (s->ly[l].kind == ET_LAYER_ATTENTION) {
+      if (!s->ly[l].trainable()) {
         // Section 5.3: a non-trainable layer's backward time joins t_dy of the closest tensor of the
         // trainable layer below it (that layer's bias)
         t_dw[2 * l] = 0.0; t_dw[2 * l + 1] = 0.0;
         double t_attn = 0.0;
-        ET_TRY(timed([&]() { return run_attn_backward(s, l, dY, st); }, &t_attn));
+        if (l >= 1) {
+          if (s->ly[l].kind == ET_LAYER_ATTENTION) ET_TRY(timed([&]() { return run_attn_backward(s, l, dY, st); }, &t_attn));
+          else if (s->dtype == ET_BF16) ET_TRY(timed([&]() { return run_im2col_backward<bf16>(s, l, dY, st); }, &t_attn));
+          else ET_TRY(timed([&]() { return run_im2col_backward<float>(s, l, dY, st); }, &t_attn));
+        }
         pending_nontrainable += t_attn;
         continue;
       }
