@@ -463,7 +463,8 @@ def run_side(args):
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
-    w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "full": wl.vit_b_full, "schedule": wl.vit_l}[args.workload]()
+    w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "full": wl.vit_b_full, "bottleneck": wl.resnet_bottleneck,
+         "schedule": wl.vit_l}[args.workload]()
     tdt = torch.bfloat16
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
     stack = et.et_stack_create(w.layers, w.M, w.dtype)
@@ -476,11 +477,11 @@ def run_side(args):
     et.et_forward_stack(stack, x, y)
     et.et_loss_mse_grad(stack, y, target, dY, None)
     torch.cuda.synchronize()
-    if args.workload in ("resnet", "prenorm", "full"):
+    if args.workload in ("resnet", "prenorm", "full", "bottleneck"):
         rep = et.Report(w.L)
         all_trainable = np.ones(2 * w.L, dtype=np.uint8)
         for l, ly in enumerate(w.layers):
-            if ly.kind == wl.KIND_ATTENTION:             # a layer without tensors cannot be selected
+            if ly.kind in (wl.KIND_ATTENTION, wl.KIND_IM2COL):   # a layer without tensors cannot be selected
                 all_trainable[2 * l] = all_trainable[2 * l + 1] = 0
         delta = [to_dev(d) for d in wl.draw_delta(w, 5)]
         imp = torch.zeros(2 * w.L, dtype=torch.float32, device=dev)
@@ -527,6 +528,21 @@ def run_side(args):
             gms = gfms = None
             print("graph capture failed:", exc, file=sys.stderr)
         extra = {}
+        if args.workload == "bottleneck":
+            # the gather kernels alone: forward writes k*k times the activation, backward reads as much
+            et.et_timing_enable(stack, True)
+            for _ in range(5):
+                et.et_forward_stack(stack, x, y)
+                et.et_backward_elastic(stack, dY, all_trainable, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep)
+            t = et.et_timing_read(stack)
+            et.et_timing_enable(stack, False)
+            g = [ly for ly in w.layers if ly.kind == wl.KIND_IM2COL]
+            nbytes = sum(2.0 * (w.M * ly.in_features + w.M * ly.out_features) * 2 for ly in g)   # fwd + bwd, bf16
+            gather_ms = t["attention"][0] / 5
+            extra = {"gather_ms_per_forward_plus_backward": gather_ms, "gather_launches": t["attention"][1] / 5,
+                     "gather_gbs": nbytes / gather_ms / 1e6,
+                     "gather_frac_of_hbm_peak": nbytes / gather_ms / 1e6 / _peaks()["hbm_gbs"],
+                     "dgrad_ms": t["dgrad"][0] / 5, "wgrad_ms": t["wgrad"][0] / 5, "forward_gemm_ms": t["forward"][0] / 5}
         if args.workload == "full":
             # the attention kernels alone, over full-backprop steps: 4 S^2 64 flops per (sequence, head)
             # forward, 2.5 times that backward (five GEMMs, one of them the recomputed scores)
@@ -620,7 +636,7 @@ def main():
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
-    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "schedule", "selector"],
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "bottleneck", "schedule", "selector"],
                     help="vit_b = the benchmark line; resnet / prenorm / schedule = side reports for the other shapes; "
                          "selector = host-side report on the selection dynamic program")
     args = ap.parse_args()
