@@ -28,7 +28,9 @@ constexpr int RB_FWD = 32;       // query rows per pass, forward: two CTAs fit o
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
 constexpr int LDK = DH + 8;      // row stride (elements) of the 64-wide bf16 tiles: breaks bank conflicts
-constexpr int MAX_OWN = 7;       // (S_MAX / 16) * (DH / 16) = 52 output tiles of dK (or dV) over 8 warps
+constexpr int THREADS_BWD = 512; // backward: 16 warps, each with a quarter of the registers' worth of dK / dV tiles
+constexpr int WARPS_BWD = THREADS_BWD / 32;
+constexpr int MAX_OWN = 4;       // (S_MAX / 16) * (DH / 16) = 52 output tiles of dK (or dV) over 16 warps
 constexpr float SCALE = 0.125f;  // 1 / sqrt(DH)
 
 __host__ __device__ inline int pad16(int s) { return (s + 15) & ~15; }
@@ -50,8 +52,9 @@ using FragBT = nvcuda::wmma::fragment<nvcuda::wmma::matrix_b, 16, 16, 16, bf16, 
 using FragC = nvcuda::wmma::fragment<nvcuda::wmma::accumulator, 16, 16, 16, float>;
 
 // rows [row0, row0 + nrows) of one head's 64 columns -> tile[r][LDK]; rows at or past S read as zeros
+template <int NT = THREADS>
 __device__ __forceinline__ void load_tile(bf16* tile, const bf16* src, size_t ld, int row0, int nrows, int S) {
-  for (int i = threadIdx.x; i < nrows * 8; i += THREADS) {
+  for (int i = threadIdx.x; i < nrows * 8; i += NT) {
     const int r = i >> 3, ch = i & 7;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (row0 + r < S) v = *reinterpret_cast<const uint4*>(src + (size_t)(row0 + r) * ld + ch * 8);
@@ -71,9 +74,9 @@ __device__ __forceinline__ void store16(bf16* dst, const float* src) {
 
 // Sf[RBT][ldsf] = A[RBT][64] * Bt[SP][64]^T (fp32).  A warp keeps its row tile's four A fragments and
 // walks over column tiles two at a time (two independent accumulator chains).
-template <int RBT>
+template <int RBT, int NW = WARPS>
 __device__ __forceinline__ void abt_tiles(const bf16* A, const bf16* Bt, float* Sf, int ntn, int ldsf, int warp) {
-  constexpr int MT = RBT / 16, G = WARPS / MT;
+  constexpr int MT = RBT / 16, G = NW / MT;
   const int mi = warp % MT, g = warp / MT;
   FragA a[DH / 16];
 #pragma unroll
@@ -98,13 +101,14 @@ __device__ __forceinline__ void abt_tiles(const bf16* A, const bf16* Bt, float* 
 }
 // Of[RBT][ldsf] (columns 0..63) = A[RBT][SP] * Bm[SP][64], A bf16 with stride lda.  64 rows: two column
 // tiles per warp sharing the A fragment; 32 rows: one tile per warp, even and odd k steps in two chains.
-template <int RBT>
+template <int RBT, int NW = WARPS>
 __device__ __forceinline__ void rows_times_head(const bf16* A, int lda, const bf16* Bm, float* Of, int ntn, int ldsf,
                                                 int warp) {
   FragC acc0, acc1;
   nvcuda::wmma::fill_fragment(acc0, 0.0f);
   nvcuda::wmma::fill_fragment(acc1, 0.0f);
-  if constexpr (RBT == 64) {
+  constexpr int MT = RBT / 16;
+  if constexpr (MT * 4 == 2 * NW) {
     const int mi = warp & 3, nj = (warp >> 2) * 2;
     for (int kk = 0; kk < ntn; ++kk) {
       FragA a;
@@ -118,8 +122,8 @@ __device__ __forceinline__ void rows_times_head(const bf16* A, int lda, const bf
     nvcuda::wmma::store_matrix_sync(Of + mi * 16 * ldsf + nj * 16, acc0, ldsf, nvcuda::wmma::mem_row_major);
     nvcuda::wmma::store_matrix_sync(Of + mi * 16 * ldsf + nj * 16 + 16, acc1, ldsf, nvcuda::wmma::mem_row_major);
   } else {
-    static_assert(RBT == 32, "row block");
-    const int mi = warp & 1, nj = warp >> 1;
+    static_assert(MT * 4 == NW, "one output tile per warp");
+    const int mi = warp % MT, nj = warp / MT;
     for (int kk = 0; kk < ntn; kk += 2) {
       FragA a0, a1;
       FragB b0, b1;
@@ -200,11 +204,14 @@ attn_forward_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float*
 }
 
 // dqkv: [M][3d] gradient of the layer's input; every element of this head's columns is written.
-static __global__ void __launch_bounds__(THREADS)
+// 16 warps: the row-wise passes use 8 lanes per row, every GEMM helper runs with 16 warps.
+static __global__ void __launch_bounds__(THREADS_BWD, 1)
 attn_backward_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out, const bf16* __restrict__ dout,
                      const float* __restrict__ lse, bf16* __restrict__ dqkv, int S, int H, int d) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ float Dsm[RB];
+  constexpr int NT = THREADS_BWD, NW = WARPS_BWD;
+  constexpr int TPR = NT / RB;                      // lanes per row in the row-wise passes: 8
   const int SP = pad16(S), ntn = SP / 16, ldsf = score_ld(SP), ldp = SP + 8;
   bf16* Ks = reinterpret_cast<bf16*>(smem);
   bf16* Vs = Ks + SP * LDK;
@@ -215,14 +222,14 @@ attn_backward_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out,
   bf16* dSb = Pb + RB * ldp;
   const int b = blockIdx.x / H, h = blockIdx.x - b * H;
   const int warp = threadIdx.x >> 5;
+  const int r = threadIdx.x / TPR, sub = threadIdx.x % TPR;       // row and lane-in-row of the row-wise passes
   const size_t ld = (size_t)3 * d;
   const bf16* base = qkv + (size_t)b * S * ld + h * DH;
   bf16* gbase = dqkv + (size_t)b * S * ld + h * DH;
   const bf16* obase = out + (size_t)b * S * d + h * DH;
   const bf16* dobase = dout + (size_t)b * S * d + h * DH;
-  load_tile(Ks, base + d, ld, 0, SP, S);
-  load_tile(Vs, base + 2 * d, ld, 0, SP, S);
-  const int own_tiles = ntn * (DH / 16);            // output tiles of dK (and of dV): [SP][64]
+  load_tile<NT>(Ks, base + d, ld, 0, SP, S);
+  load_tile<NT>(Vs, base + 2 * d, ld, 0, SP, S);
   FragC accK[MAX_OWN], accV[MAX_OWN];
 #pragma unroll
   for (int i = 0; i < MAX_OWN; ++i) {
@@ -230,89 +237,97 @@ attn_backward_kernel(const bf16* __restrict__ qkv, const bf16* __restrict__ out,
     nvcuda::wmma::fill_fragment(accV[i], 0.0f);
   }
   for (int rb0 = 0; rb0 < S; rb0 += RB) {
-    load_tile(Qs, base, ld, rb0, RB, S);
-    load_tile(dOs, dobase, (size_t)d, rb0, RB, S);
+    const bool valid = rb0 + r < S;
+    load_tile<NT>(Qs, base, ld, rb0, RB, S);
+    load_tile<NT>(dOs, dobase, (size_t)d, rb0, RB, S);
     __syncthreads();
-    abt_tiles<RB>(Qs, Ks, Sf, ntn, ldsf, warp);
-    {   // D_r = dO_r . o_r
-      const int r = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * 16;
+    abt_tiles<RB, NW>(Qs, Ks, Sf, ntn, ldsf, warp);
+    {   // D_r = dO_r . o_r, 8 columns per lane
       float s = 0.0f;
-      if (rb0 + r < S) {
-        const bf16* o = obase + (size_t)(rb0 + r) * d + c0;
+      if (valid) {
+        float ov[8], gv[8];
+        load_seg<8>(obase + (size_t)(rb0 + r) * d + sub * 8, 8, ov);
+        load_seg<8>(dOs + r * LDK + sub * 8, 8, gv);
 #pragma unroll
-        for (int c = 0; c < 16; ++c) s = fmaf(__bfloat162float(dOs[r * LDK + c0 + c]), __bfloat162float(o[c]), s);
+        for (int c = 0; c < 8; ++c) s = fmaf(gv[c], ov[c], s);
       }
-      s += __shfl_xor_sync(0xffffffffu, s, 1);
-      s += __shfl_xor_sync(0xffffffffu, s, 2);
-      if ((threadIdx.x & 3) == 0) Dsm[r] = s;
+#pragma unroll
+      for (int o = 1; o < TPR; o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (sub == 0) Dsm[r] = s;
     }
     __syncthreads();
     {   // P = exp(s / 8 - logsumexp), zero outside the sequence
-      const int r = threadIdx.x >> 2, sub = threadIdx.x & 3;
-      const bool valid = rb0 + r < S;
       const float l = valid ? lse[(size_t)blockIdx.x * S + rb0 + r] : 0.0f;
       const float* row = Sf + r * ldsf;
-      for (int c = sub; c < SP; c += 4)
-        Pb[r * ldp + c] = __float2bfloat16_rn((valid && c < S) ? __expf(row[c] * SCALE - l) : 0.0f);
+      for (int c = 2 * sub; c < SP; c += 2 * TPR) {  // two columns at a time
+        const float2 x = *reinterpret_cast<const float2*>(row + c);
+        const float p0 = (valid && c < S) ? __expf(x.x * SCALE - l) : 0.0f;
+        const float p1 = (valid && c + 1 < S) ? __expf(x.y * SCALE - l) : 0.0f;
+        *reinterpret_cast<uint32_t*>(Pb + r * ldp + c) = pack_bf16x2(p0, p1);
+      }
     }
     __syncthreads();
     // dP = dO V^T -> Sf
-    abt_tiles<RB>(dOs, Vs, Sf, ntn, ldsf, warp);
+    abt_tiles<RB, NW>(dOs, Vs, Sf, ntn, ldsf, warp);
     __syncthreads();
     {   // dS = P * (dP - D) / 8
-      const int r = threadIdx.x >> 2, sub = threadIdx.x & 3;
       const float Dr = Dsm[r];
       const float* row = Sf + r * ldsf;
-      for (int c = sub; c < SP; c += 4)
-        dSb[r * ldp + c] = __float2bfloat16_rn(__bfloat162float(Pb[r * ldp + c]) * (row[c] - Dr) * SCALE);
+      for (int c = 2 * sub; c < SP; c += 2 * TPR) {
+        const float2 x = *reinterpret_cast<const float2*>(row + c);
+        const uint32_t pp = *reinterpret_cast<const uint32_t*>(Pb + r * ldp + c);
+        const float p0 = __uint_as_float(pp << 16), p1 = __uint_as_float(pp & 0xffff0000u);
+        *reinterpret_cast<uint32_t*>(dSb + r * ldp + c) = pack_bf16x2(p0 * (x.x - Dr) * SCALE, p1 * (x.y - Dr) * SCALE);
+      }
     }
     __syncthreads();
     // dQ_blk = dS K -> Sf (columns 0..63)
-    rows_times_head<RB>(dSb, ldp, Ks, Sf, ntn, ldsf, warp);
-    // dV += P^T dO ; dK += dS^T Q   (contraction over the 64 rows of this block).  All of a warp's output
-    // tiles share their column tile nj, so the dO / Q fragments of a k step are loaded once.
+    rows_times_head<RB, NW>(dSb, ldp, Ks, Sf, ntn, ldsf, warp);
+    // dV^T += dO^T P ; dK^T += Q^T dS   (contraction over the 64 rows of this block).  Transposed so that
+    // the operand that has to be read column-wise is the small one: a warp's output tiles (64-row head
+    // tile mi = warp & 3, key tiles nj = warp / 4 + 4 i) share mi, so its four dO^T / Q^T fragments per
+    // block are loaded once, and P / dS are read row-wise.
     {
-      const int nj = warp & 3;
+      const int mi = warp & 3;
+      FragAT ot[RB / 16], qt[RB / 16];
 #pragma unroll
       for (int kk = 0; kk < RB / 16; ++kk) {
-        FragB bo, bq;
-        nvcuda::wmma::load_matrix_sync(bo, dOs + kk * 16 * LDK + nj * 16, LDK);
-        nvcuda::wmma::load_matrix_sync(bq, Qs + kk * 16 * LDK + nj * 16, LDK);
+        nvcuda::wmma::load_matrix_sync(ot[kk], dOs + kk * 16 * LDK + mi * 16, LDK);   // A[m][k] = dO[k][m]
+        nvcuda::wmma::load_matrix_sync(qt[kk], Qs + kk * 16 * LDK + mi * 16, LDK);
+      }
 #pragma unroll
-        for (int i = 0; i < MAX_OWN; ++i) {
-          const int t = warp + WARPS * i;
-          if (t < own_tiles) {
-            const int mj = t >> 2;
-            FragAT pt, st;
-            nvcuda::wmma::load_matrix_sync(pt, Pb + kk * 16 * ldp + mj * 16, ldp);     // A[m][k] = P[k][m]
-            nvcuda::wmma::load_matrix_sync(st, dSb + kk * 16 * ldp + mj * 16, ldp);
-            nvcuda::wmma::mma_sync(accV[i], pt, bo, accV[i]);
-            nvcuda::wmma::mma_sync(accK[i], st, bq, accK[i]);
+      for (int i = 0; i < MAX_OWN; ++i) {
+        const int nj = (warp >> 2) + (NW / 4) * i;
+        if (nj < ntn) {
+#pragma unroll
+          for (int kk = 0; kk < RB / 16; ++kk) {
+            FragB pb, sb;
+            nvcuda::wmma::load_matrix_sync(pb, Pb + kk * 16 * ldp + nj * 16, ldp);
+            nvcuda::wmma::load_matrix_sync(sb, dSb + kk * 16 * ldp + nj * 16, ldp);
+            nvcuda::wmma::mma_sync(accV[i], ot[kk], pb, accV[i]);
+            nvcuda::wmma::mma_sync(accK[i], qt[kk], sb, accK[i]);
           }
         }
       }
     }
     __syncthreads();
-    {
-      const int r = threadIdx.x >> 2, c0 = (threadIdx.x & 3) * 16;
-      if (rb0 + r < S) store16(gbase + (size_t)(rb0 + r) * ld + c0, Sf + r * ldsf + c0);
-    }
+    if (valid) store8(gbase + (size_t)(rb0 + r) * ld + sub * 8, Sf + r * ldsf + sub * 8);
     __syncthreads();
   }
-  // dK, then dV: accumulators -> fp32 staging [SP][64] (it fits the score buffer) -> bf16 rows
+  // dK, then dV: accumulators (transposed tiles) -> fp32 staging [SP][64] (it fits the score buffer) -> bf16 rows
   float* stage = Sf;
   for (int which = 0; which < 2; ++which) {
 #pragma unroll
     for (int i = 0; i < MAX_OWN; ++i) {
-      const int t = warp + WARPS * i;
-      if (t < own_tiles)
-        nvcuda::wmma::store_matrix_sync(stage + (t >> 2) * 16 * DH + (t & 3) * 16, which == 0 ? accK[i] : accV[i], DH,
-                                        nvcuda::wmma::mem_row_major);
+      const int nj = (warp >> 2) + (NW / 4) * i;
+      if (nj < ntn)
+        nvcuda::wmma::store_matrix_sync(stage + nj * 16 * DH + (warp & 3) * 16, which == 0 ? accK[i] : accV[i], DH,
+                                        nvcuda::wmma::mem_col_major);       // element (dh, key) -> stage[key][dh]
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < S * 4; i += THREADS) {
-      const int r = i >> 2, c0 = (i & 3) * 16;
-      store16(gbase + (size_t)r * ld + (which + 1) * d + c0, stage + r * DH + c0);
+    for (int i = threadIdx.x; i < S * 8; i += NT) {
+      const int row = i >> 3, c0 = (i & 7) * 8;
+      store8(gbase + (size_t)row * ld + (which + 1) * d + c0, stage + row * DH + c0);
     }
     __syncthreads();
   }

@@ -647,7 +647,7 @@ et_status run_attn_backward(et_stack* s, int l, const void* dY, cudaStream_t st)
   const size_t smem = et::attn::backward_smem_bytes(L.seq);
   ET_TRY(attn_allow_backward(smem));
   const int grid = (int)(s->M / L.seq) * L.heads;
-  et::attn::attn_backward_kernel<<<grid, et::attn::THREADS, smem, st>>>(
+  et::attn::attn_backward_kernel<<<grid, et::attn::THREADS_BWD, smem, st>>>(
       act_in<bf16>(s, l), (const bf16*)s->at(L.off_a_out), grad_act<bf16>(s, l + 1, dY), (const float*)s->at(L.off_lse),
       (bf16*)s->at(s->ly[l - 1].off_G_out), L.seq, L.heads, L.N);
   return after_launch();
