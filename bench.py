@@ -464,7 +464,7 @@ def run_side(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
     w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "full": wl.vit_b_full, "bottleneck": wl.resnet_bottleneck,
-         "schedule": wl.vit_l}[args.workload]()
+         "schedule": wl.vit_l, "schedule_full": wl.vit_l_full}[args.workload]()
     tdt = torch.bfloat16
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
     stack = et.et_stack_create(w.layers, w.M, w.dtype)
@@ -614,7 +614,7 @@ def run_side(args):
     el = loop.run(200, elastic=True, time_steps=True)
     T_full = t_fwd + t_dw.sum() + t_dy.sum()
     est = [t_fwd + et.et_time_selective(m, t_dw, t_dy) for m in el["masks"]]
-    print(json.dumps({"report": "vit_l_linear_bf16 elastic schedule, 200 iterations", "rho": 0.4,
+    print(json.dumps({"report": w.name + " elastic schedule, 200 iterations", "rho": 0.4,
                       "full_ms_per_step": full["ms_per_step"], "elastic_ms_per_step": el["ms_per_step"],
                       "ratio": el["ms_per_step"] / full["ms_per_step"],
                       "model_estimate_ratio": float(np.mean(est) / T_full),
@@ -636,7 +636,7 @@ def main():
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
-    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "bottleneck", "schedule", "selector"],
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "bottleneck", "schedule", "schedule_full", "selector"],
                     help="vit_b = the benchmark line; resnet / prenorm / schedule = side reports for the other shapes; "
                          "selector = host-side report on the selection dynamic program")
     args = ap.parse_args()

@@ -35,7 +35,9 @@ class ElasticLoop:
             self.master = [t for pair in zip(self.W32, self.b32) for t in pair]
         self.snap = [torch.empty_like(p) for p in (self.master or self.params)]
         self.imp = torch.zeros(2 * self.L, dtype=torch.float32, device=dev)
-        self.mask = np.ones(2 * self.L, dtype=np.uint8)
+        # layers without tensors (attention core, patch gather) hold empty slots that cannot be selected
+        self.all_mask = np.array([1 if p.numel() > 0 else 0 for p in self.params], dtype=np.uint8)
+        self.mask = self.all_mask.copy()
 
     def run(self, steps, elastic=True, time_steps=False):
         """Runs `steps` training steps.  elastic=False trains every tensor at every step (full
@@ -51,7 +53,7 @@ class ElasticLoop:
         for step in range(steps):
             phase = step % self.period
             if elastic and phase == 0:
-                self.mask = np.ones(2 * self.L, dtype=np.uint8)
+                self.mask = self.all_mask.copy()
                 for s_, p_ in zip(self.snap, self.master or self.params):
                     s_.copy_(p_)
             et.et_forward_stack(self.stack, self.x, self.y, stream=self.stream)
@@ -65,7 +67,9 @@ class ElasticLoop:
                 evaluations.append(S)
                 import time
                 t0 = time.perf_counter()
-                self.mask, _, _ = et.et_select_dp(-S, self.t_dw, self.t_dy, self.t_fwd, self.rho, self.Tq, self.variant)
+                self.mask, _, _ = et.et_select_dp(-S * self.all_mask, self.t_dw, self.t_dy, self.t_fwd, self.rho, self.Tq,
+                                                  self.variant)
+                self.mask = self.mask & self.all_mask
                 dp_ms.append(1e3 * (time.perf_counter() - t0))
             else:
                 et.et_backward_elastic(self.stack, self.dY, self.mask, None, None, None, flags, self.lr, None,
@@ -85,6 +89,12 @@ def flop_costs(layers, M):
     for when measured times are not wanted."""
     t_dw, t_dy = [], []
     for ly in layers:
+        if getattr(ly, "kind", 0) >= 2:
+            # a layer without tensors: its backward work, one pass over its rows here, is charged to the
+            # bias below it by the caller's cost vectors; as a stand-in its own slots cost nothing
+            t_dw += [0.0, 0.0]
+            t_dy += [0.0, 0.0]
+            continue
         if getattr(ly, "kind", 0) == 1:
             # normalisation layer: one pass over the rows, all of it charged to beta's error-gradient
             # time (Section 5.2)

@@ -274,6 +274,16 @@ def vit_l(seed: int = 3, params: bool = True, n_blocks: int = 24, tokens: int = 
     return _finish("vit_l_linear_bf16", layers, tokens, DT_BF16, 0.01, mask, rng, w_std=0.01, params=params)
 
 
+def vit_l_full(seed: int = 9, params: bool = True, n_blocks: int = 24, batch: int = 32, seq: int = 197,
+               d: int = 1024, ffn: int = 4096, heads: int = 16) -> Workload:
+    """bf16 ViT-L/16 with its normalisation layers and attention core; the mask starts with every
+    trainable tensor selected and is replaced by the selector while training."""
+    rng = np.random.default_rng(seed)
+    layers = vit_blocks_full(n_blocks, d, ffn, heads, seq)
+    mask = np.array([0 if ly.kind == KIND_ATTENTION else 1 for ly in layers for _ in (0, 1)], dtype=np.uint8)
+    return _finish("vit_l_full_bf16", layers, batch * seq, DT_BF16, 0.01, mask, rng, w_std=0.02, params=params)
+
+
 def resnet_1x1(seed: int = 2, p_select: float = 0.5, n_blocks: int = 6, tokens: int = 32 * 14 * 14,
                params: bool = True) -> Workload:
     """bf16 ResNet-50 conv4_x 1x1 bottleneck convs as NHWC GEMMs:
