@@ -98,3 +98,60 @@ def test_selector_on_measured_costs_bf16():
         if mask.any():
             w.mask = mask
             h.check_step(w, mask, 2e-2)
+
+
+def _trainable(layers):
+    return np.array([0 if ly.kind in (wl.KIND_ATTENTION, wl.KIND_IM2COL) else 1 for ly in layers for _ in (0, 1)], dtype=bool)
+
+
+def test_schedule_with_normalisation_layers_fp32_matches_oracle_trajectory():
+    import gpu_harness as h
+    # the pre-norm twin: gamma and beta take part in the selection like any other tensor
+    layers = wl.vit_blocks_prenorm(4, 64, 256)
+    w = wl.small_stack(layers, 197, wl.DT_F32, 18, w_std=0.05)
+    steps, period, window, rho, Tq = 60, 30, 6, 0.4, 300
+    t_dw, t_dy = flop_costs(w.layers, w.M)
+    ref = orc.train_schedule(w.layers, w.W, w.b, w.x, w.target, w.lr, steps, period, window, rho, t_dw, t_dy, Tq=Tq)
+    run = h.GpuRun(w)
+    loop = ElasticLoop(run.stack, run.W, run.b, run.x, run.target, w.lr, period, window, rho, t_dw, t_dy, Tq=Tq)
+    got = loop.run(steps)
+    assert et.et_device_status(run.stack) == et.ET_OK
+    for S_gpu, S_ref in zip(got["importances"], ref["importances"]):
+        assert np.abs(S_gpu - S_ref).max() <= 2e-3 * np.abs(S_ref).max()
+    np.testing.assert_allclose(got["losses"], ref["losses"], rtol=2e-3)
+    assert got["losses"][-1] < got["losses"][0]
+    qw, qy, budget = orc.quantise(t_dw, t_dy, 0.0, rho, Tq)
+    for step in range(steps):
+        m_gpu, m_ref = got["masks"][step], ref["masks"][step]
+        if not np.array_equal(m_gpu, m_ref):
+            I = -ref["importances"][step // period]
+            assert orc.t_selective(m_gpu, qw, qy) <= budget
+            assert abs(I[m_gpu.astype(bool)].sum() - I[m_ref.astype(bool)].sum()) <= 1e-3 * abs(I[m_ref.astype(bool)].sum())
+    final = orc.tensors_of(ref["W"], ref["b"])
+    for t, p in enumerate(run.params()):
+        assert np.abs(h.to_np(p) - final[t]).max() <= 1e-3
+
+
+def test_schedule_full_transformer_blocks_bf16_with_master_weights():
+    import gpu_harness as h
+    # normalisation layers and the attention core in the stack; layers without tensors never enter a mask
+    layers = wl.vit_blocks_full(2, 128, 256, heads=2, seq=49)
+    w = wl.small_stack(layers, 8 * 49, wl.DT_BF16, 24, w_std=0.05)
+    live = _trainable(layers)
+    steps, period, window, rho, Tq = 60, 30, 6, 0.5, 300
+    t_dw, t_dy = flop_costs(w.layers, w.M)
+    ref = orc.train_schedule(w.layers, w.W, w.b, w.x, w.target, w.lr, steps, period, window, rho, t_dw, t_dy, Tq=Tq)
+    run = h.GpuRun(w)
+    loop = ElasticLoop(run.stack, run.W, run.b, run.x, run.target, w.lr, period, window, rho, t_dw, t_dy, Tq=Tq,
+                       master=True)
+    got = loop.run(steps)
+    assert et.et_device_status(run.stack) == et.ET_OK
+    assert all(not m[~live].any() for m in got["masks"])
+    np.testing.assert_allclose(got["losses"], ref["losses"], rtol=2e-2)
+    assert got["losses"][-1] < got["losses"][0]
+    for S_gpu, S_ref in zip(got["importances"], ref["importances"]):
+        assert np.abs(S_gpu - S_ref)[live].max() <= 5e-2 * np.abs(S_ref).max()
+    final = orc.tensors_of(ref["W"], ref["b"])
+    for t, p in enumerate(loop.master):
+        if live[t]:
+            assert np.abs(h.to_np(p) - final[t]).max() <= 2e-3
