@@ -75,68 +75,76 @@ __device__ __forceinline__ void lds8(const float* p, float (&t)[8]) {
 // would spill, and such rows are long enough to keep the memory system busy on their own.
 template <typename T, int VPL> struct NormPrefetch { static constexpr bool value = VPL * (int)sizeof(T) <= 8; };
 
+// Rows a warp loads at once in the forward kernel.  With one resident wave a warp owns only two or three
+// rows: taking their loads one after the other would make the kernel a chain of that many memory
+// latencies, so they are all requested up front (12 packed registers per 768-wide bf16 row).
+template <typename T, int VPL> struct NormBatch { static constexpr int value = VPL * (int)sizeof(T) <= 6 ? 3 : 1; };
+
 template <typename T, int VPL>
-__global__ void __launch_bounds__(kNormThreads)
+__global__ void __launch_bounds__(kNormThreads, VPL <= 3 ? 6 : 1)
 norm_forward_kernel(const T* __restrict__ x, const T* __restrict__ gamma, const T* __restrict__ beta,
                     T* __restrict__ y, float2* __restrict__ stats, int M, int d, float eps) {
   __shared__ __align__(16) float s_gamma[VPL * 256], s_beta[VPL * 256];
-  constexpr bool PRE = NormPrefetch<T, VPL>::value;
+  constexpr int R = NormBatch<T, VPL>::value;
   const int lane = threadIdx.x & 31;
   const int warp = blockIdx.x * kNormWarps + (threadIdx.x >> 5);
   const int nwarps = gridDim.x * kNormWarps;
+  const float inv_d = 1.0f / (float)d;
+  RawChunk<T> raw[R][VPL];
+  auto fetch = [&](int r0) {
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+      const int r = r0 + j * nwarps;
+      if (r < M) norm_load_raw<T, VPL>(x + (size_t)r * d, d, lane, raw[j]);
+    }
+  };
+  fetch(warp);                                     // the first batch is on its way before anything else
   stage_vector<T, VPL>(gamma, d, s_gamma);
   stage_vector<T, VPL>(beta, d, s_beta);
   __syncthreads();
-  const float inv_d = 1.0f / (float)d;
-  const size_t step = (size_t)nwarps * d;
-  const T* xp = x + (size_t)warp * d;
-  T* yp = y + (size_t)warp * d;
-  RawChunk<T> nxt[VPL];
-  if (PRE && warp < M) norm_load_raw<T, VPL>(xp, d, lane, nxt);
-  for (int r = warp; r < M; r += nwarps, xp += step, yp += step) {
-    RawChunk<T> raw[VPL];
-    if constexpr (PRE) {
+  for (int r0 = warp; r0 < M; r0 += R * nwarps) {
+    if (r0 != warp) fetch(r0);
 #pragma unroll
-      for (int c = 0; c < VPL; ++c) raw[c] = nxt[c];
-      if (r + nwarps < M) norm_load_raw<T, VPL>(xp + step, d, lane, nxt);
-    } else {
-      norm_load_raw<T, VPL>(xp, d, lane, raw);
-    }
-    float v[VPL * 8];
-    float s = 0.0f;
+    for (int j = 0; j < R; ++j) {
+      const int r = r0 + j * nwarps;
+      if (r >= M) break;
+      float v[VPL * 8];
+      float s = 0.0f;
 #pragma unroll
-    for (int c = 0; c < VPL; ++c) {
-      float t[8];
-      raw_unpack(raw[c], t);
+      for (int c = 0; c < VPL; ++c) {
+        float t[8];
+        raw_unpack(raw[j][c], t);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) { v[c * 8 + e] = t[e]; s += t[e]; }
-    }
-    const float mean = warp_sum(s) * inv_d;
-    float q = 0.0f;
-#pragma unroll
-    for (int c = 0; c < VPL; ++c) {
-      const bool in = (c * 32 + lane) * 8 < d;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float t = v[c * 8 + e] - mean;
-        q += in ? t * t : 0.0f;
+        for (int e = 0; e < 8; ++e) { v[c * 8 + e] = t[e]; s += t[e]; }
       }
-    }
-    const float rstd = rsqrtf(warp_sum(q) * inv_d + eps);
-    const float shift = -mean * rstd;
+      const float mean = warp_sum(s) * inv_d;
+      float q = 0.0f;
 #pragma unroll
-    for (int c = 0; c < VPL; ++c) {
-      const int col = (c * 32 + lane) * 8;
-      if (col < d) {
-        float g[8], b[8], o[8];
-        lds8(s_gamma + col, g);
-        lds8(s_beta + col, b);
+      for (int c = 0; c < VPL; ++c) {
+        const bool in = (c * 32 + lane) * 8 < d;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) o[e] = fmaf(fmaf(v[c * 8 + e], rstd, shift), g[e], b[e]);
-        store_chunk(yp + col, o);
+        for (int e = 0; e < 8; ++e) {
+          const float t = v[c * 8 + e] - mean;
+          q += in ? t * t : 0.0f;
+        }
       }
+      const float rstd = rsqrtf(warp_sum(q) * inv_d + eps);
+      const float shift = -mean * rstd;
+      T* yp = y + (size_t)r * d;
+#pragma unroll
+      for (int c = 0; c < VPL; ++c) {
+        const int col = (c * 32 + lane) * 8;
+        if (col < d) {
+          float g[8], b[8], o[8];
+          lds8(s_gamma + col, g);
+          lds8(s_beta + col, b);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) o[e] = fmaf(fmaf(v[c * 8 + e], rstd, shift), g[e], b[e]);
+          store_chunk(yp + col, o);
+        }
+      }
+      if (lane == 0) stats[r] = make_float2(mean, rstd);
     }
-    if (lane == 0) stats[r] = make_float2(mean, rstd);
   }
 }
 
