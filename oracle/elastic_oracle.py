@@ -18,6 +18,11 @@ or, for a normalisation layer (Section 5.2; its Gamma and Beta are tensors 2*l a
     xhat    = (a_l - mean) / sqrt(var + eps)         mean, var over the features of each row
     a_{l+1} = xhat * gamma_l + beta_l
 
+or, for a batch normalisation layer (Section 5.2's subject; training mode, no running averages),
+
+    xhat    = (a_l - mean) / sqrt(var + eps)         mean, biased var of each feature over all rows
+    a_{l+1} = act_l( xhat * gamma_l + beta_l )
+
 or, for a patch-gather layer (no trainable tensors; with the dense layer after it, it is a k x k
 convolution with stride 1 and zero padding k // 2 on NHWC rows, the convolutional layer of Section 5.1),
 
@@ -46,7 +51,7 @@ from typing import Dict, List, Optional, Sequence
 import numpy as np
 
 ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
-KIND_DENSE, KIND_NORM, KIND_ATTENTION, KIND_IM2COL = 0, 1, 2, 3
+KIND_DENSE, KIND_NORM, KIND_ATTENTION, KIND_IM2COL, KIND_BATCHNORM = 0, 1, 2, 3, 4
 STRICT, INCLUSIVE = 0, 1
 
 
@@ -95,6 +100,17 @@ def forward(layers, W: Sequence[np.ndarray], b: Sequence[np.ndarray], x: np.ndar
     a = [np.asarray(x, dtype=np.float64)]
     Z = []
     for l, ly in enumerate(layers):
+        if _kind(ly) == KIND_BATCHNORM:
+            # batch normalisation, training mode: mean and biased variance of each feature over all rows;
+            # Z keeps (xhat, 1/sqrt(var + eps), pre-activation)
+            mean = a[l].mean(axis=0, keepdims=True)
+            var = ((a[l] - mean) ** 2).mean(axis=0, keepdims=True)
+            rstd = 1.0 / np.sqrt(var + ly.eps)
+            xhat = (a[l] - mean) * rstd
+            z = xhat * np.asarray(W[l], dtype=np.float64) + np.asarray(b[l], dtype=np.float64)
+            Z.append((xhat, rstd, z))
+            a.append(act_forward(z, ly.act))
+            continue
         if _kind(ly) == KIND_IM2COL:
             # patch gather of a k x k convolution, stride 1, zero padding k // 2, on NHWC rows:
             # col[(n,h,w), (kh*k + kw)*C + c] = x[n, h + kh - p, w + kw - p, c]  (0 outside the image)
@@ -203,6 +219,19 @@ def _backward_sweep(layers, W, saved: Saved, dY: np.ndarray, stop: int,
     for l in range(L - 1, stop - 1, -1):
         ly = layers[l]
         g_out = G[l + 1]
+        if _kind(ly) == KIND_BATCHNORM:
+            xhat, rstd, z = saved.Z[l]
+            dz = g_out * act_derivative(z, ly.act)
+            if want_w[l]:
+                grads[2 * l] = (dz * xhat).sum(axis=0)              # d gamma
+            if want_b[l]:
+                grads[2 * l + 1] = dz.sum(axis=0)                   # d beta
+            if l > stop:
+                # as for the row-wise normalisation, with the means taken over the rows of each column
+                gy = dz * np.asarray(W[l], dtype=np.float64)
+                dX = rstd * (gy - gy.mean(axis=0, keepdims=True) - xhat * (gy * xhat).mean(axis=0, keepdims=True))
+                G[l] = dX if G[l] is None else G[l] + dX
+            continue
         if _kind(ly) == KIND_IM2COL:
             if want_w[l]:
                 grads[2 * l] = np.zeros(0)

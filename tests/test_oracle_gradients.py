@@ -47,6 +47,9 @@ def _fd_check(layers, M, seed, h=1e-6, tol=2e-6):
                 lm = _loss(w.layers, w.W, w.b, w.x, w.target)
                 p[idx] = old
                 fd = (lp - lm) / (2 * h)
+                if np.abs(g).max() < 1e-12:          # a gradient that is identically zero (a bias right before a
+                    assert abs(fd) < 1e-7           # normalisation over the same axis): the difference quotient is noise
+                    continue
                 scale = max(abs(fd), np.abs(g).max() * 1e-3, 1e-12)
                 assert abs(fd - g[idx]) / scale < tol, (l, t, idx, fd, g[idx])
 
@@ -371,3 +374,54 @@ def test_patch_gather_closed_forms():
     corner = np.zeros((9, 1)); corner[0] = 1.0
     col = orc.forward(g, [np.zeros(0)], [np.zeros(0)], corner).a[-1]
     assert col.sum() == 4 and col[0, 4] == 1 and col[1, 3] == 1 and col[3, 1] == 1 and col[4, 0] == 1
+
+
+# ------------------------------------------------------------------ batch normalisation (Section 5.2)
+def test_batchnorm_matches_the_library_batch_norm():
+    torch = pytest.importorskip("torch")
+    F = torch.nn.functional
+    layers = [wl.Layer(5, 8), wl.batchnorm_layer(8, wl.ACT_RELU, eps=1e-5), wl.Layer(8, 6, act=wl.ACT_GELU_TANH),
+              wl.batchnorm_layer(6, eps=1e-2), wl.Layer(6, 4)]
+    w = wl.small_stack(layers, 9, wl.DT_F32, 71, w_std=0.5, bias_std=0.2)
+    saved = orc.forward(w.layers, w.W, w.b, w.x)
+    _, dY = orc.mse_loss_grad(saved.a[-1], w.target)
+    grads = orc.backward_full(w.layers, w.W, saved, dY)
+    tW = [torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in w.W]
+    tb = [torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in w.b]
+    h = torch.tensor(w.x, dtype=torch.float64)
+    for l, ly in enumerate(layers):
+        if ly.kind == wl.KIND_BATCHNORM:
+            h = F.batch_norm(h, None, None, tW[l], tb[l], training=True, eps=ly.eps)
+        else:
+            h = h @ tW[l] + tb[l]
+        if ly.act == wl.ACT_RELU:
+            h = torch.relu(h)
+        elif ly.act == wl.ACT_GELU_TANH:
+            h = F.gelu(h, approximate="tanh")
+    loss = ((h - torch.tensor(w.target, dtype=torch.float64)) ** 2).mean()
+    loss.backward()
+    assert abs(loss.item() - orc.mse_loss(saved.a[-1], w.target)) < 1e-13
+    for l in range(len(layers)):
+        assert np.allclose(grads[2 * l], tW[l].grad.numpy(), rtol=1e-8, atol=1e-13), l
+        assert np.allclose(grads[2 * l + 1], tb[l].grad.numpy(), rtol=1e-8, atol=1e-13), l
+
+
+def test_finite_differences_through_batchnorm():
+    layers = [wl.Layer(4, 6), wl.batchnorm_layer(6, wl.ACT_GELU_TANH), wl.Layer(6, 6, residual_src=2),
+              wl.batchnorm_layer(6, eps=1e-3), wl.Layer(6, 3)]
+    _fd_check(layers, M=7, seed=72, tol=5e-6)
+    _fd_check(wl.resnet_bottleneck_blocks(1, 8, 4, 3, 3, bn=True), M=18, seed=73, tol=5e-6)
+
+
+def test_batchnorm_closed_forms():
+    # every column of xhat has mean 0 and second moment var / (var + eps) over the rows; a per-column shift
+    # and scale of the input (eps = 0) leaves the output unchanged; two rows give xhat = +-1
+    rng = np.random.default_rng(5)
+    x = rng.normal(size=(11, 4)) * 3.0 + 2.0
+    ly = [wl.batchnorm_layer(4, eps=0.0)]
+    one, zero = np.ones(4), np.zeros(4)
+    xh = orc.forward(ly, [one], [zero], x).a[-1]
+    assert np.allclose(xh.mean(axis=0), 0.0, atol=1e-14) and np.allclose((xh ** 2).mean(axis=0), 1.0, atol=1e-13)
+    assert np.allclose(orc.forward(ly, [one], [zero], x * np.array([2.0, 0.5, 7.0, 1.0]) + 3.0).a[-1], xh, atol=1e-12)
+    two = orc.forward(ly, [np.array([2.0, 3.0, 4.0, 5.0])], [np.array([1.0, 1.0, 1.0, 1.0])], np.array([[1.0, 5, 2, 0], [3.0, 1, 8, 4]])).a[-1]
+    assert np.allclose(two, [[-1.0, 4.0, -3.0, -4.0], [3.0, -2.0, 5.0, 6.0]])

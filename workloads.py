@@ -27,7 +27,9 @@ ACT_NONE, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
 DT_F32, DT_BF16 = 0, 1
 # layer kinds: a dense layer (kernel, bias) or a layer normalisation over the feature axis, whose two
 # trainable tensors gamma and beta take the kernel and bias slots (Section 5.2: Gamma and Beta)
-KIND_DENSE, KIND_NORM, KIND_ATTENTION, KIND_IM2COL = 0, 1, 2, 3
+KIND_DENSE, KIND_NORM, KIND_ATTENTION, KIND_IM2COL, KIND_BATCHNORM = 0, 1, 2, 3, 4
+# KIND_BATCHNORM: batch normalisation in training mode (statistics of each feature over all rows), optional
+# activation after it; Gamma and Beta in the kernel and bias slots like KIND_NORM (Section 5.2)
 # KIND_IM2COL: the patch-gathering half of a k x k convolution (stride 1, zero padding k // 2) on NHWC
 # rows; followed by a dense layer with in_features = k * k * channels it is that convolution.  No tensors.
 # KIND_ATTENTION: the softmax attention core, a layer without trainable tensors (Section 5.3 / 5.4:
@@ -132,6 +134,10 @@ def norm_layer(d: int, eps: float = 1e-5) -> Layer:
     return Layer(d, d, kind=KIND_NORM, eps=eps)
 
 
+def batchnorm_layer(d: int, act: int = ACT_NONE, eps: float = 1e-5) -> Layer:
+    return Layer(d, d, act=act, kind=KIND_BATCHNORM, eps=eps)
+
+
 def attention_layer(d: int, heads: int, seq: int) -> Layer:
     return Layer(3 * d, d, kind=KIND_ATTENTION, heads=heads, seq=seq)
 
@@ -161,13 +167,18 @@ def conv_layers(c_in: int, c_out: int, height: int, width: int, ksize: int = 3, 
             Layer(ksize * ksize * c_in, c_out, act=act, residual_src=residual_src)]
 
 
-def resnet_bottleneck_blocks(n_blocks: int, c: int, mid: int, height: int, width: int) -> List[Layer]:
-    """ResNet bottleneck: 1x1 c->mid ReLU, 3x3 mid->mid ReLU, 1x1 mid->c + block input (4 layers)."""
+def resnet_bottleneck_blocks(n_blocks: int, c: int, mid: int, height: int, width: int, bn: bool = False) -> List[Layer]:
+    """ResNet bottleneck: 1x1 c->mid ReLU, 3x3 mid->mid ReLU, 1x1 mid->c + block input (4 layers);
+    bn=True puts a batch normalisation between each convolution and its ReLU (7 layers)."""
     layers: List[Layer] = []
     for blk in range(n_blocks):
-        base = 4 * blk
-        layers.append(Layer(c, mid, act=ACT_RELU))
-        layers += conv_layers(mid, mid, height, width, 3, act=ACT_RELU)
+        base = (7 if bn else 4) * blk
+        if bn:
+            layers += [Layer(c, mid), batchnorm_layer(mid, ACT_RELU)]
+            layers += conv_layers(mid, mid, height, width, 3) + [batchnorm_layer(mid, ACT_RELU)]
+        else:
+            layers.append(Layer(c, mid, act=ACT_RELU))
+            layers += conv_layers(mid, mid, height, width, 3, act=ACT_RELU)
         layers.append(Layer(mid, c, residual_src=base))
     return layers
 
@@ -195,7 +206,7 @@ def _draw_params(rng, layers, dtype, w_std=None, he_init=False):
         if ly.kind in (KIND_ATTENTION, KIND_IM2COL):
             W.append(np.zeros(0)); b.append(np.zeros(0))
             continue
-        if ly.kind == KIND_NORM:
+        if ly.kind in (KIND_NORM, KIND_BATCHNORM):
             W.append(_store(1.0 + rng.normal(0.0, 0.1, size=ly.out_features), dtype))     # gamma
             b.append(_store(rng.normal(0.0, 0.1, size=ly.out_features), dtype))           # beta
             continue
@@ -296,10 +307,11 @@ def resnet_1x1(seed: int = 2, p_select: float = 0.5, n_blocks: int = 6, tokens: 
 
 
 def resnet_bottleneck(seed: int = 6, p_select: float = 0.5, n_blocks: int = 6, images: int = 32, height: int = 14,
-                      width: int = 14, c: int = 1024, mid: int = 256, params: bool = True) -> Workload:
-    """bf16 ResNet-50 conv4_x bottlenecks with their 3x3 convolutions (NHWC rows)."""
+                      width: int = 14, c: int = 1024, mid: int = 256, params: bool = True, bn: bool = False) -> Workload:
+    """bf16 ResNet-50 conv4_x bottlenecks with their 3x3 convolutions (NHWC rows), optionally with their
+    batch normalisations."""
     rng = np.random.default_rng(seed)
-    layers = resnet_bottleneck_blocks(n_blocks, c, mid, height, width)
+    layers = resnet_bottleneck_blocks(n_blocks, c, mid, height, width, bn)
     mask = bernoulli_weight_mask(rng, len(layers), p_select)
     for l, ly in enumerate(layers):
         if ly.kind == KIND_IM2COL:
@@ -344,7 +356,7 @@ def draw_delta(w: Workload, seed: int, std: float = 1e-3):
         if ly.kind in (KIND_ATTENTION, KIND_IM2COL):
             out += [np.zeros(0), np.zeros(0)]
             continue
-        shape = (ly.out_features,) if ly.kind == KIND_NORM else (ly.in_features, ly.out_features)
+        shape = (ly.out_features,) if ly.kind in (KIND_NORM, KIND_BATCHNORM) else (ly.in_features, ly.out_features)
         out.append(_store(rng.normal(0.0, std, size=shape), w.dtype))
         out.append(_store(rng.normal(0.0, std, size=ly.out_features), w.dtype))
     return out
