@@ -464,6 +464,7 @@ def run_side(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
     w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "full": wl.vit_b_full, "bottleneck": wl.resnet_bottleneck,
+         "bottleneck_bn": lambda: wl.resnet_bottleneck(bn=True),
          "schedule": wl.vit_l, "schedule_full": wl.vit_l_full}[args.workload]()
     tdt = torch.bfloat16
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
@@ -477,7 +478,7 @@ def run_side(args):
     et.et_forward_stack(stack, x, y)
     et.et_loss_mse_grad(stack, y, target, dY, None)
     torch.cuda.synchronize()
-    if args.workload in ("resnet", "prenorm", "full", "bottleneck"):
+    if args.workload in ("resnet", "prenorm", "full", "bottleneck", "bottleneck_bn"):
         rep = et.Report(w.L)
         all_trainable = np.ones(2 * w.L, dtype=np.uint8)
         for l, ly in enumerate(w.layers):
@@ -528,7 +529,7 @@ def run_side(args):
             gms = gfms = None
             print("graph capture failed:", exc, file=sys.stderr)
         extra = {}
-        if args.workload == "bottleneck":
+        if args.workload in ("bottleneck", "bottleneck_bn"):
             # the gather kernels alone: forward writes k*k times the activation, backward reads as much
             et.et_timing_enable(stack, True)
             for _ in range(5):
@@ -542,7 +543,8 @@ def run_side(args):
             extra = {"gather_ms_per_forward_plus_backward": gather_ms, "gather_launches": t["attention"][1] / 5,
                      "gather_gbs": nbytes / gather_ms / 1e6,
                      "gather_frac_of_hbm_peak": nbytes / gather_ms / 1e6 / _peaks()["hbm_gbs"],
-                     "dgrad_ms": t["dgrad"][0] / 5, "wgrad_ms": t["wgrad"][0] / 5, "forward_gemm_ms": t["forward"][0] / 5}
+                     "dgrad_ms": t["dgrad"][0] / 5, "wgrad_ms": t["wgrad"][0] / 5, "forward_gemm_ms": t["forward"][0] / 5,
+                     "norm_ms_per_forward_plus_backward": t["norm"][0] / 5, "norm_timed_regions": t["norm"][1] / 5}
         if args.workload == "full":
             # the attention kernels alone, over full-backprop steps: 4 S^2 64 flops per (sequence, head)
             # forward, 2.5 times that backward (five GEMMs, one of them the recomputed scores)
@@ -636,7 +638,7 @@ def main():
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
-    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "bottleneck", "schedule", "schedule_full", "selector"],
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "bottleneck", "bottleneck_bn", "schedule", "schedule_full", "selector"],
                     help="vit_b = the benchmark line; resnet / prenorm / schedule = side reports for the other shapes; "
                          "selector = host-side report on the selection dynamic program")
     args = ap.parse_args()

@@ -29,6 +29,13 @@
  *   slots in gradient / importance / state arrays are ignored.  Its backward (above the deepest
  *   selected layer only) recomputes P from the saved per-row log-sum-exp.
  *
+ *   A layer of kind ET_LAYER_BATCHNORM is a batch normalisation in training mode, the layer Section 5.2
+ *   is written about: like ET_LAYER_NORM with the mean and the biased variance of each feature taken
+ *   over all M rows instead of over each row's features, no running averages, followed by act_l:
+ *       a_{l+1} = act_l( (a_l - mean_c) / sqrt(var_c + eps) * gamma_l + beta_l )
+ *   in_features == out_features (a multiple of 8), fold = 1, residual_src = -1; gamma and beta are
+ *   tensors 2l and 2l+1 and are costed by the same black-box rule.
+ *
  *   A layer of kind ET_LAYER_IM2COL gathers the k x k patches of a convolution (stride 1, zero
  *   padding k / 2) from NHWC rows:  a_{l+1}[(n,h,w), (kh*k + kw)*C + c] = a_l[(n, h+kh-k/2, w+kw-k/2), c].
  *   Followed by a dense layer with in_features = k*k*C it is the convolutional layer of Section 5.1
@@ -86,7 +93,9 @@ typedef enum {
 
 typedef enum { ET_F32 = 0, ET_BF16 = 1 } et_dtype;
 typedef enum { ET_ACT_NONE = 0, ET_ACT_GELU_TANH = 1, ET_ACT_RELU = 2 } et_act;
-typedef enum { ET_LAYER_DENSE = 0, ET_LAYER_NORM = 1, ET_LAYER_ATTENTION = 2, ET_LAYER_IM2COL = 3 } et_layer_kind;
+typedef enum {
+  ET_LAYER_DENSE = 0, ET_LAYER_NORM = 1, ET_LAYER_ATTENTION = 2, ET_LAYER_IM2COL = 3, ET_LAYER_BATCHNORM = 4
+} et_layer_kind;
 
 /* Cost-model reading for the selector (Section 2.2 / Eq. 7 versus the example after Eq. 3). */
 typedef enum {

@@ -35,7 +35,7 @@ class et_layer_desc(C.Structure):
                 ("ksize", C.c_int32)]
 
 
-ET_LAYER_DENSE, ET_LAYER_NORM, ET_LAYER_ATTENTION, ET_LAYER_IM2COL = 0, 1, 2, 3
+ET_LAYER_DENSE, ET_LAYER_NORM, ET_LAYER_ATTENTION, ET_LAYER_IM2COL, ET_LAYER_BATCHNORM = 0, 1, 2, 3, 4
 
 
 class et_optimizer_config(C.Structure):

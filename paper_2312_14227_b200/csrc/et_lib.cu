@@ -20,6 +20,7 @@
 #include "norm.cuh"
 #include "attn.cuh"
 #include "im2col.cuh"
+#include "batchnorm.cuh"
 
 namespace {
 
@@ -152,8 +153,10 @@ struct LayerRT {
   bool pair_fwd = false, pair_dgrad = false, pair_wgrad = false;   // CTA-pair (cta_group::2) tiles
   int imp_count_w = 0, imp_count_b = 0;
   int img_h = 0, img_w = 0, ksize = 0;   // patch gather: K = channels, N = ksize^2 * K
-  bool trainable() const { return kind == ET_LAYER_DENSE || kind == ET_LAYER_NORM; }
-  size_t w_count() const { return !trainable() ? 0 : kind == ET_LAYER_NORM ? (size_t)N : (size_t)K * N; }   // elements of tensor 2l
+  bool trainable() const { return kind == ET_LAYER_DENSE || kind == ET_LAYER_NORM || kind == ET_LAYER_BATCHNORM; }
+  bool vector_params() const { return kind == ET_LAYER_NORM || kind == ET_LAYER_BATCHNORM; }   // gamma, beta: [N]
+  size_t off_means = 0;     // batch norm: the two column means of the backward formula
+  size_t w_count() const { return !trainable() ? 0 : vector_params() ? (size_t)N : (size_t)K * N; }   // elements of tensor 2l
   // bf16 stacks: one TMA descriptor per tensor (the caller's x, y and dY get theirs per call)
   TMaps map_W, map_aout, map_Gout, map_Z, map_dZ;
   CUtensorMap map_Wd;       // W as the K-major B of the dgrad GEMM: one box = the CTA's whole B tile
@@ -605,6 +608,73 @@ et_status run_norm_backward(et_stack* s, int l, const void* dY, bool want_dx, bo
   return after_launch();
 }
 
+// ---- batch normalisation -------------------------------------------------------------------
+template <typename T>
+et_status run_bn_forward(et_stack* s, int l, void* y, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_NORM, st);
+  const LayerRT& L = s->ly[l];
+  const int M = (int)s->M, C = L.N, chunks = L.norm_blocks;
+  const T* x = act_in<T>(s, l);
+  float* part = (float*)s->at(L.off_gpart);
+  float2* stats = (float2*)s->at(L.off_stats);
+  const dim3 grid(ceil_div(C, 256), chunks), block(32, 8);
+  const float inv_m = (float)(1.0 / (double)M);
+  et::bn_colstats_kernel<T, et::kBnSum><<<grid, block, 0, st>>>(x, nullptr, nullptr, M, C, part, nullptr);
+  ET_TRY(after_launch());
+  et::bn_finalize_kernel<<<ceil_div(C, 32), dim3(32, 32), 0, st>>>(part, nullptr, chunks, C, inv_m, L.eps, 0, stats, nullptr);
+  ET_TRY(after_launch());
+  et::bn_colstats_kernel<T, et::kBnCentredSquares><<<grid, block, 0, st>>>(x, nullptr, stats, M, C, part, nullptr);
+  ET_TRY(after_launch());
+  et::bn_finalize_kernel<<<ceil_div(C, 32), dim3(32, 32), 0, st>>>(part, nullptr, chunks, C, inv_m, L.eps, 1, stats, nullptr);
+  ET_TRY(after_launch());
+  T* out = l == s->L - 1 ? (T*)y : (T*)s->at(L.off_a_out);
+  const long long total = (long long)M * (C / 8);
+  et::bn_forward_kernel<T><<<ceil_div(total, et::kBnEltThreads), et::kBnEltThreads, 0, st>>>(
+      x, (const T*)L.W, (const T*)L.b, stats, L.act != ET_ACT_NONE ? (T*)s->at(L.off_Z) : nullptr, out, L.act, s->M, C);
+  return after_launch();
+}
+// Same contract as run_norm_backward.
+template <typename T>
+et_status run_bn_backward(et_stack* s, int l, const void* dY, bool want_dx, bool want_dgamma, float* grad,
+                          const T* delta, bool sgd, float lr, int* launches, cudaStream_t st) {
+  TimedLaunch tl(s, ET_K_NORM, st);
+  const LayerRT& L = s->ly[l];
+  if (!want_dx && !want_dgamma) return ET_OK;
+  const int M = (int)s->M, C = L.N, chunks = L.norm_blocks;
+  const T* x = act_in<T>(s, l);
+  const T* dz = dz_src<T>(s, l, dY);
+  float* part0 = (float*)s->at(L.off_gpart);
+  float* part1 = part0 + (size_t)chunks * C;
+  const float2* stats = (const float2*)s->at(L.off_stats);
+  float2* means = (float2*)s->at(L.off_means);
+  et::bn_colstats_kernel<T, et::kBnBackward><<<dim3(ceil_div(C, 256), chunks), dim3(32, 8), 0, st>>>(dz, x, stats, M, C,
+                                                                                                 part0, part1);
+  ET_TRY(after_launch());
+  ++*launches;
+  if (want_dx) {
+    const LayerRT& P = s->ly[l - 1];
+    const bool need_act = P.act != ET_ACT_NONE;
+    const bool need_G = !need_act || P.residual_src >= 0;
+    et::bn_finalize_kernel<<<ceil_div(C, 32), dim3(32, 32), 0, st>>>(part0, part1, chunks, C, (float)(1.0 / (double)M),
+                                                                   L.eps, 2, nullptr, means);
+    ET_TRY(after_launch());
+    const long long total = (long long)M * (C / 8);
+    et::bn_backward_kernel<T><<<ceil_div(total, et::kBnEltThreads), et::kBnEltThreads, 0, st>>>(
+        dz, x, stats, means, (const T*)L.W, L.consumer >= 0 ? grad_act<T>(s, L.consumer + 1, dY) : nullptr,
+        need_G ? (T*)s->at(P.off_G_out) : nullptr, need_act ? (const T*)s->at(P.off_Z) : nullptr,
+        need_act ? (T*)s->at(P.off_dZ) : nullptr, P.act, s->M, C);
+    ET_TRY(after_launch());
+    *launches += 2;
+  }
+  if (!want_dgamma || (grad == nullptr && delta == nullptr && !sgd)) return ET_OK;
+  float* imp = (float*)s->at(s->off_imp_parts) + s->imp_offs[2 * l];
+  et::bias_finish_kernel<T><<<L.imp_count_w, dim3(et::kBiasCols, et::kBiasLanes), 0, st>>>(
+      part1, chunks, C, C, grad, delta, imp, (T*)L.W, opt_params(s, lr), sgd ? 1 : 0, s->delta_is_snapshot ? 1 : 0, L.W32,
+      L.st1[0], L.st2[0]);
+  ++*launches;
+  return after_launch();
+}
+
 // ---- attention core --------------------------------------------------------------------------
 // Dynamic shared memory above 48 KB has to be allowed per kernel and device.
 et_status attn_allow_forward(size_t bytes) {
@@ -857,7 +927,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
     if (two) CU_TRY(cudaEventRecord(s->chain_ev[L], cs));  // dZ_{L-1} is ready
     for (int l = L - 1; l >= d; --l) {
       const LayerRT& Y = s->ly[l];
-      const bool norm = Y.kind == ET_LAYER_NORM;
+      const bool norm = Y.vector_params();
       const double gemm = Y.kind != ET_LAYER_DENSE ? 0.0 : 2.0 * (double)s->M * Y.K * Y.N;
       if (mask[2 * l + 1]) {
         // On the tensor-core path the column partials of dZ_l were left by dgrad(l+1) in this
@@ -887,7 +957,11 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         // partials of d gamma (if selected); it reads gamma, so the finisher that may update gamma
         // follows it on the same stream
         if (l > d || mask[2 * l]) {
-          ET_TRY(run_norm_backward<T>(s, l, dY, l > d, mask[2 * l] != 0, grads ? grads[2 * l] : nullptr,
+          if (Y.kind == ET_LAYER_NORM)
+            ET_TRY(run_norm_backward<T>(s, l, dY, l > d, mask[2 * l] != 0, grads ? grads[2 * l] : nullptr,
+                                        delta ? (const T*)delta[2 * l] : nullptr, sgd, lr, &launches, cs));
+          else
+            ET_TRY(run_bn_backward<T>(s, l, dY, l > d, mask[2 * l] != 0, grads ? grads[2 * l] : nullptr,
                                       delta ? (const T*)delta[2 * l] : nullptr, sgd, lr, &launches, cs));
         }
         if (two && l > d) CU_TRY(cudaEventRecord(s->chain_ev[l], cs));
@@ -954,6 +1028,7 @@ et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
   s->x = x;
   for (int l = 0; l < s->L; ++l) {
     if (s->ly[l].kind == ET_LAYER_NORM) ET_TRY(run_norm_forward<T>(s, l, y, st));
+    else if (s->ly[l].kind == ET_LAYER_BATCHNORM) ET_TRY(run_bn_forward<T>(s, l, y, st));
     else if (s->ly[l].kind == ET_LAYER_ATTENTION) ET_TRY(run_attn_forward(s, l, st));
     else if (s->ly[l].kind == ET_LAYER_IM2COL) ET_TRY(run_im2col_forward<T>(s, l, st));
     else ET_TRY(run_forward_layer<T>(s, l, y, st));
@@ -999,8 +1074,12 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (d.fold > 1 && d.act != ET_ACT_NONE) { err = ET_ERR_UNSUPPORTED; break; }
     y.K = d.in_features; y.N = d.out_features; y.fold = d.fold; y.Nw = d.out_features / d.fold;
     y.act = d.act; y.residual_src = d.residual_src;
-    if (d.kind < ET_LAYER_DENSE || d.kind > ET_LAYER_IM2COL) { err = ET_ERR_INVALID_ARG; break; }
+    if (d.kind < ET_LAYER_DENSE || d.kind > ET_LAYER_BATCHNORM) { err = ET_ERR_INVALID_ARG; break; }
     y.kind = d.kind; y.eps = d.eps;
+    if (y.kind == ET_LAYER_BATCHNORM) {
+      if (y.K != y.N || y.fold != 1 || y.residual_src != -1 || !(y.eps >= 0.f)) { err = ET_ERR_INVALID_ARG; break; }
+      if (y.N % 8) { err = ET_ERR_UNSUPPORTED; break; }
+    }
     if (y.kind == ET_LAYER_IM2COL) {
       y.img_h = d.height; y.img_w = d.width; y.ksize = d.ksize;
       if (y.fold != 1 || y.act != ET_ACT_NONE || y.residual_src != -1 || y.img_h < 1 || y.img_w < 1 || y.ksize < 1 ||
@@ -1062,6 +1141,11 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
     if (y.kind == ET_LAYER_ATTENTION) {
       y.off_lse = take((size_t)M * y.heads * sizeof(float));
+    } else if (y.kind == ET_LAYER_BATCHNORM) {
+      y.off_stats = take((size_t)y.N * sizeof(float2));
+      y.off_means = take((size_t)y.N * sizeof(float2));
+      y.norm_blocks = ceil_div(M, et::kBnRows);                           // chunks of the column reductions
+      y.off_gpart = take((size_t)2 * y.norm_blocks * y.N * sizeof(float));
     } else if (y.kind == ET_LAYER_NORM) {
       y.off_stats = take((size_t)M * sizeof(float2));
       y.norm_blocks = std::min(ceil_div(M, et::kNormWarps), s->sms * 8);
@@ -1091,10 +1175,10 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
       s->imp_counts[2 * l] = s->imp_counts[2 * l + 1] = 0;
       continue;
     }
-    max_partial = std::max(max_partial, y.kind == ET_LAYER_NORM ? (size_t)y.N * sizeof(float)
+    max_partial = std::max(max_partial, y.vector_params() ? (size_t)y.N * sizeof(float)
                                                                 : (size_t)y.split * y.K * y.N * sizeof(float));
     y.off_biaspart = take((size_t)std::max(chunks, ceil_div(M, 256) * 8 + 8) * y.Nw * sizeof(float));
-    y.imp_count_w = y.kind == ET_LAYER_NORM ? ceil_div(y.N, et::kBiasCols)
+    y.imp_count_w = y.vector_params() ? ceil_div(y.N, et::kBiasCols)
                                             : ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
     y.imp_count_b = ceil_div(y.N, et::kBiasCols);
     s->imp_offs[2 * l] = imp_total; s->imp_counts[2 * l] = y.imp_count_w; imp_total += y.imp_count_w;
@@ -1262,7 +1346,7 @@ et_status et_importance(et_stack* s, const uint8_t* mask, int32_t n_tensors, flo
     const size_t count = is_w ? y.w_count() : (size_t)y.N;
     const int blocks = s->imp_counts[t];
     float* out = parts + s->imp_offs[t];
-    const bool wide = is_w && y.kind != ET_LAYER_NORM;       // 8 elements per thread; gamma goes like a bias
+    const bool wide = is_w && !y.vector_params();           // 8 elements per thread; gamma goes like a bias
     if (s->dtype == ET_BF16) {
       if (wide) et::importance_kernel<bf16, 8><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const bf16*)delta[t], count, out);
       else      et::importance_kernel<bf16, 1><<<blocks, et::kEltThreads, 0, st>>>(grads[t], (const bf16*)delta[t], count, out);
@@ -1297,7 +1381,7 @@ et_status et_tensor_metric(et_stack* s, const uint8_t* mask, int32_t n_tensors, 
     const size_t count = is_w ? y.w_count() : (size_t)y.N;
     const int blocks = s->imp_counts[t];
     float* out = parts + s->imp_offs[t];
-    const bool wide = is_w && y.kind != ET_LAYER_NORM;
+    const bool wide = is_w && !y.vector_params();
     const float* f32 = kind == ET_METRIC_GRADIENT_MAGNITUDE ? grads[t] : (is_w ? y.W32 : y.b32);   // masters if attached
     const void* stored = is_w ? y.W : y.b;
     if (f32 != nullptr || s->dtype == ET_F32) {
@@ -1446,6 +1530,20 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
         double* slot; double v;
         ~AddCarried() { *slot += v; }
       } add_carried{&t_dy[2 * l + 1], carried};
+      if (s->ly[l].kind == ET_LAYER_BATCHNORM) {
+        // Section 5.2, its own subject: one black box, all of its backward time in t_dy of beta
+        t_dw[2 * l] = 0.0; t_dw[2 * l + 1] = 0.0;
+        double t_box = 0.0, t_beta = 0.0;
+        if (s->dtype == ET_BF16) {
+          ET_TRY(timed([&]() { return run_bn_backward<bf16>(s, l, dY, l >= 1, true, scratch_grad, nullptr, false, 0.f, &dummy, st); }, &t_box));
+          ET_TRY(timed([&]() { return run_bgrad_layer<bf16>(s, l, dY, nullptr, nullptr, false, 0.f, &dummy, st); }, &t_beta));
+        } else {
+          ET_TRY(timed([&]() { return run_bn_backward<float>(s, l, dY, l >= 1, true, scratch_grad, nullptr, false, 0.f, &dummy, st); }, &t_box));
+          ET_TRY(timed([&]() { return run_bgrad_layer<float>(s, l, dY, nullptr, nullptr, false, 0.f, &dummy, st); }, &t_beta));
+        }
+        t_dy[2 * l + 1] = t_box + t_beta;
+        continue;
+      }
       if (s->ly[l].kind == ET_LAYER_NORM) {
         // Section 5.2: the layer is one black box whose whole backward time belongs to t_dy of beta
         t_dw[2 * l] = 0.0; t_dw[2 * l + 1] = 0.0;

@@ -89,13 +89,13 @@ def flop_costs(layers, M):
     for when measured times are not wanted."""
     t_dw, t_dy = [], []
     for ly in layers:
-        if getattr(ly, "kind", 0) >= 2:
+        if getattr(ly, "kind", 0) in (2, 3):
             # a layer without tensors: its backward work, one pass over its rows here, is charged to the
             # bias below it by the caller's cost vectors; as a stand-in its own slots cost nothing
             t_dw += [0.0, 0.0]
             t_dy += [0.0, 0.0]
             continue
-        if getattr(ly, "kind", 0) == 1:
+        if getattr(ly, "kind", 0) in (1, 4):
             # normalisation layer: one pass over the rows, all of it charged to beta's error-gradient
             # time (Section 5.2)
             t_dw += [0.0, 0.0]

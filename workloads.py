@@ -167,18 +167,19 @@ def conv_layers(c_in: int, c_out: int, height: int, width: int, ksize: int = 3, 
             Layer(ksize * ksize * c_in, c_out, act=act, residual_src=residual_src)]
 
 
-def resnet_bottleneck_blocks(n_blocks: int, c: int, mid: int, height: int, width: int, bn: bool = False) -> List[Layer]:
+def resnet_bottleneck_blocks(n_blocks: int, c: int, mid: int, height: int, width: int, bn: bool = False,
+                             act: int = ACT_RELU) -> List[Layer]:
     """ResNet bottleneck: 1x1 c->mid ReLU, 3x3 mid->mid ReLU, 1x1 mid->c + block input (4 layers);
-    bn=True puts a batch normalisation between each convolution and its ReLU (7 layers)."""
+    bn=True puts a batch normalisation between each of the first two convolutions and its ReLU (6 layers)."""
     layers: List[Layer] = []
     for blk in range(n_blocks):
-        base = (7 if bn else 4) * blk
+        base = (6 if bn else 4) * blk
         if bn:
-            layers += [Layer(c, mid), batchnorm_layer(mid, ACT_RELU)]
-            layers += conv_layers(mid, mid, height, width, 3) + [batchnorm_layer(mid, ACT_RELU)]
+            layers += [Layer(c, mid), batchnorm_layer(mid, act)]
+            layers += conv_layers(mid, mid, height, width, 3) + [batchnorm_layer(mid, act)]
         else:
-            layers.append(Layer(c, mid, act=ACT_RELU))
-            layers += conv_layers(mid, mid, height, width, 3, act=ACT_RELU)
+            layers.append(Layer(c, mid, act=act))
+            layers += conv_layers(mid, mid, height, width, 3, act=act)
         layers.append(Layer(mid, c, residual_src=base))
     return layers
 
@@ -307,17 +308,18 @@ def resnet_1x1(seed: int = 2, p_select: float = 0.5, n_blocks: int = 6, tokens: 
 
 
 def resnet_bottleneck(seed: int = 6, p_select: float = 0.5, n_blocks: int = 6, images: int = 32, height: int = 14,
-                      width: int = 14, c: int = 1024, mid: int = 256, params: bool = True, bn: bool = False) -> Workload:
+                      width: int = 14, c: int = 1024, mid: int = 256, params: bool = True, bn: bool = False,
+                      act: int = ACT_RELU, dtype: int = DT_BF16) -> Workload:
     """bf16 ResNet-50 conv4_x bottlenecks with their 3x3 convolutions (NHWC rows), optionally with their
     batch normalisations."""
     rng = np.random.default_rng(seed)
-    layers = resnet_bottleneck_blocks(n_blocks, c, mid, height, width, bn)
+    layers = resnet_bottleneck_blocks(n_blocks, c, mid, height, width, bn, act)
     mask = bernoulli_weight_mask(rng, len(layers), p_select)
     for l, ly in enumerate(layers):
         if ly.kind == KIND_IM2COL:
             mask[2 * l] = mask[2 * l + 1] = 0
-    return _finish("resnet50_conv4_bottleneck_bf16", layers, images * height * width, DT_BF16, 0.01, mask, rng,
-                   he_init=True, params=params)
+    return _finish("resnet50_conv4_bottleneck" + ("_bn" if bn else ""), layers, images * height * width, dtype, 0.01, mask,
+                   rng, he_init=True, params=params)
 
 
 def small_stack(layers: List[Layer], M: int, dtype: int, seed: int, mask=None, w_std: float = 0.05,
