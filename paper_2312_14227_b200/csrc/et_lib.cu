@@ -149,8 +149,11 @@ struct LayerRT {
   size_t off_biaspart = 0;  // column partials of dZ_l for the bias gradient (own buffer per layer, so
                             // that finishing a bias never has to be ordered against later GEMMs)
   int split = 1;            // wgrad contraction splits
+  int split_shared = 1;     // the same while the error-gradient chain runs beside the weight gradients (dense masks)
   int bn_fwd = 256, bn_dgrad = 256, bn_wgrad = 256;   // tile widths chosen per GEMM
   bool pair_fwd = false, pair_dgrad = false, pair_wgrad = false;   // CTA-pair (cta_group::2) tiles
+  int bn_dgrad_sh = 256; bool pair_dgrad_sh = false;   // dgrad tiles while the two streams share the GPU
+  bool big_gemm = false;    // its GEMMs run for tens of microseconds (10 GFLOP and more)
   int imp_count_w = 0, imp_count_b = 0;
   int img_h = 0, img_w = 0, ksize = 0;   // patch gather: K = channels, N = ksize^2 * K
   bool trainable() const { return kind == ET_LAYER_DENSE || kind == ET_LAYER_NORM || kind == ET_LAYER_BATCHNORM; }
@@ -160,6 +163,7 @@ struct LayerRT {
   // bf16 stacks: one TMA descriptor per tensor (the caller's x, y and dY get theirs per call)
   TMaps map_W, map_aout, map_Gout, map_Z, map_dZ;
   CUtensorMap map_Wd;       // W as the K-major B of the dgrad GEMM: one box = the CTA's whole B tile
+  CUtensorMap map_Wd_sh;    // the same for the shared-GPU tile shape
 };
 
 }  // namespace
@@ -216,7 +220,10 @@ using et::bf16;
 // gets units.  A CTA pair (cta_group::2) loads half of B per CTA and so moves fewer L2 bytes per
 // flop; a 192-wide pair tile needs 32-row B boxes and therefore a K-major B (dgrad only).
 struct TilePlan { int bn; int split; bool pair; };
-TilePlan choose_tiles(int rows, int cols, int kb_total, int sms, bool allow_split, bool b_k_major, int n_multiple) {
+// fractional: the GEMM shares the GPU with another stream's work, which fills the SMs a partly filled
+// last wave leaves idle, so the cost is the work itself (fractional waves), not whole waves.
+TilePlan choose_tiles(int rows, int cols, int kb_total, int sms, bool allow_split, bool b_k_major, int n_multiple,
+                      bool fractional = false) {
   TilePlan best{256, 1, false};
   double best_cost = -1.0;
   const double sm_flops = 10.5e12, sm_l2_bytes = 10.5e12 / 148.0;
@@ -234,8 +241,8 @@ TilePlan choose_tiles(int rows, int cols, int kb_total, int sms, bool allow_spli
       for (int sp = 1; sp <= smax; ++sp) {
         const int kbs = ceil_div(kb_total, sp);
         if ((long long)(sp - 1) * kbs >= kb_total) continue;         // an empty split
-        const long long waves = ceil_div(tiles * sp, workers);
-        const double cost = (double)waves * (kbs + 6) * kb_time;
+        const double waves = fractional ? std::max(1.0, (double)(tiles * sp) / workers) : (double)ceil_div(tiles * sp, workers);
+        const double cost = waves * (kbs + 6) * kb_time;
         if (best_cost < 0 || cost < best_cost * 0.999) { best_cost = cost; best = {bn, sp, pair != 0}; }
       }
     }
@@ -433,7 +440,8 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
 // G_l = dZ_l W_l^T (+ skip gradient), dZ_{l-1} = G_l * act'(Z_{l-1});  l >= 1
 // Row blocks of 32 that the dgrad GEMM of layer l writes fused column sums for.
 int dgrad_row_blocks(const et_stack* s, int l) {
-  const int tile_m = s->ly[l].pair_dgrad ? 2 * et::tc::BM : et::tc::BM;
+  const bool pair = s->chain_shares_gpu ? s->ly[l].pair_dgrad_sh : s->ly[l].pair_dgrad;
+  const int tile_m = pair ? 2 * et::tc::BM : et::tc::BM;
   return ceil_div(s->M, tile_m) * (tile_m / 32);
 }
 
@@ -452,7 +460,14 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
     p.b_k_seg_stride = L.Nw;
     et::tc::EpiMaps em;
     const CUtensorMap& gout = P.map_Gout.b128;                // G_l lives in layer l-1's buffer
-    const CUtensorMap& wmap = L.map_Wd;
+    // Two tile plans: alone on the GPU whole waves count (768-wide outputs on 12608 rows: 192-wide pair
+    // tiles, 200 units in 3 waves at 90 %); beside the weight-gradient stream the idle SMs of a last wave are
+    // not lost, and the wider tile with less operand traffic per flop wins (256-wide: 150 units; measured on
+    // the ViT-B step 2.45 -> 2.33 ms).
+    const bool sh = s->chain_shares_gpu;
+    const int bn_d = sh ? L.bn_dgrad_sh : L.bn_dgrad;
+    const bool pair_d = sh ? L.pair_dgrad_sh : L.pair_dgrad;
+    const CUtensorMap& wmap = sh ? L.map_Wd_sh : L.map_Wd;
     const CUtensorMap& skip = need_skip ? g_map(s, L.consumer + 1).b128 : gout;
     const CUtensorMap& zmap = P.map_Z.b128;
     const CUtensorMap& dzout = P.map_dZ.b128;
@@ -462,7 +477,7 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
       epi.mul_act = false; epi.act_prev = P.act;
       epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = skip; em.out[0] = gout; em.in[1] = gout; em.out[1] = gout;
-      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
+      return launch_tc<false, false>(bn_d, pair_d, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
     }
     if (!need_skip && !need_G) {                              // dZ_{l-1} = acc * act'(Z_{l-1})
       et::DgradEpiS<1> epi;
@@ -470,14 +485,14 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
       epi.mul_act = true; epi.act_prev = P.act;
       epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
       em.in[0] = zmap; em.out[0] = dzout; em.in[1] = zmap; em.out[1] = dzout;
-      return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
+      return launch_tc<false, false>(bn_d, pair_d, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
     }
     et::DgradEpiS<2> epi;                                     // both G_l and dZ_{l-1}
     epi.has_in[0] = need_skip; epi.has_in[1] = true; epi.has_out[0] = need_G; epi.has_out[1] = true;
     epi.mul_act = false; epi.act_prev = P.act;
     epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
     em.in[0] = skip; em.out[0] = gout; em.in[1] = zmap; em.out[1] = dzout;
-    return launch_tc<false, false>(L.bn_dgrad, L.pair_dgrad, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
+    return launch_tc<false, false>(bn_d, pair_d, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
   } else {
     et::DgradEpi<T> epi;
     epi.skip = need_skip ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
@@ -763,7 +778,7 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   {
     TimedLaunch tl(s, ET_K_WGRAD, st);
     if constexpr (is_bf16<T>::value) {
-      split = L.split;
+      split = (s->chain_shares_gpu && !s->wgrad_one_unit) ? L.split_shared : L.split;
       et::tc::Params p = tc_params(s, L.K, L.N, (int)s->M, 1, split);
       p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
       et::tc::EpiMaps em;
@@ -1157,11 +1172,18 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
       const TilePlan w = choose_tiles(y.K, y.N, ceil_div(M, et::tc::BK), s->sms, true, false, y.fold > 1 ? y.Nw : 0);
       y.bn_fwd = f.bn; y.pair_fwd = f.pair;
       y.bn_dgrad = d.bn; y.pair_dgrad = d.pair;
+      // The shared-GPU variants assume kernels long enough to keep the GPU busy; GEMMs of a few microseconds
+      // (the 1x1 convolutions of a ResNet block: 3.3 GFLOP) are launch-bound, the other stream finds the GPU
+      // mostly idle and is better off with the stand-alone plan (its full backprop went 0.34 -> 0.41 ms otherwise).
+      y.big_gemm = 2.0 * (double)M * y.K * y.N >= 10e9;
+      const TilePlan dsh = y.big_gemm ? choose_tiles((int)M, y.K, kb_n, s->sms, false, true, 0, true) : d;
+      y.bn_dgrad_sh = dsh.bn; y.pair_dgrad_sh = dsh.pair;
       y.bn_wgrad = w.bn; y.pair_wgrad = w.pair; y.split = w.split;
       if (const char* force = getenv("ET_DEBUG_TILES")) {          // debug: "<bn>,<pair>[,<split>]" for every GEMM
         int fb = 0, fp = 0, fs = 0;
         if (sscanf(force, "%d,%d,%d", &fb, &fp, &fs) >= 2 && (fb == 128 || fb == 192 || fb == 256)) {
           y.bn_dgrad = fb; y.pair_dgrad = fp != 0;
+          y.bn_dgrad_sh = fb; y.pair_dgrad_sh = fp != 0;
           const int fbm = (fb == 192) ? 256 : fb;                   // MN-major B has no 192-wide pair tile
           y.bn_fwd = fp ? fbm : fb; y.pair_fwd = fp != 0;
           if (y.fold == 1 || y.Nw % (fp ? fbm : fb) == 0) { y.bn_wgrad = fp ? fbm : fb; y.pair_wgrad = fp != 0; }
@@ -1175,8 +1197,19 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
       s->imp_counts[2 * l] = s->imp_counts[2 * l + 1] = 0;
       continue;
     }
+    // Weight gradients that run persistently beside the error-gradient chain (dense masks) need not fill the
+    // GPU by themselves: at most two splits keep the partial-sum traffic and the reducers small, the chain
+    // takes the SMs they leave free (ViT-B full backprop 4.33 -> 4.02 ms; "as many splits as give every SM
+    // pair a unit" gave 4.23 ms, a single split 4.59 ms).
+    y.split_shared = y.split;
+    if (y.kind == ET_LAYER_DENSE && dtype == ET_BF16 && y.big_gemm && getenv("ET_DEBUG_TILES") == nullptr) {
+      const int kb = ceil_div(M, et::tc::BK);
+      int sp = std::min(y.split, 2);
+      while (sp > 1 && (long long)(sp - 1) * ceil_div(kb, sp) >= kb) --sp;
+      y.split_shared = sp;
+    }
     max_partial = std::max(max_partial, y.vector_params() ? (size_t)y.N * sizeof(float)
-                                                                : (size_t)y.split * y.K * y.N * sizeof(float));
+                                                          : (size_t)std::max(y.split, y.split_shared) * y.K * y.N * sizeof(float));
     y.off_biaspart = take((size_t)std::max(chunks, ceil_div(M, 256) * 8 + 8) * y.Nw * sizeof(float));
     y.imp_count_w = y.vector_params() ? ceil_div(y.N, et::kBiasCols)
                                             : ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
@@ -1232,6 +1265,7 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
       if (y.kind == ET_LAYER_DENSE) {
         ET_TRY(make_tmaps(&y.map_W, y.W, y.N, y.K));
         ET_TRY(make_map(&y.map_Wd, y.W, y.N, y.K, y.pair_dgrad ? y.bn_dgrad / 2 : y.bn_dgrad));
+        ET_TRY(make_map(&y.map_Wd_sh, y.W, y.N, y.K, y.pair_dgrad_sh ? y.bn_dgrad_sh / 2 : y.bn_dgrad_sh));
       }
       if (l < s->L - 1) {
         ET_TRY(make_tmaps(&y.map_aout, s->at(y.off_a_out), y.Nw, s->M));
@@ -1506,6 +1540,8 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
     for (int l = 0; l < L; ++l)
       if (!s->ly[l].trainable()) ones[2 * l] = ones[2 * l + 1] = 0;
     ET_TRY(et_backward_elastic(s, dY, ones.data(), 2 * L, nullptr, nullptr, nullptr, 0, 0.f, nullptr, stream));
+    s->chain_shares_gpu = false;                              // the launches below run one at a time
+    s->wgrad_one_unit = false;
     float* scratch_grad = (float*)s->at(s->off_partial);      // in-place: each element is read before it is written
     double pending_nontrainable = 0.0;
     for (int l = L - 1; l >= 0; --l) {
