@@ -107,3 +107,22 @@ def test_profiled_costs_follow_the_papers_rules_for_non_dense_layers():
     imp[6:8] = 0.0
     mask, val, est = et.et_select_dp(imp, t_dw, t_dy, t_fwd, 0.6, 1000)
     assert mask[6] == 0 and mask[7] == 0 and est <= 0.6 * (t_fwd + t_dw.sum() + t_dy.sum()) - t_fwd + 12 * (t_dw.sum() + t_dy.sum()) / 1000
+
+
+def test_full_block_is_deterministic():
+    # normalisation, attention and dense kernels: two runs from the same inputs give identical bits
+    import torch
+    h = _h()
+    w = wl.vit_b_full(seed=86, p_select=0.5, n_blocks=2, batch=3, seq=197, d=128, ffn=256, heads=2)
+    m = _mask_all(w.layers)
+    outs = []
+    for _ in range(2):
+        run = h.GpuRun(w)
+        run.forward_loss()
+        grads = run.alloc_grads(m)
+        delta = [h.to_dev(d, w.dtype) for d in wl.draw_delta(w, 4)]
+        run.backward(m, grads, delta)
+        outs.append(([g.clone() for g in grads if g is not None], run.importance.clone(), run.y.clone()))
+    for a, b in zip(outs[0][0], outs[1][0]):
+        assert torch.equal(a, b)
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
