@@ -48,6 +48,16 @@ def _peaks():
     return dict(hbm_gbs=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
 
 
+NOMINAL_BF16_TFLOPS = 2250.0      # dense bf16 tensor peak of the part, for context beside the measured peaks
+NOMINAL_HBM_GBS = 8000.0
+
+
+def tensor_fracs(tf: float, peaks: dict) -> dict:
+    """One achieved TFLOP/s figure against the three denominators in use."""
+    return {"of_measured_burst": tf / peaks["tf_burst"], "of_measured_sustained": tf / peaks["tf_sustained"],
+            "of_nominal_dense": tf / NOMINAL_BF16_TFLOPS}
+
+
 def _dgrad_traffic():
     """DRAM bytes per dgrad launch from the committed ncu capture, or None once the GEMM sources
     have changed since the counters were taken."""
@@ -143,6 +153,23 @@ def oracle_sample(w_full: wl.Workload, n_blocks: int):
     return step, f"oracle masked backward + importance + SGD on the top {n_blocks} of 12 blocks, all {w.M} tokens, float64"
 
 
+ORACLE_SAMPLE_BLOCKS = 1      # both the reference arm and the cpu_baseline leg time this sample
+
+
+def time_oracle(w_full: wl.Workload, steps: int, warmup: int):
+    """Times the oracle as it stands on the bounded sample: `warmup` untimed calls, then `steps` timed ones.
+    Returns (list of seconds, executed flops per step, description of the sample)."""
+    step, sample = oracle_sample(w_full, ORACLE_SAMPLE_BLOCKS)
+    for _ in range(warmup):
+        step()
+    times, flops = [], 0.0
+    for _ in range(steps):
+        dt, flops = step()
+        times.append(dt)
+    sample += f" (the top {ORACLE_SAMPLE_BLOCKS} of 12 blocks with its own mask bits: about 1/12 of the configuration's work)"
+    return times, flops, sample
+
+
 def blas_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -157,22 +184,18 @@ def run_reference(args):
     if rank != 0:
         return
     w = wl.vit_b(params=False)
-    step, sample = oracle_sample(w, 1)          # one block per step keeps K steps within minutes
-    for _ in range(min(args.warmup, 1)):
-        step()
-    times, flops = [], 0.0
-    for _ in range(args.steps):
-        dt, flops = step()
-        times.append(dt)
+    warm = max(1, min(args.warmup, 3))          # one block per step keeps K steps within minutes
+    times, flops, sample = time_oracle(w, args.steps, warm)
     ms = 1e3 * float(np.mean(times))
     val = flops / (ms * 1e-3) / 1e12
     cores = blas_threads()
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "vit_b_linear_bf16 (oracle sample)", "sample": sample},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                         "median_value": flops / float(np.median(times)) / 1e12},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -303,53 +326,64 @@ def run_own(args):
     clocks = sampler.stop()     # sampled from the full-backprop run to the end of the end-to-end run
 
     # per-kernel-class device time over the same steps (event pair around every launch; while
-    # this is on, the library keeps all kernels on one stream so that a pair brackets one kernel)
-    et.et_timing_enable(stack, True)
-    inst_ms, _ = timed(lambda: step(w.mask), args.steps, 1)
-    classes = et.et_timing_read(stack)
-    # the first (warm-up) step is included in the record: normalise by launches
-    et.et_timing_enable(stack, False)
-
+    # this is on, the library keeps all kernels on one stream so that a pair brackets one kernel).
+    # Taken twice: with the tile plan the two-stream step above really launches ("shared": tile shapes
+    # chosen for a GPU shared between the chain and the weight gradients) and with the plan a
+    # single-stream caller gets ("alone").
     peaks = _peaks()
-    # algorithmic work per class for the elastic mask
     M = w.M
     first = next(l for l in range(w.L) if w.mask[2 * l] or w.mask[2 * l + 1])
     dgrad_flops = sum(2.0 * M * ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if l > first)
     wgrad_flops = sum(2.0 * M * ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if w.mask[2 * l])
-    n_steps_rec = args.steps + 1
-
-    def per_step(cls):
-        t, n = classes[cls]
-        return t / n_steps_rec, n / n_steps_rec
-
-    dg_ms, dg_n = per_step("dgrad")
-    wg_ms, wg_n = per_step("wgrad")
-    rd_ms, rd_n = per_step("wgrad_reduce")
-    bg_ms, bg_n = per_step("bgrad")
-    ot_ms, ot_n = per_step("other")
+    sel_params = sum(ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if w.mask[2 * l])
     # bytes the reducer must move per selected kernel tensor of P parameters: S*4P partial reads
     # are its own scratch traffic; the algorithmic part is 4P (gradient) + 2P (dW) + 2P + 2P (W in/out)
-    sel_params = sum(ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if w.mask[2 * l])
     reduce_bytes = 10.0 * sel_params
-    bgrad_bytes = sum(2.0 * M * ly.out_width for l, ly in enumerate(w.layers) if w.mask[2 * l + 1])
-    dg_tf = dgrad_flops / (dg_ms * 1e-3) / 1e12 if dg_ms > 0 else 0.0
-    kernels = {
-        "dgrad_gemm": {"launches_per_step": dg_n, "ms_per_step": dg_ms, "achieved": dg_tf, "unit": "TFLOP/s",
-                       "frac_of_sustained_peak": dg_tf / peaks["tf_sustained"]},
-        "wgrad_gemm": {"launches_per_step": wg_n, "ms_per_step": wg_ms,
-                       "achieved": wgrad_flops / (wg_ms * 1e-3) / 1e12 if wg_ms > 0 else 0.0, "unit": "TFLOP/s"},
-        "wgrad_reduce_importance_sgd": {"launches_per_step": rd_n, "ms_per_step": rd_ms,
-                                        "achieved": reduce_bytes / (rd_ms * 1e-3) / 1e9 if rd_ms > 0 else 0.0,
-                                        "unit": "GB/s"},
-        "bias_grad": {"launches_per_step": bg_n, "ms_per_step": bg_ms,
-                      "achieved": bgrad_bytes / (bg_ms * 1e-3) / 1e9 if bg_ms > 0 else 0.0, "unit": "GB/s"},
-        "other": {"launches_per_step": ot_n, "ms_per_step": ot_ms},
-        "instrumented_step_ms": inst_ms,
-    }
-    kernels["wgrad_gemm"]["frac_of_sustained_peak"] = kernels["wgrad_gemm"]["achieved"] / peaks["tf_sustained"]
-    kernels["wgrad_reduce_importance_sgd"]["frac_of_hbm_peak"] = \
-        kernels["wgrad_reduce_importance_sgd"]["achieved"] / peaks["hbm_gbs"]
-    kernels["bias_grad"]["frac_of_hbm_peak"] = kernels["bias_grad"]["achieved"] / peaks["hbm_gbs"]
+
+    def instrumented(plan):
+        et.et_stack_set_option(stack, et.ET_OPTION_TILE_PLAN, plan)
+        et.et_timing_enable(stack, True)
+        inst_ms, _ = timed(lambda: step(w.mask), args.steps, 1)
+        classes = et.et_timing_read(stack)
+        et.et_timing_enable(stack, False)
+        et.et_stack_set_option(stack, et.ET_OPTION_TILE_PLAN, et.ET_TILE_PLAN_AUTO)
+        n_rec = args.steps + 1          # the warm-up step is in the record too: normalise by recorded steps
+
+        def per_step(cls):
+            t, n = classes[cls]
+            return t / n_rec, n / n_rec
+
+        dg_ms, dg_n = per_step("dgrad")
+        wg_ms, wg_n = per_step("wgrad")
+        rd_ms, rd_n = per_step("wgrad_reduce")
+        bg_ms, bg_n = per_step("bgrad")
+        ot_ms, ot_n = per_step("other")
+        dg_tf = dgrad_flops / (dg_ms * 1e-3) / 1e12 if dg_ms > 0 else 0.0
+        wg_tf = wgrad_flops / (wg_ms * 1e-3) / 1e12 if wg_ms > 0 else 0.0
+        rd_gbs = reduce_bytes / (rd_ms * 1e-3) / 1e9 if rd_ms > 0 else 0.0
+        return {
+            "dgrad_gemm": {"launches_per_step": dg_n, "ms_per_step": dg_ms, "achieved": dg_tf, "unit": "TFLOP/s",
+                           "frac": tensor_fracs(dg_tf, peaks)},
+            "wgrad_gemm": {"launches_per_step": wg_n, "ms_per_step": wg_ms, "achieved": wg_tf, "unit": "TFLOP/s",
+                           "frac": tensor_fracs(wg_tf, peaks)},
+            "wgrad_reduce_importance_sgd": {"launches_per_step": rd_n, "ms_per_step": rd_ms, "achieved": rd_gbs,
+                                            "unit": "GB/s", "algorithmic_bytes_per_step": reduce_bytes,
+                                            "frac_of_hbm_peak": rd_gbs / peaks["hbm_gbs"]},
+            "bias_grad": {"launches_per_step": bg_n, "ms_per_step": bg_ms,
+                          "note": "finishing kernels only (the column sums come out of the dgrad epilogue): a few MB of "
+                                  "partials per step, latency-bound, reported as time"},
+            "other": {"launches_per_step": ot_n, "ms_per_step": ot_ms},
+            "instrumented_step_ms": inst_ms,
+        }
+
+    kernels = {"shared_plan": instrumented(et.ET_TILE_PLAN_SHARED), "alone_plan": instrumented(et.ET_TILE_PLAN_ALONE)}
+    kernels["note"] = ("shared_plan = the tile shapes the timed two-stream step launches; alone_plan = the shapes a "
+                       "single-stream caller gets; both timed one kernel at a time on one stream")
+    dg = kernels["shared_plan"]["dgrad_gemm"]
+    dg_tf = dg["achieved"]
+    timed_span_s = ms * args.steps * 1e-3
+    use_burst = timed_span_s < 1.0
+    peak = peaks["tf_burst"] if use_burst else peaks["tf_sustained"]
 
     if rank != 0:
         if dist is not None:
@@ -359,16 +393,16 @@ def run_own(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": w.name, "blocks": 12, "tokens": w.M, "d": 768, "ffn": 3072,
+        "config": {"workload": w.name, "blocks": args.blocks, "tokens": w.M, "d": 768, "ffn": 3072,
                    "mask": "Bernoulli(0.3) per kernel tensor, seed 1, bias follows kernel",
                    "selected_tensors": int(w.mask.sum()), "deepest_selected_layer": first,
                    "step": "et_backward_elastic with fused importance and " + {"sgd": "SGD", "sgdw": "SGDW (fp32 master weights)", "adam": "Adam (fp32 master weights)"}[args.optimizer],
                    "l2": "inputs larger than L2 (a step streams > 1 GB of activations and gradients)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "executed_flops_per_step": flops,
-        "pct_of_measured_bf16_peak": {"sustained": value / world / peaks["tf_sustained"],
-                                      "burst": value / world / peaks["tf_burst"], "source": peaks["source"]},
+        "step_frac_of_bf16_peak": dict(tensor_fracs(value / world, peaks), source=peaks["source"]),
         "full_backprop": {"ms_per_step": full_ms, "tflops": full_flops / (full_ms * 1e-3) / 1e12,
+                          "frac": tensor_fracs(full_flops / (full_ms * 1e-3) / 1e12, peaks),
                           "executed_flops_per_step": full_flops, "elastic_speedup": full_ms / ms},
         "forward_ms": fwd_ms,
         "clocks": clocks,
@@ -376,17 +410,27 @@ def run_own(args):
                 "h2d_bytes_per_step": dY_host.numel() * dY_host.element_size(),
                 "d2h_bytes_per_step": imp_host.numel() * 4},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "gemm_tc_kernel<dgrad>", "bound": "tensor", "achieved": dg_tf,
-                     "peak": peaks["tf_sustained"], "unit": "TFLOP/s", "frac": dg_tf / peaks["tf_sustained"],
-                     "peak_source": peaks["source"] + " (sustained cuBLAS bf16)", "traffic": _dgrad_traffic(),
+        "roofline": {"kernel": "gemm_tc_kernel<dgrad> (tile plan of the timed step)", "bound": "tensor",
+                     "achieved": dg_tf, "peak": peak, "unit": "TFLOP/s", "frac": dg_tf / peak,
+                     "peak_source": peaks["source"] + (" cuBLAS bf16 burst" if use_burst else " cuBLAS bf16 sustained"),
+                     "peak_choice": f"the timed region lasts {timed_span_s:.2f} s: " +
+                                    ("burst peak (a kernel timed in a short run)" if use_burst else
+                                     "sustained peak (a kernel timed inside a seconds-long step)"),
+                     "frac_all": tensor_fracs(dg_tf, peaks),
+                     "flops_per_step": dgrad_flops, "ms_per_step": dg["ms_per_step"],
+                     "launches_per_step": dg["launches_per_step"],
+                     "ms_x_sm_mhz": (dg["ms_per_step"] * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None,
+                     "traffic": _dgrad_traffic(),
                      "traffic_note": "DRAM bytes per launch, mean over the dgrad GEMMs of one block (ncu, cold cache)"},
         "kernels": kernels,
     }
     if world == 1:
-        cpu_step, sample = oracle_sample(w, 2)
-        dt, fl = cpu_step()
-        line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                                "sample": sample, "seconds": dt}
+        # the oracle as it stands on the host cores: the sample the reference arm times, one warm-up call,
+        # median of five
+        times, fl, sample = time_oracle(w, 5, 1)
+        line["cpu_baseline"] = {"value": fl / float(np.median(times)) / 1e12, "unit": UNIT, "cores": blas_threads(),
+                                "kind": "oracle", "sample": sample, "seconds_per_step": float(np.median(times)),
+                                "timed_steps": len(times), "warmup_steps": 1}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -398,7 +442,7 @@ def run_selector(args):
     time falls with threads when there are thousands of tensors.  No GPU work."""
     import time
     import paper_2312_14227_b200 as et
-    from paper_2312_14227_b200.elastic_loop import flop_costs
+    from workloads import flop_costs
 
     def timed(fn, reps=3):
         best = None
@@ -449,6 +493,67 @@ def run_selector(args):
     out["large_instances"] = big
     out["host_cores"] = os.cpu_count()
     print(json.dumps(out))
+
+
+def run_dp_budget(args):
+    """The ViT-B-shaped stack with masks from the host selector at time budgets rho of the full backward pass
+    (per-tensor times measured on this GPU, seeded Uniform(0,1) importances, T_fwd = 0, T_q = 1000): per rho the
+    selection, the time the model of Section 2.2 predicts for it and the measured step time."""
+    import torch
+    import paper_2312_14227_b200 as et
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    w = wl.vit_b() if args.blocks == 12 else wl.vit_b(n_blocks=args.blocks)
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).to(dev).contiguous()
+    stack = et.et_stack_create(w.layers, w.M, w.dtype)
+    W, b = [to_dev(a) for a in w.W], [to_dev(a) for a in w.b]
+    ws = torch.empty(et.et_stack_workspace_bytes(stack), dtype=torch.uint8, device=dev)
+    et.et_stack_bind(stack, W, b, ws)
+    x, target = to_dev(w.x), to_dev(w.target)
+    y = torch.empty((w.M, w.layers[-1].out_width), dtype=torch.bfloat16, device=dev)
+    dY = torch.empty_like(y)
+    et.et_forward_stack(stack, x, y)
+    et.et_loss_mse_grad(stack, y, target, dY, None)
+    t_dw, t_dy, t_fwd = et.et_profile_costs(stack, x, y, dY, iters=20)
+    et.et_forward_stack(stack, x, y)
+    delta = [to_dev(d) for d in wl.draw_delta(w, 5)]
+    imp = torch.zeros(2 * w.L, dtype=torch.float32, device=dev)
+    rep_ = et.Report(w.L)
+    I = np.random.default_rng(9).random(2 * w.L)
+    total = float(t_dw.sum() + t_dy.sum())
+
+    def measure(mask, two_streams):
+        et.et_stack_set_option(stack, et.ET_OPTION_TWO_STREAMS, 1 if two_streams else 0)
+        for _ in range(max(args.warmup, 3)):
+            et.et_backward_elastic(stack, dY, mask, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep_)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            et.et_backward_elastic(stack, dY, mask, None, delta, imp, et.ET_FLAG_FUSE_SGD, w.lr, rep_)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    rows = []
+    for rho in (0.25, 0.5, 1.0):
+        t0 = time.perf_counter()
+        mask, val, est = et.et_select_dp(I, t_dw, t_dy, 0.0, rho, 1000, et.ET_COST_STRICT)
+        dp_ms = 1e3 * (time.perf_counter() - t0)
+        one = measure(mask, False)
+        two = measure(mask, True)
+        rows.append({"rho": rho, "selected_tensors": int(mask.sum()), "objective": val, "selector_ms": dp_ms,
+                     "budget_ms": rho * total, "estimated_ms": est,
+                     "measured_ms_one_stream": one, "measured_over_estimated_one_stream": one / est if est > 0 else None,
+                     "measured_ms_two_streams": two, "measured_over_estimated_two_streams": two / est if est > 0 else None,
+                     "executed_tflops_two_streams": rep_.flops_executed / two / 1e9})
+    assert et.et_device_status(stack) == et.ET_OK
+    print(json.dumps({"report": w.name + " selector masks at time budgets (T_fwd = 0, T_q = 1000)",
+                      "profiled_full_backward_ms": total, "profiled_forward_ms": t_fwd, "budgets": rows,
+                      "note": "estimated = sum of per-tensor times measured one kernel at a time (the model of "
+                              "Section 2.2); one stream runs the same kernels back to back, two streams overlap the "
+                              "weight gradients with the error-gradient chain"}))
 
 
 def run_side(args):
@@ -638,13 +743,15 @@ def main():
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
-    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "resnet", "prenorm", "full", "bottleneck", "bottleneck_bn", "schedule", "schedule_full", "selector"],
+    ap.add_argument("--workload", default="vit_b", choices=["vit_b", "dp_budget", "resnet", "prenorm", "full", "bottleneck", "bottleneck_bn", "schedule", "schedule_full", "selector"],
                     help="vit_b = the benchmark line; resnet / prenorm / schedule = side reports for the other shapes; "
                          "selector = host-side report on the selection dynamic program")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "own" else args.warmup
     if args.workload == "selector":
         run_selector(args)
+    elif args.workload == "dp_budget":
+        run_dp_budget(args)
     elif args.workload != "vit_b":
         run_side(args)
     elif args.impl == "reference":

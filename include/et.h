@@ -88,7 +88,8 @@ typedef enum {
   ET_ERR_UNSUPPORTED = 6,   /* shape outside what the kernels handle */
   ET_ERR_CUDA = 7,          /* a CUDA runtime call failed; see et_last_cuda_error */
   ET_ERR_TIMEOUT = 8,       /* a bounded device-side wait gave up */
-  ET_ERR_TOO_LARGE = 9      /* problem exceeds the fixed built-in scratch of a *_noalloc call */
+  ET_ERR_TOO_LARGE = 9,     /* problem exceeds the fixed built-in scratch of a *_noalloc call */
+  ET_ERR_GUARD = 10         /* et_debug_check_guards found a guard word overwritten */
 } et_status;
 
 typedef enum { ET_F32 = 0, ET_BF16 = 1 } et_dtype;
@@ -149,6 +150,20 @@ typedef struct et_stack et_stack;
 et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_dtype dtype,
                           et_stack** out);
 et_status et_stack_destroy(et_stack* s);
+
+/* Execution options of a stack (host state; take effect from the next call on).  They change how the
+ * work is launched, never what is computed.
+ *   ET_OPTION_TWO_STREAMS    1 (default): et_backward_elastic runs the error-gradient chain on an internal
+ *                            high-priority stream beside the weight gradients; 0: everything on the caller's stream.
+ *   ET_OPTION_LAUNCH_OVERLAP 1 (default): consecutive GEMMs of one stream start their prologue under the
+ *                            previous kernel's tail (programmatic dependent launch); 0: plain launches.
+ *   ET_OPTION_TILE_PLAN      ET_TILE_PLAN_AUTO (default): GEMM tile shapes made for a GPU shared by the two
+ *                            streams when they run, for a GPU to itself otherwise; ET_TILE_PLAN_ALONE /
+ *                            ET_TILE_PLAN_SHARED force one (per-kernel timing keeps kernels on one stream and
+ *                            can still time the shapes the two-stream step launches). */
+typedef enum { ET_OPTION_TWO_STREAMS = 1, ET_OPTION_LAUNCH_OVERLAP = 2, ET_OPTION_TILE_PLAN = 3 } et_option;
+typedef enum { ET_TILE_PLAN_AUTO = 0, ET_TILE_PLAN_ALONE = 1, ET_TILE_PLAN_SHARED = 2 } et_tile_plan;
+et_status et_stack_set_option(et_stack* s, int32_t option, int32_t value);
 
 /* Bytes of device workspace et_stack_bind needs (a multiple of 256). */
 et_status et_stack_workspace_bytes(const et_stack* s, size_t* bytes);
@@ -289,11 +304,13 @@ et_status et_update_masked(et_stack* s, const uint8_t* mask, int32_t n_tensors, 
  *   db     device float[width]
  * The stage-1 partial sums live in a fixed array compiled into the library:
  * ET_NOALLOC_SCRATCH_FLOATS floats (4 MiB) on every GPU that loads the library, kept until
- * the process ends.  A problem needs ceil(M / 128) * width floats of it; a larger one is
- * refused with ET_ERR_TOO_LARGE and nothing is launched.  The call itself performs no
- * cudaMalloc / cudaFree and calls no allocating routine.
- * The first call on each device looks up the device address of that array (with that
- * device current); make that first call outside any stream capture.
+ * the process ends.  A problem needs ceil(M / 128) * width floats of it; a larger one (or one
+ * of more than 65535 * 128 rows) is refused with ET_ERR_TOO_LARGE and nothing is launched.
+ * The call itself performs no cudaMalloc / cudaFree and calls no allocating routine.
+ * Every call looks up the device address of that array for the current device (nothing is
+ * remembered between calls, so the call stays valid after the application resets the device
+ * or switches the current context).  The first call on a device may load the library's
+ * device code: make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps whatever the last call left in
  * it.  No clearing is needed (each call overwrites every entry it later reads), but two
  * calls that run concurrently on the same GPU -- different streams, or different host
@@ -357,6 +374,19 @@ et_status et_select_dp_int_ex(const double* importance, const int64_t* t_dw, con
 et_status et_select_dp_int(const double* importance, const int64_t* t_dw, const int64_t* t_dy,
                            int32_t n, int64_t budget, int32_t variant,
                            uint8_t* mask_out, double* value_out);
+
+/* ---- debugging aid: guard words round the workspace regions ------------------------- */
+
+/* on != 0: every stack created from now on (in this process) lays its workspace out with 256 guard
+ * bytes after each region (saved activations, error gradients, split partials, bias partials, ...);
+ * et_stack_bind fills them with a pattern.  A kernel that writes past the end of its region hits
+ * them first.  Stands in for a memory checker on stacks whose kernels index by hand.  Costs 256 bytes
+ * per region and nothing at run time. */
+et_status et_debug_guard_regions(int32_t on);
+/* Copies the guard words back and compares them (synchronises `stream`).  ET_OK, or ET_ERR_GUARD with
+ * the index of the first damaged region (in layout order) in *first_bad_region (may be NULL).
+ * A stack created without guards always returns ET_OK. */
+et_status et_debug_check_guards(et_stack* s, void* stream, int32_t* first_bad_region);
 
 /* ---- per-kernel timing (measurement support) ---------------------------------------- */
 

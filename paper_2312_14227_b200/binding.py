@@ -25,6 +25,7 @@ ET_FLAG_DELTA_IS_SNAPSHOT = 2
 ET_ERR_INVALID_ARG, ET_ERR_SHAPE, ET_ERR_DTYPE, ET_ERR_STATE = 1, 2, 3, 4
 ET_ERR_WORKSPACE, ET_ERR_UNSUPPORTED, ET_ERR_CUDA, ET_ERR_TIMEOUT = 5, 6, 7, 8
 ET_ERR_TOO_LARGE = 9
+ET_ERR_GUARD = 10
 ET_NOALLOC_SCRATCH_FLOATS = 1 << 20
 
 
@@ -64,6 +65,7 @@ _SIGS = {
     "et_stack_create": [_vp, _i32, _i64, _i32, C.POINTER(_vp)],
     "et_stack_destroy": [_vp],
     "et_stack_workspace_bytes": [_vp, C.POINTER(C.c_size_t)],
+    "et_stack_set_option": [_vp, _i32, _i32],
     "et_stack_bind": [_vp, _vp, _vp, _vp, C.c_size_t, _vp],
     "et_stack_bind_master": [_vp, _vp, _vp],
     "et_forward_stack": [_vp, _vp, _vp, _vp],
@@ -83,6 +85,8 @@ _SIGS = {
     "et_select_dp_ex": [_vp, _vp, _vp, _i32, _f64, _f64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp],
     "et_select_dp_int_ex": [_vp, _vp, _vp, _i32, _i64, _i32, _i32, _i32, _vp, _vp, _vp],
     "et_device_status": [_vp, _vp],
+    "et_debug_guard_regions": [_i32],
+    "et_debug_check_guards": [_vp, _vp, _vp],
     "et_bias_grad_noalloc": [_vp, _i64, _i32, _i32, _vp, _vp],
     "et_timing_enable": [_vp, _i32],
     "et_timing_read": [_vp, _vp, _vp],
@@ -268,6 +272,14 @@ def et_stack_destroy(s: Stack):
     s.close()
 
 
+ET_OPTION_TWO_STREAMS, ET_OPTION_LAUNCH_OVERLAP, ET_OPTION_TILE_PLAN = 1, 2, 3
+ET_TILE_PLAN_AUTO, ET_TILE_PLAN_ALONE, ET_TILE_PLAN_SHARED = 0, 1, 2
+
+
+def et_stack_set_option(s: Stack, option: int, value: int):
+    _check(_lib.et_stack_set_option(s.handle, int(option), int(value)), "et_stack_set_option")
+
+
 def et_stack_workspace_bytes(s: Stack) -> int:
     out = C.c_size_t()
     _check(_lib.et_stack_workspace_bytes(s.handle, C.byref(out)), "et_stack_workspace_bytes")
@@ -391,6 +403,17 @@ def et_bias_grad_noalloc(dZ, M: int, width: int, dtype: int, db, stream=None):
     memory.  Problems over ET_NOALLOC_SCRATCH_FLOATS raise EtError(ET_ERR_TOO_LARGE)."""
     _check(_lib.et_bias_grad_noalloc(_ptr(dZ), int(M), int(width), dtype, _ptr(db), _stream_ptr(stream)),
            "et_bias_grad_noalloc")
+
+
+def et_debug_guard_regions(on: bool):
+    _check(_lib.et_debug_guard_regions(1 if on else 0), "et_debug_guard_regions")
+
+
+def et_debug_check_guards(s: Stack, stream=None):
+    """(status, index of the first damaged region or -1)."""
+    bad = C.c_int32(-1)
+    st = int(_lib.et_debug_check_guards(s.handle, _stream_ptr(stream), C.addressof(bad)))
+    return st, bad.value
 
 
 def et_device_status(s: Stack, stream=None) -> int:

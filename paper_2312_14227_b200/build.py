@@ -1,6 +1,10 @@
 """Builds libet.so (the C-ABI library) in-tree with nvcc for sm_100a.
 
-    python -m paper_2312_14227_b200.build [--verbose]
+    python paper_2312_14227_b200/build.py [--force] [--verbose] [--debug-hooks]
+
+Rebuilds only when a source is newer than the library (--force: always).  --debug-hooks compiles the
+development switches in (forced tile shapes from the environment); the library built without it
+reads nothing from the environment.
 """
 from __future__ import annotations
 
@@ -20,7 +24,7 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug_hooks: bool = False) -> str:
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -33,6 +37,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     ]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    if debug_hooks:
+        cmd += ["-DET_DEBUG_HOOKS"]
     cmd += [os.path.join(CSRC, f) for f in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
@@ -43,4 +49,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv or "--debug-hooks" in sys.argv, verbose="--verbose" in sys.argv,
+                debug_hooks="--debug-hooks" in sys.argv))

@@ -6,6 +6,7 @@
 #include <cstdlib>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <type_traits>
 #include <vector>
@@ -26,6 +27,9 @@ namespace {
 
 thread_local int g_last_cuda = 0;
 std::atomic<long long> g_launches{0};
+std::atomic<int> g_guard_regions{0};      // et_debug_guard_regions: stacks created from now on get guard words
+constexpr size_t kGuardBytes = 256;
+constexpr unsigned char kGuardByte = 0xA5;
 
 #define CU_TRY(expr)                                   \
   do {                                                 \
@@ -53,19 +57,22 @@ inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn lookup_encode_fn() {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+      q == cudaDriverEntryPointSuccess)
+    return (EncodeTiledFn)p;
+  (void)cudaGetLastError();
+  return nullptr;
+}
 EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
+  static const EncodeTiledFn fn = lookup_encode_fn();     // initialised once, thread-safe
   return fn;
 }
+// Guards the per-device caches of kernel attributes and occupancy answers below: stacks may be driven
+// from several host threads.
+std::mutex g_cache_mutex;
 // Row-major bf16 matrix [outer x inner]: box of 64 columns x box_rows rows, 128-byte swizzle,
 // zero fill outside.
 et_status make_map(CUtensorMap* m, const void* ptr, int inner, long long outer, int box_rows = 64) {
@@ -177,6 +184,7 @@ struct et_stack {
   std::vector<LayerRT> ly;
   std::vector<int> imp_offs, imp_counts;
   size_t ws_bytes = 0;
+  std::vector<size_t> guards;          // offsets of the guard words that follow each workspace region (debug aid)
   size_t off_status = 0, off_partial = 0, off_imp_parts = 0, off_imp_offs = 0,
          off_imp_counts = 0, off_loss_parts = 0, off_dy_stage = 0, off_imp_stage = 0;
   int imp_total = 0;
@@ -193,6 +201,9 @@ struct et_stack {
   bool wgrad_one_unit = false;         // per call: weight-gradient CTAs take one unit each and leave
   bool overlap_launch = true;          // forward / dgrad kernels start their prologue under the previous kernel's tail
   bool chain_shares_gpu = false;       // per call: weight gradients run beside the error-gradient chain
+  bool shared_plan = false;            // per call: the GEMMs use the tile plan made for that case
+  bool opt_two_streams = true;         // et_stack_set_option
+  int opt_tile_plan = ET_TILE_PLAN_AUTO;
   // second stream: the error-gradient chain runs here while weight gradients run on the caller's
   cudaStream_t chain_stream = nullptr;
   std::vector<cudaEvent_t> chain_ev;   // [l] = dgrad(l) finished; [L] = top-layer dZ ready; [L+1] = join
@@ -303,8 +314,9 @@ et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::t
   int dev = 0;
   CU_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
+  std::unique_lock<std::mutex> cache_lock(g_cache_mutex);
   bool& attr_done = attr_done_dev[dev];
-  int& max_clusters = max_clusters_dev[dev];
+  int& max_clusters_ref = max_clusters_dev[dev];
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[2];
   cfg.blockDim = dim3(et::tc::THREADS);
@@ -331,13 +343,15 @@ et_status launch_tc_bn(const CUtensorMap& ma, const CUtensorMap& mb, const et::t
       cfg.gridDim = dim3(sms & ~1);
       cudaLaunchConfig_t occ = cfg;
       occ.numAttrs = n_plain_attrs;
-      if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &occ) != cudaSuccess || max_clusters < 1) {
+      if (cudaOccupancyMaxActiveClusters(&max_clusters_ref, kern, &occ) != cudaSuccess || max_clusters_ref < 1) {
         (void)cudaGetLastError();
-        max_clusters = sms / 2;
+        max_clusters_ref = sms / 2;
       }
     }
     attr_done = true;
   }
+  const int max_clusters = max_clusters_ref;
+  cache_lock.unlock();
   p.tiles_m = ceil_div(p.rows, PAIR ? 2 * et::tc::BM : et::tc::BM);
   p.tiles_n = ceil_div(p.cols, BN);
   const int units = p.tiles_m * p.tiles_n * p.split;
@@ -440,7 +454,7 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
 // G_l = dZ_l W_l^T (+ skip gradient), dZ_{l-1} = G_l * act'(Z_{l-1});  l >= 1
 // Row blocks of 32 that the dgrad GEMM of layer l writes fused column sums for.
 int dgrad_row_blocks(const et_stack* s, int l) {
-  const bool pair = s->chain_shares_gpu ? s->ly[l].pair_dgrad_sh : s->ly[l].pair_dgrad;
+  const bool pair = s->shared_plan ? s->ly[l].pair_dgrad_sh : s->ly[l].pair_dgrad;
   const int tile_m = pair ? 2 * et::tc::BM : et::tc::BM;
   return ceil_div(s->M, tile_m) * (tile_m / 32);
 }
@@ -464,7 +478,7 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
     // tiles, 200 units in 3 waves at 90 %); beside the weight-gradient stream the idle SMs of a last wave are
     // not lost, and the wider tile with less operand traffic per flop wins (256-wide: 150 units; measured on
     // the ViT-B step 2.45 -> 2.33 ms).
-    const bool sh = s->chain_shares_gpu;
+    const bool sh = s->shared_plan;
     const int bn_d = sh ? L.bn_dgrad_sh : L.bn_dgrad;
     const bool pair_d = sh ? L.pair_dgrad_sh : L.pair_dgrad;
     const CUtensorMap& wmap = sh ? L.map_Wd_sh : L.map_Wd;
@@ -550,6 +564,7 @@ template <class K>
 int norm_blocks_per_sm(K kern) {
   struct Seen { const void* fn; int dev, per_sm; };
   static std::vector<Seen> seen;
+  std::lock_guard<std::mutex> cache_lock(g_cache_mutex);
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 1; }
   for (const auto& e : seen)
@@ -697,6 +712,7 @@ et_status attn_allow_forward(size_t bytes) {
   int dev = 0;
   CU_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> cache_lock(g_cache_mutex);
   if (bytes > allowed[dev]) {
     CU_TRY(cudaFuncSetAttribute(et::attn::attn_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
     allowed[dev] = bytes;
@@ -708,6 +724,7 @@ et_status attn_allow_backward(size_t bytes) {
   int dev = 0;
   CU_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> cache_lock(g_cache_mutex);
   if (bytes > allowed[dev]) {
     CU_TRY(cudaFuncSetAttribute(et::attn::attn_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
     allowed[dev] = bytes;
@@ -778,7 +795,7 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
   {
     TimedLaunch tl(s, ET_K_WGRAD, st);
     if constexpr (is_bf16<T>::value) {
-      split = (s->chain_shares_gpu && !s->wgrad_one_unit) ? L.split_shared : L.split;
+      split = (s->shared_plan && !s->wgrad_one_unit) ? L.split_shared : L.split;
       et::tc::Params p = tc_params(s, L.K, L.N, (int)s->M, 1, split);
       p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
       et::tc::EpiMaps em;
@@ -852,11 +869,11 @@ et_status check_ready(const et_stack* s, const uint8_t* mask, int n_tensors) {
 // The dgrad chain dZ_{L-1} -> dZ_{L-2} -> ... is the critical path of the backward pass; weight
 // gradients only hang off it.  Running the chain on its own high-priority stream lets weight-gradient
 // CTAs fill the SMs a chain kernel leaves idle in its last wave and during its prologue and drain.
-// Streams and events are host objects (no device memory).  ET_SINGLE_STREAM=1 turns this off.
+// Streams and events are host objects (no device memory).  et_stack_set_option(ET_OPTION_TWO_STREAMS, 0)
+// turns this off.
 bool setup_two_streams(et_stack* s) {
   if (s->two_streams >= 0) return s->two_streams == 1;
   s->two_streams = 0;
-  if (getenv("ET_SINGLE_STREAM") != nullptr) return false;
   int least = 0, greatest = 0;
   if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess) { (void)cudaGetLastError(); return false; }
   if (cudaStreamCreateWithPriority(&s->chain_stream, cudaStreamNonBlocking, greatest) != cudaSuccess) {
@@ -914,14 +931,17 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         s->map_dy_ptr = dY;
       }
     }
-    const bool two = !s->timing && setup_two_streams(s);   // per-kernel timing wants kernels one at a time
+    const bool two = !s->timing && s->opt_two_streams && setup_two_streams(s);   // per-kernel timing wants kernels one at a time
     // Sharing the GPU with the higher-priority error-gradient chain: when few kernels are selected
     // the weight gradients are filler work and should hand their SMs back after every unit; when
     // they are as much work as the chain itself, persistent CTAs (epilogue overlap) pay more (ViT-B step:
     // 2.33 ms with one-unit CTAs against 2.46 ms persistent; full backprop 4.0 ms persistent against 4.5 ms).
     int n_w = 0;
     for (int l = d; l < L; ++l) n_w += mask[2 * l] ? 1 : 0;
-    s->wgrad_one_unit = two && 2 * n_w <= L - d;
+    // Tile plan: the one made for a shared GPU whenever the two streams run (or on request, so that
+    // per-kernel timing on one stream can time the very kernels the two-stream step launches).
+    s->shared_plan = s->opt_tile_plan == ET_TILE_PLAN_SHARED || (s->opt_tile_plan == ET_TILE_PLAN_AUTO && two);
+    s->wgrad_one_unit = s->shared_plan && 2 * n_w <= L - d;
     // With a second stream the weight-gradient CTAs get their SMs in the gaps between the chain's
     // kernels; a chain kernel that took over each SM the moment its predecessor left would starve
     // them until the chain ends (measured: 2.45 -> 2.62 ms per ViT-B step), so no launch overlap then.
@@ -1065,12 +1085,13 @@ extern "C" {
 
 et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_dtype dtype, et_stack** out) {
   if (layers == nullptr || out == nullptr || L < 1 || L > 1024 || M < 1 || M > (1ll << 30)) return ET_ERR_INVALID_ARG;
+  // the column-sum kernels run one grid row per 128 rows of the activations: at most 65535 of them
+  if ((M + et::kColsumRows - 1) / et::kColsumRows > 65535) return ET_ERR_UNSUPPORTED;
   if (dtype != ET_F32 && dtype != ET_BF16) return ET_ERR_DTYPE;
   et_stack* s = new (std::nothrow) et_stack();
   if (s == nullptr) return ET_ERR_INVALID_ARG;
   s->L = L; s->M = M; s->dtype = dtype; s->elt = dtype == ET_BF16 ? 2 : 4;
   s->ly.resize(L);
-  s->overlap_launch = getenv("ET_NO_LAUNCH_OVERLAP") == nullptr;
   {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) == cudaSuccess &&
@@ -1144,7 +1165,13 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
 
   // ---- workspace layout
   size_t off = 0;
-  auto take = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
+  const bool guarded = g_guard_regions.load() != 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off += align256(bytes);
+    if (guarded) { s->guards.push_back(off); off += kGuardBytes; }   // a region's overrun lands here first
+    return o;
+  };
   s->off_status = take(256);
   size_t max_partial = 0;
   const int chunks = ceil_div(M, et::kColsumRows);
@@ -1180,7 +1207,8 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
       const TilePlan dsh = y.big_gemm ? choose_tiles((int)M, y.K, kb_n, s->sms, false, true, 0, true) : d;
       y.bn_dgrad_sh = dsh.bn; y.pair_dgrad_sh = dsh.pair;
       y.bn_wgrad = w.bn; y.pair_wgrad = w.pair; y.split = w.split;
-      if (const char* force = getenv("ET_DEBUG_TILES")) {          // debug: "<bn>,<pair>[,<split>]" for every GEMM
+#ifdef ET_DEBUG_HOOKS
+      if (const char* force = getenv("ET_DEBUG_TILES")) {          // debug builds only: "<bn>,<pair>[,<split>]" for every GEMM
         int fb = 0, fp = 0, fs = 0;
         if (sscanf(force, "%d,%d,%d", &fb, &fp, &fs) >= 2 && (fb == 128 || fb == 192 || fb == 256)) {
           y.bn_dgrad = fb; y.pair_dgrad = fp != 0;
@@ -1191,6 +1219,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
           if (fs > 0) y.split = std::min(fs, ceil_div(M, et::tc::BK));
         }
       }
+#endif
     }
     if (!y.trainable()) {                                  // no tensors: no partials, no importance slots
       y.imp_count_w = y.imp_count_b = 0;
@@ -1203,7 +1232,11 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     // takes the SMs they leave free (ViT-B full backprop 4.33 -> 4.02 ms; "as many splits as give every SM
     // pair a unit" gave 4.23 ms, a single split 4.59 ms).
     y.split_shared = y.split;
-    if (y.kind == ET_LAYER_DENSE && dtype == ET_BF16 && y.big_gemm && getenv("ET_DEBUG_TILES") == nullptr) {
+    bool forced_tiles = false;
+#ifdef ET_DEBUG_HOOKS
+    forced_tiles = getenv("ET_DEBUG_TILES") != nullptr;
+#endif
+    if (y.kind == ET_LAYER_DENSE && dtype == ET_BF16 && y.big_gemm && !forced_tiles) {
       const int kb = ceil_div(M, et::tc::BK);
       int sp = std::min(y.split, 2);
       while (sp > 1 && (long long)(sp - 1) * ceil_div(kb, sp) >= kb) --sp;
@@ -1238,6 +1271,26 @@ et_status et_stack_destroy(et_stack* s) {
   destroy_two_streams(s);
   delete s;
   return ET_OK;
+}
+
+et_status et_stack_set_option(et_stack* s, int32_t option, int32_t value) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  switch (option) {
+    case ET_OPTION_TWO_STREAMS:
+      if (value != 0 && value != 1) return ET_ERR_INVALID_ARG;
+      s->opt_two_streams = value != 0;
+      return ET_OK;
+    case ET_OPTION_LAUNCH_OVERLAP:
+      if (value != 0 && value != 1) return ET_ERR_INVALID_ARG;
+      s->overlap_launch = value != 0;
+      return ET_OK;
+    case ET_OPTION_TILE_PLAN:
+      if (value != ET_TILE_PLAN_AUTO && value != ET_TILE_PLAN_ALONE && value != ET_TILE_PLAN_SHARED) return ET_ERR_INVALID_ARG;
+      s->opt_tile_plan = value;
+      return ET_OK;
+    default:
+      return ET_ERR_INVALID_ARG;
+  }
 }
 
 et_status et_stack_workspace_bytes(const et_stack* s, size_t* bytes) {
@@ -1279,6 +1332,7 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
     }
   }
   CU_TRY(cudaMemsetAsync(s->at(s->off_status), 0, 256, st));
+  for (size_t g : s->guards) CU_TRY(cudaMemsetAsync(s->at(g), kGuardByte, kGuardBytes, st));
   CU_TRY(cudaMemcpyAsync(s->at(s->off_imp_offs), s->imp_offs.data(), sizeof(int) * 2 * s->L, cudaMemcpyHostToDevice, st));
   CU_TRY(cudaMemcpyAsync(s->at(s->off_imp_counts), s->imp_counts.data(), sizeof(int) * 2 * s->L, cudaMemcpyHostToDevice, st));
   CU_TRY(cudaStreamSynchronize(st));     // the host vectors may be freed / changed afterwards
@@ -1542,6 +1596,7 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
       if (!s->ly[l].trainable()) ones[2 * l] = ones[2 * l + 1] = 0;
     ET_TRY(et_backward_elastic(s, dY, ones.data(), 2 * L, nullptr, nullptr, nullptr, 0, 0.f, nullptr, stream));
     s->chain_shares_gpu = false;                              // the launches below run one at a time
+    s->shared_plan = false;
     s->wgrad_one_unit = false;
     float* scratch_grad = (float*)s->at(s->off_partial);      // in-place: each element is read before it is written
     double pending_nontrainable = 0.0;
@@ -1648,6 +1703,29 @@ et_status et_timing_read(et_stack* s, double* ms, int64_t* launches) {
   return rc;
 }
 
+et_status et_debug_guard_regions(int32_t on) {
+  g_guard_regions.store(on != 0 ? 1 : 0);
+  return ET_OK;
+}
+
+et_status et_debug_check_guards(et_stack* s, void* stream, int32_t* first_bad_region) {
+  if (s == nullptr) return ET_ERR_INVALID_ARG;
+  if (!s->bound) return ET_ERR_STATE;
+  if (first_bad_region != nullptr) *first_bad_region = -1;
+  if (s->guards.empty()) return ET_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  std::vector<unsigned char> host(s->guards.size() * kGuardBytes);
+  for (size_t i = 0; i < s->guards.size(); ++i)
+    CU_TRY(cudaMemcpyAsync(host.data() + i * kGuardBytes, s->at(s->guards[i]), kGuardBytes, cudaMemcpyDeviceToHost, st));
+  CU_TRY(cudaStreamSynchronize(st));
+  for (size_t i = 0; i < host.size(); ++i)
+    if (host[i] != kGuardByte) {
+      if (first_bad_region != nullptr) *first_bad_region = (int32_t)(i / kGuardBytes);
+      return ET_ERR_GUARD;
+    }
+  return ET_OK;
+}
+
 et_status et_device_status(et_stack* s, void* stream) {
   if (s == nullptr) return ET_ERR_INVALID_ARG;
   if (!s->bound) return ET_ERR_STATE;
@@ -1670,6 +1748,7 @@ const char* et_status_string(et_status st) {
     case ET_ERR_CUDA: return "CUDA call failed";
     case ET_ERR_TIMEOUT: return "device-side wait timed out";
     case ET_ERR_TOO_LARGE: return "problem exceeds the built-in scratch capacity of the no-allocation call";
+    case ET_ERR_GUARD: return "a guard word after a workspace region was overwritten";
   }
   return "unknown status";
 }

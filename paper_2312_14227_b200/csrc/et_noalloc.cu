@@ -1,8 +1,6 @@
 // et_bias_grad_noalloc: the bias gradient (column sums of an error-gradient matrix) for callers
 // that cannot allocate device memory.  The scratch that the two-stage reduction needs lives in a
 // fixed array inside the library image instead of in a caller-provided workspace.
-#include <mutex>
-
 #include <cuda_runtime.h>
 
 #include "et.h"
@@ -14,25 +12,18 @@ namespace {
 // library, held until the process exits.
 static __device__ __align__(256) float g_noalloc_scratch[ET_NOALLOC_SCRATCH_FLOATS];
 
-constexpr int kMaxDevices = 64;
-std::mutex g_setup_mutex;
-float* g_scratch_addr[kMaxDevices] = {nullptr};
-
-// In host code `g_noalloc_scratch` is only a handle for the symbol; the address a kernel can
-// use has to be asked for, once per device, with that device current.
+// In host code `g_noalloc_scratch` is only a handle for the symbol; the address a kernel can use
+// has to be asked for with the device current.  It is asked for on every call and never cached:
+// once the module is loaded the lookup is a host-side table read, while a remembered address
+// would go stale if the embedding application reset the device or made another context current
+// (a kernel given a stale address faults instead of returning a status).
 et_status scratch_for_current_device(float** out) {
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ET_ERR_CUDA;
-  std::lock_guard<std::mutex> lock(g_setup_mutex);
-  if (g_scratch_addr[dev] == nullptr) {
-    float* p = nullptr;
-    if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
-      (void)cudaGetLastError();
-      return ET_ERR_CUDA;
-    }
-    g_scratch_addr[dev] = p;
+  float* p = nullptr;
+  if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
+    (void)cudaGetLastError();
+    return ET_ERR_CUDA;
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return ET_OK;
 }
 
@@ -58,6 +49,7 @@ extern "C" et_status et_bias_grad_noalloc(const void* dZ, int64_t M, int32_t wid
   if (dtype != ET_F32 && dtype != ET_BF16) return ET_ERR_DTYPE;
   const int64_t chunks = (M + et::kColsumRows - 1) / et::kColsumRows;
   if (chunks * (int64_t)width > (int64_t)ET_NOALLOC_SCRATCH_FLOATS) return ET_ERR_TOO_LARGE;
+  if (chunks > 65535) return ET_ERR_TOO_LARGE;     // one grid row per chunk (narrow matrices with millions of rows)
   float* scratch = nullptr;
   et_status st = scratch_for_current_device(&scratch);
   if (st != ET_OK) return st;

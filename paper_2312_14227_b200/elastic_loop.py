@@ -82,26 +82,3 @@ class ElasticLoop:
         out["losses"] = losses.cpu().numpy().astype(np.float64)
         return out
 
-
-def flop_costs(layers, M):
-    """Per-tensor cost vectors proportional to the work of each backward operation
-    (kernel: 2*M*K*N for both the weight gradient and the error gradient; bias: M*N and 0),
-    for when measured times are not wanted."""
-    t_dw, t_dy = [], []
-    for ly in layers:
-        if getattr(ly, "kind", 0) in (2, 3):
-            # a layer without tensors: its backward work, one pass over its rows here, is charged to the
-            # bias below it by the caller's cost vectors; as a stand-in its own slots cost nothing
-            t_dw += [0.0, 0.0]
-            t_dy += [0.0, 0.0]
-            continue
-        if getattr(ly, "kind", 0) in (1, 4):
-            # normalisation layer: one pass over the rows, all of it charged to beta's error-gradient
-            # time (Section 5.2)
-            t_dw += [0.0, 0.0]
-            t_dy += [0.0, 8.0 * M * ly.out_features]
-            continue
-        f = 2.0 * M * ly.in_features * ly.out_features
-        t_dw += [f, float(M * ly.out_features)]
-        t_dy += [f, 0.0]
-    return np.array(t_dw), np.array(t_dy)

@@ -9,13 +9,11 @@ if ROOT not in sys.path:
 
 
 def _ensure_library():
-    """Build libet.so in-tree if it is missing or stale (run as a script: importing the
-    package itself needs the library)."""
+    """Build libet.so in-tree if it is missing or older than its sources (the build script compares
+    modification times itself and returns at once when the library is fresh; it is run as a script
+    because importing the package needs the library)."""
     import subprocess
     script = os.path.join(ROOT, "paper_2312_14227_b200", "build.py")
-    lib = os.path.join(ROOT, "paper_2312_14227_b200", "libet.so")
-    if os.path.exists(lib):
-        return
     subprocess.run([sys.executable, script], check=True, capture_output=True)
 
 

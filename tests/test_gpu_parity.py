@@ -42,6 +42,10 @@ def test_importance_of_a_gradient_step_fp32_and_bf16():
     w = wl.vit_b(seed=12, p_select=0.5, n_blocks=2, tokens=520, d=256, ffn=768)
     w.mask[:] = 1
     h.check_step(w, w.mask, TOL_BF16, aligned_delta=True)
+    # the same through the snapshot form of the call (dw = W - snapshot formed on the fly)
+    c = h.StepChecker(w, TOL_BF16)
+    c.check(w.mask, aligned_delta=True, snapshot=True)
+    c.check(w.mask, snapshot=True)
 
 
 def _all_kinds_layers(scale=1):
@@ -160,7 +164,12 @@ def test_bf16_resnet_1x1_config():
     w = wl.resnet_1x1()
     # He-initialised weights reach 0.5 and gradients reach 35 here: a bf16 store alone is
     # off by up to 2^-9 |w| ~ 1e-3, so the weight bound is the derived one
-    h.check_step(w, w.mask, TOL_BF16, derived_w_tol=True)
+    c = h.StepChecker(w, TOL_BF16)
+    stats = {}
+    c.check(w.mask, derived_w_tol=True, stats=stats)
+    # Eq. 2 with the update a gradient step makes (dw = -c g): plain relative error of every importance
+    c.check(w.mask, derived_w_tol=True, stats=stats, aligned_delta=True)
+    print("resnet_1x1 parity diagnostics", stats)
 
 
 def test_bf16_deterministic():
@@ -180,14 +189,73 @@ def test_bf16_deterministic():
     assert torch.equal(outs[0][1], outs[1][1])
 
 
-def test_bf16_vit_b_full_size_config():
+@pytest.fixture(scope="module")
+def vit_b_checker():
+    """The benchmark configuration (12 blocks, 12608 tokens) bound once: the oracle's forward pass of
+    the whole stack takes about half a minute and does not depend on the mask."""
+    c = _h().StepChecker(wl.vit_b(), TOL_BF16)
+    yield c
+    del c
+    torch.cuda.empty_cache()
+
+
+def test_bf16_vit_b_full_size_config(vit_b_checker):
     """The benchmark configuration itself (12 blocks, 12608 tokens, Bernoulli(0.3) mask),
-    launched exactly as bench.py launches it, against the full oracle."""
-    h = _h()
-    w = wl.vit_b()
+    launched exactly as bench.py launches it, against the full oracle; the importances both for a
+    random dw (bound relative to ||g||_inf ||dw||_2) and for dw = -c g (plain relative error)."""
+    c = vit_b_checker
     stats = {}
-    h.check_step(w, w.mask, TOL_BF16, stats=stats)
-    print("vit_b worst gradient error", stats)
+    c.check(c.w.mask, stats=stats)
+    c.check(c.w.mask, stats=stats, aligned_delta=True)
+    print("vit_b parity diagnostics", stats)
+
+
+def test_bf16_vit_b_full_size_selector_masks(vit_b_checker):
+    """Masks chosen by the host selector (Section 6, Eq. 3) at time budgets rho of the full backward
+    pass on per-tensor times measured on this stack, seeded Uniform(0,1) importances, T_fwd = 0,
+    T_q = 1000: every mask runs at full size and matches the oracle."""
+    c = vit_b_checker
+    run, w = c.run, c.w
+    t_dw, t_dy, t_fwd = et.et_profile_costs(run.stack, run.x, run.y, run.dY, iters=5)
+    run.forward_loss()
+    assert t_fwd > 0 and (t_dy[1::2] == 0).all() and t_dy[0] == 0 and (t_dw > 0).all() and (t_dy[2::2] > 0).all()
+    I = np.random.default_rng(9).random(2 * w.L)
+    total = t_dw.sum() + t_dy.sum()
+    prev, stats = -1, {}
+    for rho in (0.25, 0.5, 1.0):
+        mask, val, est = et.et_select_dp(I, t_dw, t_dy, 0.0, rho, 1000, et.ET_COST_STRICT)
+        assert est <= rho * total * 1.03
+        assert mask.sum() >= prev
+        prev = int(mask.sum())
+        if rho == 1.0:
+            assert mask.all()
+        assert mask.any()
+        rep = c.check(mask, stats=stats)
+        print(f"rho={rho}: {prev} tensors, deepest layer {rep.deepest}, estimated {est:.3f} ms of {total:.3f} ms")
+    print("vit_b selector-mask parity diagnostics", stats)
+
+
+def test_bf16_vit_l_shapes_snapshot_importance_and_master_weights():
+    """The shapes of the elastic-schedule configuration (d = 1024, FFN 4096, QKV 3072, 6304 tokens; 4 of
+    its 24 blocks: tile plans depend on widths and rows, not on depth), driven the way the schedule
+    drives them: fp32 master weights, importances from the weight change since a snapshot (Section 3.1).
+    One all-tensor step as in the window, one step with a selector mask at rho = 0.4."""
+    h = _h()
+    full = wl.vit_l(params=False)
+    w = wl.vit_l(n_blocks=4)
+    assert w.M == full.M and [(l.in_features, l.out_features) for l in w.layers] == \
+        [(l.in_features, l.out_features) for l in full.layers[:w.L]]
+    c = h.StepChecker(w, TOL_BF16, master=True)
+    stats = {}
+    ones = np.ones(2 * w.L, dtype=np.uint8)
+    c.check(ones, snapshot=True, stats=stats)
+    c.check(ones, snapshot=True, aligned_delta=True, stats=stats)
+    t_dw, t_dy = wl.flop_costs(w.layers, w.M)
+    I = np.random.default_rng(10).random(2 * w.L)
+    mask, _, _ = et.et_select_dp(I, t_dw, t_dy, 0.0, 0.4, 1000, et.ET_COST_STRICT)
+    assert mask.any() and not mask.all()
+    c.check(mask, snapshot=True, stats=stats)
+    print("vit_l-shape parity diagnostics", stats)
 
 
 def test_device_status_reports_a_recorded_timeout():

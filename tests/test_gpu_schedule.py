@@ -6,7 +6,8 @@ import pytest
 import torch
 
 import paper_2312_14227_b200 as et
-from paper_2312_14227_b200.elastic_loop import ElasticLoop, flop_costs
+from paper_2312_14227_b200.elastic_loop import ElasticLoop
+from workloads import flop_costs
 import workloads as wl
 from oracle import elastic_oracle as orc
 

@@ -223,3 +223,45 @@ def test_resolution_sweep_converges():
         value.append(val)
     assert overrun[-1] < 1e-3 and overrun[-1] <= overrun[0] + 1e-12
     assert abs(value[-1] - value[-2]) <= 0.02 * value[-1]
+
+
+# ------------------------------------------------------------------ options, guard words, no-allocation call (host side)
+def test_stack_options_are_validated():
+    s = et.et_stack_create([(8, 16, 0, 1, -1)], 4, et.ET_F32)
+    et.et_stack_set_option(s, et.ET_OPTION_TWO_STREAMS, 0)
+    et.et_stack_set_option(s, et.ET_OPTION_LAUNCH_OVERLAP, 0)
+    et.et_stack_set_option(s, et.ET_OPTION_TILE_PLAN, et.ET_TILE_PLAN_SHARED)
+    for opt, val in ((et.ET_OPTION_TWO_STREAMS, 2), (et.ET_OPTION_TILE_PLAN, 7), (99, 0)):
+        with pytest.raises(et.EtError) as e:
+            et.et_stack_set_option(s, opt, val)
+        assert e.value.status == et.ET_ERR_INVALID_ARG
+
+
+def test_guard_words_enlarge_the_workspace_and_need_a_bound_stack():
+    layers = [(8, 16, 1, 1, -1), (16, 8, 0, 1, 0)]
+    plain = et.et_stack_workspace_bytes(et.et_stack_create(layers, 4, et.ET_F32))
+    et.et_debug_guard_regions(True)
+    try:
+        guarded = et.et_stack_create(layers, 4, et.ET_F32)
+    finally:
+        et.et_debug_guard_regions(False)
+    extra = et.et_stack_workspace_bytes(guarded) - plain
+    assert extra > 0 and extra % 256 == 0                          # 256 guard bytes after every region
+    assert et.et_stack_workspace_bytes(et.et_stack_create(layers, 4, et.ET_F32)) == plain   # the switch is off again
+    st, bad = et.et_debug_check_guards(guarded)
+    assert st == et.ET_ERR_STATE and bad == -1                     # nothing bound yet: nothing to read
+
+
+def test_create_refuses_more_rows_than_the_column_sum_grid_holds():
+    assert _err([(8, 16, 0, 1, -1)], M=65535 * 128 + 1) == et.ET_ERR_UNSUPPORTED
+    et.et_stack_create([(8, 16, 0, 1, -1)], 65535 * 128, et.ET_F32)
+
+
+def test_noalloc_argument_checks_come_before_any_device_work():
+    x = np.zeros(4, dtype=np.float32)        # any non-null address: refused calls dereference nothing
+    for M, width, dtype, want in ((0, 8, et.ET_F32, et.ET_ERR_INVALID_ARG), (8, 8, 5, et.ET_ERR_DTYPE),
+                                  (128 * (et.ET_NOALLOC_SCRATCH_FLOATS // 4096) + 1, 4096, et.ET_F32, et.ET_ERR_TOO_LARGE),
+                                  (65535 * 128 + 1, 8, et.ET_F32, et.ET_ERR_TOO_LARGE)):
+        with pytest.raises(et.EtError) as e:
+            et.et_bias_grad_noalloc(x, M, width, dtype, x)
+        assert e.value.status == want, (M, width)

@@ -65,3 +65,19 @@ def test_noalloc_rejects_sizes_beyond_the_builtin_scratch():
     with pytest.raises(et.EtError) as e:
         et.et_bias_grad_noalloc(dummy, 0, width, wl.DT_F32, dummy)
     assert e.value.status == et.ET_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("M,width", [(12608, 3072), (128 * 256, 4096)])
+def test_noalloc_bias_grad_up_to_the_whole_scratch(M, width):
+    # 99 and 256 chunks of partial sums: the finishing kernel's strided loop over more than 32 chunks, and
+    # (second shape) a problem that fills the built-in array to its last float
+    assert -(-M // 128) * width <= et.ET_NOALLOC_SCRATCH_FLOATS
+    gen = torch.Generator(device="cpu").manual_seed(99)
+    dY = torch.randn((M, width), generator=gen).to(torch.bfloat16).to(DEV).contiguous()
+    got = torch.full((width,), float("nan"), dtype=torch.float32, device=DEV)
+    et.et_bias_grad_noalloc(dY, M, width, wl.DT_BF16, got)
+    torch.cuda.synchronize()
+    direct = dY.double().sum(dim=0)
+    assert float((got.double() - direct).abs().max()) <= 1e-4 * float(direct.abs().max())
+    want = _reference_bias_grad(dY, wl.DT_BF16)
+    assert float((got - want).abs().max()) <= 1e-5 * float(want.abs().max())

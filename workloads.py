@@ -362,3 +362,24 @@ def draw_delta(w: Workload, seed: int, std: float = 1e-3):
         out.append(_store(rng.normal(0.0, std, size=shape), w.dtype))
         out.append(_store(rng.normal(0.0, std, size=ly.out_features), w.dtype))
     return out
+
+
+def flop_costs(layers, M: int):
+    """Per-tensor cost vectors (t_dw, t_dy) proportional to the work of each backward operation, for
+    selector inputs when measured times are not wanted: a kernel costs 2*M*K*N for its weight gradient
+    and as much for passing the error gradient on, a bias M*N and 0 (Section 5.1); a normalisation layer
+    is one pass over its rows, all of it charged to beta's error-gradient time (Section 5.2); layers
+    without tensors have empty slots that cost nothing."""
+    t_dw, t_dy = [], []
+    for ly in layers:
+        if ly.kind in (KIND_ATTENTION, KIND_IM2COL):
+            t_dw += [0.0, 0.0]
+            t_dy += [0.0, 0.0]
+        elif ly.kind in (KIND_NORM, KIND_BATCHNORM):
+            t_dw += [0.0, 0.0]
+            t_dy += [0.0, 8.0 * M * ly.out_features]
+        else:
+            f = 2.0 * M * ly.in_features * ly.out_features
+            t_dw += [f, float(M * ly.out_features)]
+            t_dy += [f, 0.0]
+    return np.array(t_dw), np.array(t_dy)
