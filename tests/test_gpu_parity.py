@@ -216,6 +216,8 @@ def test_bf16_vit_b_full_size_selector_masks(vit_b_checker):
     T_q = 1000: every mask runs at full size and matches the oracle."""
     c = vit_b_checker
     run, w = c.run, c.w
+    c._restore()         # the profiler re-runs the forward pass: it must see the weights the oracle has,
+                         # not the ones the previous check's fused update left behind
     t_dw, t_dy, t_fwd = et.et_profile_costs(run.stack, run.x, run.y, run.dY, iters=5)
     run.forward_loss()
     assert t_fwd > 0 and (t_dy[1::2] == 0).all() and t_dy[0] == 0 and (t_dw > 0).all() and (t_dy[2::2] > 0).all()
@@ -224,7 +226,12 @@ def test_bf16_vit_b_full_size_selector_masks(vit_b_checker):
     prev, stats = -1, {}
     for rho in (0.25, 0.5, 1.0):
         mask, val, est = et.et_select_dp(I, t_dw, t_dy, 0.0, rho, 1000, et.ET_COST_STRICT)
-        assert est <= rho * total * 1.03
+        # Eq. 8 floors every time to a multiple of total / T_q, so each term the selector adds up may be
+        # under-estimated by less than one quantum: the true time of a feasible mask exceeds the budget by
+        # at most one quantum per selected tensor (t_dw) plus one per layer above the deepest (t_dy)
+        deepest = int(np.flatnonzero(mask)[0]) // 2
+        terms = int(mask.sum()) + (w.L - 1 - deepest)
+        assert est <= rho * total + terms * total / 1000
         assert mask.sum() >= prev
         prev = int(mask.sum())
         if rho == 1.0:
