@@ -58,18 +58,21 @@ def tensor_fracs(tf: float, peaks: dict) -> dict:
             "of_nominal_dense": tf / NOMINAL_BF16_TFLOPS}
 
 
-def _dgrad_traffic():
-    """DRAM bytes per dgrad launch from the committed ncu capture, or None once the GEMM sources
-    have changed since the counters were taken."""
+def _list_traffic(blocks: int):
+    """DRAM bytes of one gemm_list_kernel launch from the committed ncu capture (taken on a reduced stack of the
+    same shapes, scaled by executed flops), or None once the GEMM sources have changed since the counters were
+    taken."""
     import hashlib
     try:
-        with open(os.path.join(ROOT, "profiles", "dgrad_dram_traffic.json")) as f:
+        with open(os.path.join(ROOT, "profiles", "gemm_list_dram_traffic.json")) as f:
             rec = json.load(f)
         h = hashlib.sha256()
-        for name in ("gemm_tc.cuh", "epilogue.cuh"):
+        for name in ("gemm_tc.cuh", "gemm_list.cuh", "epilogue.cuh"):
             with open(os.path.join(ROOT, "paper_2312_14227_b200", "csrc", name), "rb") as f:
                 h.update(f.read())
-        return rec["bytes_per_launch"] if h.hexdigest() == rec["source_sha256"] else None
+        if h.hexdigest() != rec["source_sha256"]:
+            return None
+        return rec["bytes_per_tflop"] * rec["tflop_of_benchmark_step"] if blocks == 12 else None
     except (OSError, KeyError, ValueError):
         return None
 
@@ -247,6 +250,8 @@ def run_own(args):
         return torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()
 
     stack = et.et_stack_create(w.layers, w.M, w.dtype)
+    if args.plain_launch:
+        et.et_stack_set_option(stack, et.ET_OPTION_LIST_COOPERATIVE, 0)
     W = [to_dev(a) for a in w.W]
     b = [to_dev(a) for a in w.b]
     ws = torch.empty(et.et_stack_workspace_bytes(stack), dtype=torch.uint8, device=dev)
@@ -325,62 +330,75 @@ def run_own(args):
     e2e_value = aggregate_value(flops, e2e_ms, world)
     clocks = sampler.stop()     # sampled from the full-backprop run to the end of the end-to-end run
 
-    # per-kernel-class device time over the same steps (event pair around every launch; while
-    # this is on, the library keeps all kernels on one stream so that a pair brackets one kernel).
-    # Taken twice: with the tile plan the two-stream step above really launches ("shared": tile shapes
-    # chosen for a GPU shared between the chain and the weight gradients) and with the plan a
-    # single-stream caller gets ("alone").
+    # Device time per kernel class (a CUDA-event pair around every launch, recorded by the library on the
+    # launching stream over the same steps).  The timed step above runs every GEMM of the pass in ONE
+    # cooperative launch (gemm_list_kernel), followed by one grouped split reducer and one grouped bias
+    # finisher: that launch is the dominant kernel.  For comparison the same step is also timed launched GEMM by
+    # GEMM (the path stacks with other layer kinds take), as a two-stream step and class by class.
     peaks = _peaks()
     M = w.M
     first = next(l for l in range(w.L) if w.mask[2 * l] or w.mask[2 * l + 1])
     dgrad_flops = sum(2.0 * M * ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if l > first)
     wgrad_flops = sum(2.0 * M * ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if w.mask[2 * l])
     sel_params = sum(ly.in_features * ly.out_features for l, ly in enumerate(w.layers) if w.mask[2 * l])
-    # bytes the reducer must move per selected kernel tensor of P parameters: S*4P partial reads
-    # are its own scratch traffic; the algorithmic part is 4P (gradient) + 2P (dW) + 2P + 2P (W in/out)
+    # bytes the reducer must move per selected kernel tensor of P parameters: 4P (gradient) + 2P (dW) + 2P + 2P
+    # (W in / out); re-reading more than one split's partial sums is its own scratch traffic
     reduce_bytes = 10.0 * sel_params
 
-    def instrumented(plan):
-        et.et_stack_set_option(stack, et.ET_OPTION_TILE_PLAN, plan)
+    def classes_of(step_fn, n_steps):
         et.et_timing_enable(stack, True)
-        inst_ms, _ = timed(lambda: step(w.mask), args.steps, 1)
+        inst_ms, _ = timed(step_fn, n_steps, 1)
         classes = et.et_timing_read(stack)
         et.et_timing_enable(stack, False)
-        et.et_stack_set_option(stack, et.ET_OPTION_TILE_PLAN, et.ET_TILE_PLAN_AUTO)
-        n_rec = args.steps + 1          # the warm-up step is in the record too: normalise by recorded steps
+        n_rec = n_steps + 1             # the warm-up step is in the record too: normalise by recorded steps
+        return {k: (t / n_rec, n / n_rec) for k, (t, n) in classes.items()}, inst_ms
 
-        def per_step(cls):
-            t, n = classes[cls]
-            return t / n_rec, n / n_rec
+    def gb(ms_):
+        return reduce_bytes / (ms_ * 1e-3) / 1e9 if ms_ > 0 else 0.0
 
-        dg_ms, dg_n = per_step("dgrad")
-        wg_ms, wg_n = per_step("wgrad")
-        rd_ms, rd_n = per_step("wgrad_reduce")
-        bg_ms, bg_n = per_step("bgrad")
-        ot_ms, ot_n = per_step("other")
-        dg_tf = dgrad_flops / (dg_ms * 1e-3) / 1e12 if dg_ms > 0 else 0.0
-        wg_tf = wgrad_flops / (wg_ms * 1e-3) / 1e12 if wg_ms > 0 else 0.0
-        rd_gbs = reduce_bytes / (rd_ms * 1e-3) / 1e9 if rd_ms > 0 else 0.0
-        return {
-            "dgrad_gemm": {"launches_per_step": dg_n, "ms_per_step": dg_ms, "achieved": dg_tf, "unit": "TFLOP/s",
-                           "frac": tensor_fracs(dg_tf, peaks)},
-            "wgrad_gemm": {"launches_per_step": wg_n, "ms_per_step": wg_ms, "achieved": wg_tf, "unit": "TFLOP/s",
-                           "frac": tensor_fracs(wg_tf, peaks)},
-            "wgrad_reduce_importance_sgd": {"launches_per_step": rd_n, "ms_per_step": rd_ms, "achieved": rd_gbs,
-                                            "unit": "GB/s", "algorithmic_bytes_per_step": reduce_bytes,
-                                            "frac_of_hbm_peak": rd_gbs / peaks["hbm_gbs"]},
-            "bias_grad": {"launches_per_step": bg_n, "ms_per_step": bg_ms,
-                          "note": "finishing kernels only (the column sums come out of the dgrad epilogue): a few MB of "
-                                  "partials per step, latency-bound, reported as time"},
-            "other": {"launches_per_step": ot_n, "ms_per_step": ot_ms},
-            "instrumented_step_ms": inst_ms,
-        }
-
-    kernels = {"shared_plan": instrumented(et.ET_TILE_PLAN_SHARED), "alone_plan": instrumented(et.ET_TILE_PLAN_ALONE)}
-    kernels["note"] = ("shared_plan = the tile shapes the timed two-stream step launches; alone_plan = the shapes a "
-                       "single-stream caller gets; both timed one kernel at a time on one stream")
-    dg = kernels["shared_plan"]["dgrad_gemm"]
-    dg_tf = dg["achieved"]
+    cls, inst_ms = classes_of(lambda: step(w.mask), args.steps)
+    ls_ms, ls_n = cls["gemm_list"]
+    ls_tf = flops / (ls_ms * 1e-3) / 1e12 if ls_ms > 0 else 0.0
+    one_launch = {
+        "gemm_list": {"launches_per_step": ls_n, "ms_per_step": ls_ms, "achieved": ls_tf, "unit": "TFLOP/s",
+                      "flops_per_launch": flops, "frac": tensor_fracs(ls_tf, peaks),
+                      "what": "all %d error-gradient and %d weight-gradient GEMMs of the step as work units of one "
+                              "cooperative launch" % (int(rep.dgrad.sum()), int(rep.wgrad.sum()))},
+        "wgrad_reduce_importance_sgd": {"launches_per_step": cls["wgrad_reduce"][1], "ms_per_step": cls["wgrad_reduce"][0],
+                                        "achieved": gb(cls["wgrad_reduce"][0]), "unit": "GB/s",
+                                        "algorithmic_bytes_per_step": reduce_bytes,
+                                        "frac_of_hbm_peak": gb(cls["wgrad_reduce"][0]) / peaks["hbm_gbs"]},
+        "bias_grad": {"launches_per_step": cls["bgrad"][1], "ms_per_step": cls["bgrad"][0],
+                      "note": "top layer's column sums + one grouped finisher (the other column sums come out of the "
+                              "error-gradient epilogues): a few MB of partials per step, reported as time"},
+        "other": {"launches_per_step": cls["other"][1], "ms_per_step": cls["other"][0]},
+        "instrumented_step_ms": inst_ms,
+    }
+    # the same step, one launch per GEMM
+    et.et_stack_set_option(stack, et.ET_OPTION_GEMM_LIST, 0)
+    pl_ms, pl_launches = timed(lambda: step(w.mask), args.steps, args.warmup)
+    pl_full_ms, _ = timed(lambda: step(ones), max(2, args.steps // 4), 2)
+    et.et_stack_set_option(stack, et.ET_OPTION_TILE_PLAN, et.ET_TILE_PLAN_SHARED)
+    pcls, p_inst = classes_of(lambda: step(w.mask), max(2, args.steps // 4))
+    et.et_stack_set_option(stack, et.ET_OPTION_TILE_PLAN, et.ET_TILE_PLAN_AUTO)
+    et.et_stack_set_option(stack, et.ET_OPTION_GEMM_LIST, 1)
+    dg_tf = dgrad_flops / (pcls["dgrad"][0] * 1e-3) / 1e12 if pcls["dgrad"][0] > 0 else 0.0
+    wg_tf = wgrad_flops / (pcls["wgrad"][0] * 1e-3) / 1e12 if pcls["wgrad"][0] > 0 else 0.0
+    per_layer = {
+        "two_stream_step_ms": pl_ms, "two_stream_step_tflops": flops / (pl_ms * 1e-3) / 1e12,
+        "two_stream_full_backprop_ms": pl_full_ms, "launches_per_step": pl_launches / args.steps,
+        "dgrad_gemm": {"launches_per_step": pcls["dgrad"][1], "ms_per_step": pcls["dgrad"][0], "achieved": dg_tf,
+                       "unit": "TFLOP/s", "frac": tensor_fracs(dg_tf, peaks)},
+        "wgrad_gemm": {"launches_per_step": pcls["wgrad"][1], "ms_per_step": pcls["wgrad"][0], "achieved": wg_tf,
+                       "unit": "TFLOP/s", "frac": tensor_fracs(wg_tf, peaks)},
+        "wgrad_reduce_importance_sgd": {"launches_per_step": pcls["wgrad_reduce"][1], "ms_per_step": pcls["wgrad_reduce"][0],
+                                        "achieved": gb(pcls["wgrad_reduce"][0]), "unit": "GB/s",
+                                        "frac_of_hbm_peak": gb(pcls["wgrad_reduce"][0]) / peaks["hbm_gbs"]},
+        "bias_grad": {"launches_per_step": pcls["bgrad"][1], "ms_per_step": pcls["bgrad"][0]},
+        "note": "classes timed one kernel at a time on one stream (event pair per launch, which adds about 3 us to "
+                "each), with the tile shapes the two-stream step launches",
+    }
+    kernels = {"one_launch": one_launch, "per_layer": per_layer}
     timed_span_s = ms * args.steps * 1e-3
     use_burst = timed_span_s < 1.0
     peak = peaks["tf_burst"] if use_burst else peaks["tf_sustained"]
@@ -410,18 +428,18 @@ def run_own(args):
                 "h2d_bytes_per_step": dY_host.numel() * dY_host.element_size(),
                 "d2h_bytes_per_step": imp_host.numel() * 4},
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "gemm_tc_kernel<dgrad> (tile plan of the timed step)", "bound": "tensor",
-                     "achieved": dg_tf, "peak": peak, "unit": "TFLOP/s", "frac": dg_tf / peak,
+        "roofline": {"kernel": "gemm_list_kernel (every GEMM of the step in one cooperative launch)", "bound": "tensor",
+                     "achieved": ls_tf, "peak": peak, "unit": "TFLOP/s", "frac": ls_tf / peak,
                      "peak_source": peaks["source"] + (" cuBLAS bf16 burst" if use_burst else " cuBLAS bf16 sustained"),
                      "peak_choice": f"the timed region lasts {timed_span_s:.2f} s: " +
                                     ("burst peak (a kernel timed in a short run)" if use_burst else
                                      "sustained peak (a kernel timed inside a seconds-long step)"),
-                     "frac_all": tensor_fracs(dg_tf, peaks),
-                     "flops_per_step": dgrad_flops, "ms_per_step": dg["ms_per_step"],
-                     "launches_per_step": dg["launches_per_step"],
-                     "ms_x_sm_mhz": (dg["ms_per_step"] * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None,
-                     "traffic": _dgrad_traffic(),
-                     "traffic_note": "DRAM bytes per launch, mean over the dgrad GEMMs of one block (ncu, cold cache)"},
+                     "frac_all": tensor_fracs(ls_tf, peaks),
+                     "flops_per_launch": flops, "ms_per_launch": ls_ms, "launches_per_step": ls_n,
+                     "ms_x_sm_mhz": (ls_ms * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None,
+                     "traffic": _list_traffic(args.blocks),
+                     "traffic_note": "DRAM bytes per launch: ncu capture of the same launch on the 2-block stack "
+                                     "(same shapes and token count), scaled by the GEMM flops of this stack"},
         "kernels": kernels,
     }
     if world == 1:
@@ -741,6 +759,9 @@ def main():
     ap.add_argument("--blocks", type=int, default=12, help="transformer blocks of the stack (12 = the benchmark workload)")
     ap.add_argument("--profile", action="store_true",
                     help="short run for ncu: one forward and two all-selected backward steps, no timing")
+    ap.add_argument("--plain-launch", action="store_true",
+                    help="launch the one-launch backward as a plain (not cooperative) grid: for runs under a profiler, "
+                         "which does not take the cooperative launch")
     ap.add_argument("--optimizer", default="sgd", choices=["sgd", "sgdw", "adam"],
                     help="update fused into the step: plain SGD (the benchmark line) or the paper's SGDW / Adam")
     ap.add_argument("--workload", default="vit_b", choices=["vit_b", "dp_budget", "resnet", "prenorm", "full", "bottleneck", "bottleneck_bn", "schedule", "schedule_full", "selector"],

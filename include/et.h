@@ -160,8 +160,20 @@ et_status et_stack_destroy(et_stack* s);
  *   ET_OPTION_TILE_PLAN      ET_TILE_PLAN_AUTO (default): GEMM tile shapes made for a GPU shared by the two
  *                            streams when they run, for a GPU to itself otherwise; ET_TILE_PLAN_ALONE /
  *                            ET_TILE_PLAN_SHARED force one (per-kernel timing keeps kernels on one stream and
- *                            can still time the shapes the two-stream step launches). */
-typedef enum { ET_OPTION_TWO_STREAMS = 1, ET_OPTION_LAUNCH_OVERLAP = 2, ET_OPTION_TILE_PLAN = 3 } et_option;
+ *                            can still time the shapes the two-stream step launches).
+ *   ET_OPTION_GEMM_LIST      1 (default): where every layer from the deepest selected one upwards is a dense layer
+ *                            with widths that are multiples of 64 (bf16 stacks), et_backward_elastic runs all
+ *                            error-gradient and weight-gradient GEMMs of the call as ONE cooperative launch whose
+ *                            work units wait on one another row tile by row tile, followed by one grouped launch
+ *                            for the split reductions (gradient export, Eq. 2, update) and one for the bias
+ *                            gradients; 0: one launch per GEMM (the path other stacks always take).
+ *   ET_OPTION_LIST_COOPERATIVE 1 (default): that launch is a cooperative one, which is what guarantees that all its
+ *                            CTAs are resident while they wait on one another.  0: a plain launch of the same grid,
+ *                            for a profiler that does not take cooperative launches; only safe while nothing else
+ *                            runs on the GPU (every CTA then becomes resident at once because the grid is sized to
+ *                            the device). */
+typedef enum { ET_OPTION_TWO_STREAMS = 1, ET_OPTION_LAUNCH_OVERLAP = 2, ET_OPTION_TILE_PLAN = 3,
+               ET_OPTION_GEMM_LIST = 4, ET_OPTION_LIST_COOPERATIVE = 5 } et_option;
 typedef enum { ET_TILE_PLAN_AUTO = 0, ET_TILE_PLAN_ALONE = 1, ET_TILE_PLAN_SHARED = 2 } et_tile_plan;
 et_status et_stack_set_option(et_stack* s, int32_t option, int32_t value);
 
@@ -400,7 +412,8 @@ typedef enum {
   ET_K_OTHER = 5,          /* loss gradient, top-layer activation backward, importance finalise */
   ET_K_NORM = 6,           /* normalisation layers: forward, backward (error gradient + d gamma), gamma finish */
   ET_K_ATTENTION = 7,      /* layers without tensors: attention core, patch gather; forward, backward */
-  ET_K_CLASSES = 8
+  ET_K_LIST = 8,           /* the one-launch backward: every dgrad and wgrad GEMM of a call in one kernel */
+  ET_K_CLASSES = 9
 } et_kernel_class;
 
 /* on != 0: every kernel this stack launches from now on is bracketed by a pair of CUDA

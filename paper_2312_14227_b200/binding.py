@@ -272,7 +272,8 @@ def et_stack_destroy(s: Stack):
     s.close()
 
 
-ET_OPTION_TWO_STREAMS, ET_OPTION_LAUNCH_OVERLAP, ET_OPTION_TILE_PLAN = 1, 2, 3
+ET_OPTION_TWO_STREAMS, ET_OPTION_LAUNCH_OVERLAP, ET_OPTION_TILE_PLAN, ET_OPTION_GEMM_LIST = 1, 2, 3, 4
+ET_OPTION_LIST_COOPERATIVE = 5
 ET_TILE_PLAN_AUTO, ET_TILE_PLAN_ALONE, ET_TILE_PLAN_SHARED = 0, 1, 2
 
 
@@ -382,7 +383,7 @@ def et_profile_costs(s: Stack, x, y, dY, iters: int = 20, stream=None):
     return t_dw, t_dy, t_fwd.value
 
 
-KERNEL_CLASSES = ("forward", "dgrad", "wgrad", "wgrad_reduce", "bgrad", "other", "norm", "attention")
+KERNEL_CLASSES = ("forward", "dgrad", "wgrad", "wgrad_reduce", "bgrad", "other", "norm", "attention", "gemm_list")
 
 
 def et_timing_enable(s: Stack, on: bool):

@@ -17,6 +17,7 @@
 #include "et.h"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_list.cuh"
 #include "kernels.cuh"
 #include "norm.cuh"
 #include "attn.cuh"
@@ -171,6 +172,11 @@ struct LayerRT {
   TMaps map_W, map_aout, map_Gout, map_Z, map_dZ;
   CUtensorMap map_Wd;       // W as the K-major B of the dgrad GEMM: one box = the CTA's whole B tile
   CUtensorMap map_Wd_sh;    // the same for the shared-GPU tile shape
+  CUtensorMap map_Wd_list;  // the same for the 256-wide pair tiles of the one-launch backward (128-row boxes)
+  int split_list = 1;       // wgrad contraction splits in the one-launch backward
+  size_t off_partial_list = 0;   // this layer's own split partials there (kept until the grouped reducer runs)
+  bool list_ok = false;     // shapes the one-launch backward takes (bf16 dense layer, widths multiples of 64)
+  int split_now = 1;        // per task list: splits of this layer's weight-gradient task
 };
 
 }  // namespace
@@ -204,6 +210,19 @@ struct et_stack {
   bool shared_plan = false;            // per call: the GEMMs use the tile plan made for that case
   bool opt_two_streams = true;         // et_stack_set_option
   int opt_tile_plan = ET_TILE_PLAN_AUTO;
+  bool opt_gemm_list = true;
+  bool opt_list_cooperative = true;
+  // one-launch backward: task list, dependency counters and the grouped reducers' tables (device, in the
+  // workspace) with the host copies they were last filled from
+  size_t off_tasks = 0, off_counters = 0, off_rtab = 0, off_btab = 0;
+  int max_counters = 0;
+  std::vector<et::tl::Task> tasks_host;
+  std::vector<uint8_t> tasks_key;      // mask and pointers the device task list was built for
+  int tasks_units = 0, tasks_counters = 0;
+  std::vector<et::ReduceEntry> rtab_host;
+  std::vector<et::BiasEntry> btab_host;
+  int list_state = 0;                  // 0 = untried, 1 = works, -1 = the cooperative launch was refused: per-layer path
+  unsigned bind_serial = 0;
   // second stream: the error-gradient chain runs here while weight gradients run on the caller's
   cudaStream_t chain_stream = nullptr;
   std::vector<cudaEvent_t> chain_ev;   // [l] = dgrad(l) finished; [L] = top-layer dZ ready; [L+1] = join
@@ -896,6 +915,299 @@ void destroy_two_streams(et_stack* s) {
   s->fork_ev = nullptr; s->chain_stream = nullptr; s->two_streams = -1;
 }
 
+// ---- one-launch backward -----------------------------------------------------------------------
+// CTA pairs of gemm_list_kernel that fit on the current device at once (0 if that cannot be found out).
+int list_max_clusters(int sms) {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return 0; }
+  std::lock_guard<std::mutex> cache_lock(g_cache_mutex);
+  if (cached[dev] == 0) {
+    cached[dev] = -1;
+    auto kern = et::tl::gemm_list_kernel;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)et::tl::LSMEM_BYTES) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cudaLaunchAttribute attr[1];
+      cfg.gridDim = dim3(sms & ~1); cfg.blockDim = dim3(et::tc::THREADS); cfg.dynamicSmemBytes = et::tl::LSMEM_BYTES;
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n >= 1) cached[dev] = n;
+    }
+    (void)cudaGetLastError();
+  }
+  return cached[dev] > 0 ? cached[dev] : 0;
+}
+
+// The epilogue dgrad(l) needs, as the list kernel has it: one input chunk (skip gradient, or Z of the layer
+// below) and one output (G_l, or dZ_{l-1}).  False when both G_l and dZ_{l-1} must be stored.
+bool list_dgrad_form(const et_stack* s, int l, bool* has_in, bool* mul_act) {
+  const LayerRT& Y = s->ly[l];
+  const LayerRT& P = s->ly[l - 1];
+  const bool need_skip = Y.consumer >= 0;
+  const bool need_act = P.act != ET_ACT_NONE;
+  const bool need_G = !need_act || P.residual_src >= 0;
+  if (!need_act) { *has_in = need_skip; *mul_act = false; return true; }
+  if (!need_skip && !need_G) { *has_in = true; *mul_act = true; return true; }
+  return false;
+}
+bool list_eligible(const et_stack* s, int d) {
+  if (s->dtype != ET_BF16 || !s->opt_gemm_list || s->list_state < 0) return false;
+  for (int l = d; l < s->L; ++l)
+    if (!s->ly[l].list_ok) return false;
+  for (int l = d + 1; l < s->L; ++l) {
+    bool a, b;
+    if (!list_dgrad_form(s, l, &a, &b)) return false;
+  }
+  return list_max_clusters(s->sms) > 0;
+}
+
+// Every GEMM of the pass as one task list and one cooperative launch of gemm_list_kernel, then one grouped
+// launch each for the split reductions and the bias finishers.  *refused: the device would not take the
+// cooperative launch; nothing of the pass has been changed, the caller runs the per-layer path instead.
+et_status backward_list(et_stack* s, const void* dY, const uint8_t* mask, float* const* grads,
+                        const void* const* delta, bool sgd, float lr, int d, int* launches_out, double* flops_out,
+                        cudaStream_t st, bool* refused) {
+  namespace tl = et::tl;
+  const int L = s->L;
+  const long long M = s->M;
+  int launches = 0;
+  *refused = false;
+  const LayerRT& top = s->ly[L - 1];
+  if (top.act != ET_ACT_NONE) {
+    TimedLaunch tlch(s, ET_K_OTHER, st);
+    const size_t count = (size_t)M * top.N;
+    et::act_backward_kernel<bf16><<<ceil_div(count, et::kEltThreads * et::kVec), et::kEltThreads, 0, st>>>(
+        (const bf16*)dY, (const bf16*)s->at(top.off_Z), (bf16*)s->at(top.off_dZ), count, top.act);
+    ET_TRY(after_launch());
+    ++launches;
+  }
+  const int top_chunks = ceil_div(M, et::kColsumRows);
+  if (mask[2 * (L - 1) + 1]) {
+    TimedLaunch tlch(s, ET_K_BGRAD, st);
+    dim3 grid(ceil_div(top.Nw, 256), top_chunks), block(32, 8);
+    et::colsum_partial_kernel<bf16><<<grid, block, 0, st>>>(dz_src<bf16>(s, L - 1, dY), (int)M, top.Nw,
+                                                            (float*)s->at(top.off_biaspart));
+    ET_TRY(after_launch());
+    ++launches;
+  }
+
+  // ---- the task list (rebuilt only when the mask, dY or the binding changed)
+  std::vector<uint8_t> key(mask, mask + 2 * L);
+  {
+    const void* p = dY;
+    const unsigned serial = s->bind_serial;
+    key.insert(key.end(), (const uint8_t*)&p, (const uint8_t*)&p + sizeof(p));
+    key.insert(key.end(), (const uint8_t*)&serial, (const uint8_t*)&serial + sizeof(serial));
+    for (int l = d; l < L; ++l) {                 // the reduce tasks hold these pointers
+      if (!mask[2 * l]) continue;
+      const void* q[2] = {grads ? (const void*)grads[2 * l] : nullptr, delta ? delta[2 * l] : nullptr};
+      key.insert(key.end(), (const uint8_t*)q, (const uint8_t*)q + sizeof(q));
+    }
+    key.push_back(sgd ? 1 : 0);
+  }
+  const int tiles_m_tok = ceil_div(M, 2 * et::tc::BM);
+  if (key != s->tasks_key) {
+    std::vector<tl::Task>& tk = s->tasks_host;
+    tk.clear();
+    std::vector<int> sig_base(L + 1, -1), tiles_n_of(L + 1, 0);
+    int counters = 0, units = 0;
+    auto add_dgrad = [&](int l) {
+      const LayerRT& Y = s->ly[l];
+      const LayerRT& P = s->ly[l - 1];
+      tl::Task t;
+      std::memset(&t, 0, sizeof(t));
+      bool has_in = false, mul_act = false;
+      list_dgrad_form(s, l, &has_in, &mul_act);
+      t.kind = tl::kDgrad;
+      t.rows = (int)M; t.cols = Y.K;
+      t.tiles_m = tiles_m_tok; t.tiles_n = ceil_div(Y.K, tl::LBN); t.split = 1;
+      t.kb_per_seg = ceil_div(Y.Nw, et::tc::BK); t.kb_total = t.kb_per_seg * Y.fold; t.kb_per_split = t.kb_total;
+      t.b_k_seg_stride = Y.Nw; t.b_mn_wrap = 0;
+      t.map_a = dz_map(s, l).b128;
+      t.map_b = Y.map_Wd_list;
+      if (mul_act) { t.map_in = P.map_Z.b128; t.map_out = P.map_dZ.b128; }
+      else { t.map_in = has_in ? g_map(s, Y.consumer + 1).b128 : P.map_Gout.b128; t.map_out = P.map_Gout.b128; }
+      t.has_in = has_in ? 1 : 0; t.mul_act = mul_act ? 1 : 0; t.act_prev = P.act; t.ld = Y.K;
+      t.colsum = mask[2 * (l - 1) + 1] ? (float*)s->at(P.off_biaspart) : nullptr;
+      t.unit_begin = units; t.units = t.tiles_m * t.tiles_n; units += t.units;
+      t.wait_base = l + 1 <= L - 1 ? sig_base[l + 1] : -1; t.wait_per_row = 1;
+      t.wait_target = 4u * (unsigned)tiles_n_of[l + 1];
+      t.wait2_base = -1; t.wait2_target = 0;
+      if (!mul_act && has_in && Y.consumer + 1 <= L - 1) {
+        t.wait2_base = sig_base[Y.consumer + 1];
+        t.wait2_target = 4u * (unsigned)tiles_n_of[Y.consumer + 1];
+      }
+      t.signal_base = counters; sig_base[l] = counters; tiles_n_of[l] = t.tiles_n;
+      counters += t.tiles_m + 1;
+      tk.push_back(t);
+    };
+    auto add_wgrad = [&](int l) {
+      const LayerRT& Y = s->ly[l];
+      tl::Task t;
+      std::memset(&t, 0, sizeof(t));
+      t.kind = tl::kWgrad;
+      t.rows = Y.K; t.cols = Y.N;
+      t.tiles_m = ceil_div(Y.K, 2 * et::tc::BM); t.tiles_n = ceil_div(Y.N, tl::LBN); t.split = s->ly[l].split_now;
+      t.kb_per_seg = ceil_div(M, et::tc::BK); t.kb_total = t.kb_per_seg; t.kb_per_split = ceil_div(t.kb_total, t.split);
+      t.b_k_seg_stride = 0; t.b_mn_wrap = Y.fold > 1 ? Y.Nw : 0;
+      t.map_a = a_map(s, l).c3[0];
+      t.map_b = dz_map(s, l).c3[0];
+      t.map_in = t.map_a; t.map_out = t.map_a;                 // unused by this kind
+      t.partial = (float*)s->at(Y.off_partial_list); t.split_stride = (unsigned long long)Y.K * Y.N; t.ld_out = Y.N;
+      t.unit_begin = units; t.units = t.tiles_m * t.tiles_n * t.split; units += t.units;
+      t.wait_base = -1; t.wait_per_row = 0; t.wait_target = 0;
+      if (l + 1 <= L - 1) {                                    // dZ_l is complete once every unit of dgrad(l+1) is
+        t.wait_base = sig_base[l + 1] + tiles_m_tok;
+        t.wait_target = 4u * (unsigned)tiles_m_tok * (unsigned)tiles_n_of[l + 1];
+      }
+      t.wait2_base = -1; t.signal_base = -1;
+      tk.push_back(t);
+    };
+    // Order: the whole error-gradient chain first, then the weight gradients.  (Interleaved, a CTA busy with a
+    // long weight-gradient unit holds up the chain units queued behind it and every row tile below them;
+    // measured on the ViT-B- and ViT-L-shaped stacks the chain-first list is 2 to 10 % faster, on the narrow 1x1
+    // convolution stack the two orders tie.)
+    // Contraction splits: with the chain out of the way a weight gradient runs unsplit, so that its partial sum
+    // is the gradient and nothing is written and read twice; the last two of the list are cut into shorter
+    // units so that the launch does not end on a few CTAs working through 200-k-block units while the rest idle.
+    std::vector<int> sel;                                      // selected kernels, top first
+    for (int l = L - 1; l >= d; --l)
+      if (mask[2 * l]) sel.push_back(l);
+    for (size_t i = 0; i < sel.size(); ++i)
+      s->ly[sel[i]].split_now = i + 2 < sel.size() ? 1 : s->ly[sel[i]].split_list;
+    for (int l = L - 1; l > d; --l) add_dgrad(l);
+    for (int l : sel) add_wgrad(l);
+    s->tasks_units = units;
+    s->tasks_counters = counters;
+    if (counters > s->max_counters || tk.size() > (size_t)2 * L) return ET_ERR_WORKSPACE;
+    if (!tk.empty())
+      CU_TRY(cudaMemcpyAsync(s->at(s->off_tasks), tk.data(), tk.size() * sizeof(tl::Task), cudaMemcpyHostToDevice, st));
+    s->tasks_key = key;
+  }
+  double flops = 0.0;
+  for (int l = d; l < L; ++l) {
+    const double gemm = 2.0 * (double)M * s->ly[l].K * s->ly[l].N;
+    if (l > d) flops += gemm;
+    if (mask[2 * l]) flops += gemm;
+  }
+
+  const et::OptParams opt = opt_params(s, lr);
+  const int snap = s->delta_is_snapshot ? 1 : 0;
+  if (s->tasks_units > 0) {
+    if (s->tasks_counters > 0)
+      CU_TRY(cudaMemsetAsync(s->at(s->off_counters), 0, sizeof(unsigned) * (size_t)s->tasks_counters, st));
+    TimedLaunch tlch(s, ET_K_LIST, st);
+    const int workers = std::min(s->tasks_units, list_max_clusters(s->sms));
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[2];
+    cfg.gridDim = dim3(2 * workers); cfg.blockDim = dim3(et::tc::THREADS); cfg.dynamicSmemBytes = tl::LSMEM_BYTES;
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;           // every CTA resident: units may wait on one another
+    attr[1].val.cooperative = 1;
+    cfg.attrs = attr; cfg.numAttrs = s->opt_list_cooperative ? 2 : 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tl::gemm_list_kernel, (const tl::Task*)s->at(s->off_tasks),
+                                             s->tasks_units, (unsigned*)s->at(s->off_counters),
+                                             (uint32_t*)s->at(s->off_status));
+    if (e != cudaSuccess) {
+      (void)cudaGetLastError();
+      if (s->list_state == 0) { s->list_state = -1; *refused = true; return ET_OK; }
+      g_last_cuda = (int)e;
+      return ET_ERR_CUDA;
+    }
+    s->list_state = 1;
+    ET_TRY(after_launch());
+    ++launches;
+  }
+
+  // ---- grouped split reduction (gradient export, Eq. 2, update) and grouped bias finishers
+  float* imp_parts = (float*)s->at(s->off_imp_parts);
+  {
+    std::vector<et::ReduceEntry> tab;
+    std::vector<int> chunk_blocks;                  // blocks of each launch of at most kGroupMax tensors
+    int blocks = 0;
+    for (int l = d; l < L; ++l) {
+      if (!mask[2 * l]) continue;
+      const LayerRT& Y = s->ly[l];
+      float* g = grads ? grads[2 * l] : nullptr;
+      const void* dl = delta ? delta[2 * l] : nullptr;
+      if (g == nullptr && dl == nullptr && !sgd) continue;       // nothing consumes the gradient
+      et::ReduceEntry e;
+      std::memset(&e, 0, sizeof(e));
+      e.partial = (const float*)s->at(Y.off_partial_list); e.grad = g; e.delta = dl;
+      e.imp_part = imp_parts + s->imp_offs[2 * l]; e.W = Y.W; e.master = Y.W32; e.m_state = Y.st1[0]; e.v_state = Y.st2[0];
+      e.count = (unsigned long long)Y.K * Y.N; e.splits = Y.split_now;
+      if (tab.size() % et::kGroupMax == 0) { chunk_blocks.push_back(0); blocks = 0; }   // a new launch starts here
+      e.block_begin = blocks;
+      blocks += Y.imp_count_w;
+      chunk_blocks.back() = blocks;
+      tab.push_back(e);
+    }
+    if (!tab.empty()) {
+      if (tab.size() != s->rtab_host.size() ||
+          std::memcmp(tab.data(), s->rtab_host.data(), tab.size() * sizeof(et::ReduceEntry)) != 0) {
+        CU_TRY(cudaMemcpyAsync(s->at(s->off_rtab), tab.data(), tab.size() * sizeof(et::ReduceEntry),
+                               cudaMemcpyHostToDevice, st));
+        s->rtab_host = tab;
+      }
+      for (size_t i0 = 0; i0 < tab.size(); i0 += et::kGroupMax) {
+        const int n = (int)std::min(tab.size() - i0, (size_t)et::kGroupMax);
+        const int nb = chunk_blocks[i0 / et::kGroupMax];
+        TimedLaunch tlch(s, ET_K_WGRAD_REDUCE, st);
+        et::wgrad_reduce_group_kernel<bf16><<<std::min(nb, s->sms * 8), et::kEltThreads, 0, st>>>(
+            (const et::ReduceEntry*)s->at(s->off_rtab) + i0, n, nb, opt, sgd ? 1 : 0, snap);
+        ET_TRY(after_launch());
+        ++launches;
+      }
+    }
+  }
+  {
+    std::vector<et::BiasEntry> tab;
+    std::vector<int> chunk_blocks;
+    int blocks = 0;
+    for (int l = d; l < L; ++l) {
+      if (!mask[2 * l + 1]) continue;
+      const LayerRT& Y = s->ly[l];
+      et::BiasEntry e;
+      std::memset(&e, 0, sizeof(e));
+      e.part = (const float*)s->at(Y.off_biaspart);
+      e.grad = grads ? grads[2 * l + 1] : nullptr; e.delta = delta ? delta[2 * l + 1] : nullptr;
+      e.imp_part = imp_parts + s->imp_offs[2 * l + 1]; e.b = Y.b; e.master = Y.b32; e.m_state = Y.st1[1]; e.v_state = Y.st2[1];
+      // row blocks the partials come in: 32-row blocks of the dgrad epilogue above, 128-row chunks for the top layer
+      e.chunks = l == L - 1 ? top_chunks : tiles_m_tok * (2 * et::tc::BM / 32);
+      e.width = Y.Nw; e.count = Y.N;
+      if (tab.size() % et::kGroupMax == 0) { chunk_blocks.push_back(0); blocks = 0; }
+      e.block_begin = blocks;
+      blocks += Y.imp_count_b;
+      chunk_blocks.back() = blocks;
+      tab.push_back(e);
+    }
+    if (!tab.empty()) {
+      if (tab.size() != s->btab_host.size() ||
+          std::memcmp(tab.data(), s->btab_host.data(), tab.size() * sizeof(et::BiasEntry)) != 0) {
+        CU_TRY(cudaMemcpyAsync(s->at(s->off_btab), tab.data(), tab.size() * sizeof(et::BiasEntry),
+                               cudaMemcpyHostToDevice, st));
+        s->btab_host = tab;
+      }
+      for (size_t i0 = 0; i0 < tab.size(); i0 += et::kGroupMax) {
+        const int n = (int)std::min(tab.size() - i0, (size_t)et::kGroupMax);
+        const int nb = chunk_blocks[i0 / et::kGroupMax];
+        TimedLaunch tlch(s, ET_K_BGRAD, st);
+        et::bias_finish_group_kernel<bf16><<<std::min(nb, s->sms * 2), dim3(et::kBiasCols, et::kBiasLanes), 0, st>>>(
+            (const et::BiasEntry*)s->at(s->off_btab) + i0, n, nb, opt, sgd ? 1 : 0, snap);
+        ET_TRY(after_launch());
+        ++launches;
+      }
+    }
+  }
+  *launches_out += launches;
+  *flops_out += flops;
+  return ET_OK;
+}
+
 template <typename T>
 et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float* const* grads,
                         const void* const* delta, float* importance_dev, uint32_t flags, float lr,
@@ -931,6 +1243,17 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
         s->map_dy_ptr = dY;
       }
     }
+    // Stacks of plain dense layers take the one-launch path: all GEMMs of the pass in one cooperative kernel,
+    // one grouped reducer, one grouped bias finisher.
+    bool done_by_list = false;
+    if constexpr (is_bf16<T>::value) {
+      if (list_eligible(s, d)) {
+        bool refused = false;
+        ET_TRY(backward_list(s, dY, mask, grads, delta, sgd, lr, d, &launches, &flops, st, &refused));
+        done_by_list = !refused;
+      }
+    }
+    if (!done_by_list) {
     const bool two = !s->timing && s->opt_two_streams && setup_two_streams(s);   // per-kernel timing wants kernels one at a time
     // Sharing the GPU with the higher-priority error-gradient chain: when few kernels are selected
     // the weight gradients are filler work and should hand their SMs back after every unit; when
@@ -1022,6 +1345,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
       CU_TRY(cudaEventRecord(s->chain_ev[L + 1], cs));
       CU_TRY(cudaStreamWaitEvent(st, s->chain_ev[L + 1], 0));
     }
+    }   // per-layer path
     if (delta != nullptr) {
       TimedLaunch tl(s, ET_K_OTHER, st);
       et::importance_finalize_kernel<<<2 * L, 128, 0, st>>>((const float*)s->at(s->off_imp_parts),
@@ -1207,6 +1531,17 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
       const TilePlan dsh = y.big_gemm ? choose_tiles((int)M, y.K, kb_n, s->sms, false, true, 0, true) : d;
       y.bn_dgrad_sh = dsh.bn; y.pair_dgrad_sh = dsh.pair;
       y.bn_wgrad = w.bn; y.pair_wgrad = w.pair; y.split = w.split;
+      // One-launch backward: units of all GEMMs share the CTAs, so a weight gradient need not fill the GPU by
+      // itself.  Splits of about 32 k-blocks for small tensors (units of a size with the error-gradient tiles),
+      // fewer for large ones: every split writes and re-reads 4 bytes per parameter (at most 24 MB per tensor).
+      y.list_ok = y.kind == ET_LAYER_DENSE && y.K % 64 == 0 && y.Nw % 64 == 0;
+      if (y.list_ok) {
+        const int kb = ceil_div(M, et::tc::BK);
+        int sp = std::max(1, std::min(8, kb / 32));
+        while (sp > 1 && (double)sp * y.K * y.N * 4.0 > 24e6) --sp;
+        while (sp > 1 && (long long)(sp - 1) * ceil_div(kb, sp) >= kb) --sp;
+        y.split_list = sp;
+      }
 #ifdef ET_DEBUG_HOOKS
       if (const char* force = getenv("ET_DEBUG_TILES")) {          // debug builds only: "<bn>,<pair>[,<split>]" for every GEMM
         int fb = 0, fp = 0, fs = 0;
@@ -1245,6 +1580,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
     max_partial = std::max(max_partial, y.vector_params() ? (size_t)y.N * sizeof(float)
                                                           : (size_t)std::max(y.split, y.split_shared) * y.K * y.N * sizeof(float));
     y.off_biaspart = take((size_t)std::max(chunks, ceil_div(M, 256) * 8 + 8) * y.Nw * sizeof(float));
+    if (y.list_ok) y.off_partial_list = take((size_t)y.split_list * y.K * y.N * sizeof(float));
     y.imp_count_w = y.vector_params() ? ceil_div(y.N, et::kBiasCols)
                                             : ceil_div((long long)y.K * y.N, et::kEltThreads * et::kVec);
     y.imp_count_b = ceil_div(y.N, et::kBiasCols);
@@ -1260,6 +1596,13 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
   s->off_loss_parts = take((size_t)ceil_div(out_count, et::kEltThreads * et::kVec) * sizeof(float));
   s->off_dy_stage = take(out_count * s->elt);
   s->off_imp_stage = take((size_t)2 * L * sizeof(float));
+  if (dtype == ET_BF16) {
+    s->off_tasks = take((size_t)2 * L * sizeof(et::tl::Task));
+    s->max_counters = L * (ceil_div(M, 2 * et::tc::BM) + 1);
+    s->off_counters = take((size_t)s->max_counters * sizeof(unsigned));
+    s->off_rtab = take((size_t)L * sizeof(et::ReduceEntry));
+    s->off_btab = take((size_t)L * sizeof(et::BiasEntry));
+  }
   s->ws_bytes = off;
   *out = s;
   return ET_OK;
@@ -1287,6 +1630,14 @@ et_status et_stack_set_option(et_stack* s, int32_t option, int32_t value) {
     case ET_OPTION_TILE_PLAN:
       if (value != ET_TILE_PLAN_AUTO && value != ET_TILE_PLAN_ALONE && value != ET_TILE_PLAN_SHARED) return ET_ERR_INVALID_ARG;
       s->opt_tile_plan = value;
+      return ET_OK;
+    case ET_OPTION_GEMM_LIST:
+      if (value != 0 && value != 1) return ET_ERR_INVALID_ARG;
+      s->opt_gemm_list = value != 0;
+      return ET_OK;
+    case ET_OPTION_LIST_COOPERATIVE:
+      if (value != 0 && value != 1) return ET_ERR_INVALID_ARG;
+      s->opt_list_cooperative = value != 0;
       return ET_OK;
     default:
       return ET_ERR_INVALID_ARG;
@@ -1320,6 +1671,7 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
         ET_TRY(make_tmaps(&y.map_W, y.W, y.N, y.K));
         ET_TRY(make_map(&y.map_Wd, y.W, y.N, y.K, y.pair_dgrad ? y.bn_dgrad / 2 : y.bn_dgrad));
         ET_TRY(make_map(&y.map_Wd_sh, y.W, y.N, y.K, y.pair_dgrad_sh ? y.bn_dgrad_sh / 2 : y.bn_dgrad_sh));
+        if (y.list_ok) ET_TRY(make_map(&y.map_Wd_list, y.W, y.N, y.K, et::tl::LBNH));
       }
       if (l < s->L - 1) {
         ET_TRY(make_tmaps(&y.map_aout, s->at(y.off_a_out), y.Nw, s->M));
@@ -1336,6 +1688,10 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   CU_TRY(cudaMemcpyAsync(s->at(s->off_imp_offs), s->imp_offs.data(), sizeof(int) * 2 * s->L, cudaMemcpyHostToDevice, st));
   CU_TRY(cudaMemcpyAsync(s->at(s->off_imp_counts), s->imp_counts.data(), sizeof(int) * 2 * s->L, cudaMemcpyHostToDevice, st));
   CU_TRY(cudaStreamSynchronize(st));     // the host vectors may be freed / changed afterwards
+  ++s->bind_serial;                      // device tables of the one-launch backward are rebuilt on next use
+  s->tasks_key.clear();
+  s->rtab_host.clear();
+  s->btab_host.clear();
   s->bound = true;
   s->forwarded = false;
   s->map_dy_ptr = nullptr;
@@ -1358,6 +1714,7 @@ et_status et_stack_bind_master(et_stack* s, float* const* W32, float* const* b32
     s->ly[l].W32 = W32 ? W32[l] : nullptr;
     s->ly[l].b32 = b32 ? b32[l] : nullptr;
   }
+  ++s->bind_serial;                      // task lists hold these pointers
   return ET_OK;
 }
 
@@ -1550,6 +1907,7 @@ et_status et_stack_set_optimizer(et_stack* s, const et_optimizer_config* cfg, fl
   s->opt_cfg = c;
   s->opt_step = 1;
   s->opt_wd_now = c.weight_decay;
+  ++s->bind_serial;                      // task lists hold the state pointers
   return ET_OK;
 }
 

@@ -195,6 +195,11 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
                ::"l"(map), "r"(src), "r"(c0), "r"(c1)
                : "memory");
 }
+// The TMA unit reads a descriptor from memory the first time an instruction names it (about a
+// microsecond); asking for it at kernel entry hides that behind the barrier and TMEM set-up.
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void tma_store_wait_read() {
@@ -363,6 +368,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
+  if (warp == 0 && lane == 0) { prefetch_tmap(&map_a); prefetch_tmap(&map_b); }
+  if constexpr (SLOTS > 0) {
+    if (warp >= 2 + 4 * EPI_GROUPS && lane == 0) {
+#pragma unroll
+      for (int s = 0; s < SLOTS; ++s) {
+        if (epi_in.has_in[s]) prefetch_tmap(&emaps.in[s]);
+        if (epi_in.has_out[s]) prefetch_tmap(&emaps.out[s]);
+      }
+    }
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(acc_full_bar(s), 1); mbar_init(acc_empty_bar(s), PAIR ? 16 : 8); }

@@ -63,14 +63,36 @@ __device__ __forceinline__ void opt_update_seg(float (&w)[8], const float (&g)[8
 //   master != nullptr: the weight lives in fp32 there (W is its rounded copy): the update and
 //                  the snapshot difference use it, and a snapshot `delta` is fp32 as well
 template <typename T>
-__global__ void __launch_bounds__(kEltThreads)
-wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_t count,
-                    float* grad /* may alias partial: each thread reads its elements before writing them */, const T* __restrict__ delta, float* __restrict__ imp_part,
-                    T* __restrict__ W, OptParams opt, int do_sgd, int delta_is_snapshot, float* __restrict__ master,
-                    float* __restrict__ m_state, float* __restrict__ v_state) {
-  const size_t i0 = ((size_t)blockIdx.x * kEltThreads + threadIdx.x) * kVec;
+__device__ __forceinline__ float wgrad_reduce_elems(size_t i0, const float* partial, int splits, size_t split_stride,
+                                                    size_t count, float* grad, const T* __restrict__ delta,
+                                                    T* __restrict__ W, const OptParams& opt, int do_sgd,
+                                                    int delta_is_snapshot, float* __restrict__ master,
+                                                    float* __restrict__ m_state, float* __restrict__ v_state);
+template <typename T>
+__device__ __forceinline__ void wgrad_reduce_block(int block, const float* partial, int splits, size_t split_stride,
+                                                   size_t count, float* grad, const T* __restrict__ delta,
+                                                   float* __restrict__ imp_part, T* __restrict__ W, const OptParams& opt,
+                                                   int do_sgd, int delta_is_snapshot, float* __restrict__ master,
+                                                   float* __restrict__ m_state, float* __restrict__ v_state) {
+  const size_t i0 = ((size_t)block * kEltThreads + threadIdx.x) * kVec;
   float dot = 0.0f;
-  if (i0 < count) {
+  if (i0 < count)
+    dot = wgrad_reduce_elems<T>(i0, partial, splits, split_stride, count, grad, delta, W, opt, do_sgd, delta_is_snapshot,
+                                master, m_state, v_state);
+  if (delta != nullptr) {
+    dot = block_sum(dot);
+    if (threadIdx.x == 0) imp_part[block] = dot;
+  }
+}
+// The work on kVec consecutive elements starting at i0 < count; returns their share of sum(g * dw).
+template <typename T>
+__device__ __forceinline__ float wgrad_reduce_elems(size_t i0, const float* partial, int splits, size_t split_stride,
+                                                    size_t count, float* grad, const T* __restrict__ delta,
+                                                    T* __restrict__ W, const OptParams& opt, int do_sgd,
+                                                    int delta_is_snapshot, float* __restrict__ master,
+                                                    float* __restrict__ m_state, float* __restrict__ v_state) {
+  float dot = 0.0f;
+  {
     const int n = (int)min((size_t)kVec, count - i0);
     float g[kVec], t[kVec], w[kVec];
     load_seg<kVec>(partial + i0, n, g);
@@ -102,9 +124,55 @@ wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_
       store_seg<kVec>(W + i0, n, w);
     }
   }
-  if (delta != nullptr) {
-    dot = block_sum(dot);
-    if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
+  return dot;
+}
+template <typename T>
+__global__ void __launch_bounds__(kEltThreads)
+wgrad_reduce_kernel(const float* partial, int splits, size_t split_stride, size_t count,
+                    float* grad /* may alias partial: each thread reads its elements before writing them */, const T* __restrict__ delta, float* __restrict__ imp_part,
+                    T* __restrict__ W, OptParams opt, int do_sgd, int delta_is_snapshot, float* __restrict__ master,
+                    float* __restrict__ m_state, float* __restrict__ v_state) {
+  wgrad_reduce_block<T>((int)blockIdx.x, partial, splits, split_stride, count, grad, delta, imp_part, W, opt, do_sgd,
+                        delta_is_snapshot, master, m_state, v_state);
+}
+
+// One launch for every selected kernel tensor of a step: a table in device memory names each tensor's
+// partial sums, outputs and first block; a block finds its tensor by binary search and does exactly what
+// a wgrad_reduce_kernel block of that tensor does (same elements, same order: results are identical).
+struct ReduceEntry {
+  const float* partial;
+  float* grad;
+  const void* delta;
+  float* imp_part;
+  void* W;
+  float* master;
+  float* m_state;
+  float* v_state;
+  unsigned long long count;
+  int splits;
+  int block_begin;         // first block of this tensor in the grouped grid
+};
+// The grid is a few blocks per SM; each walks the concatenated block range with the table held in shared
+// memory, so that finding a block's tensor costs no chain of global loads.
+constexpr int kGroupMax = 128;                          // table entries per launch
+template <typename T>
+__global__ void __launch_bounds__(kEltThreads)
+wgrad_reduce_group_kernel(const ReduceEntry* __restrict__ tab, int n, int total_blocks, OptParams opt, int do_sgd,
+                          int delta_is_snapshot) {
+  __shared__ ReduceEntry sh[kGroupMax];
+  for (int i = threadIdx.x; i < n * (int)(sizeof(ReduceEntry) / 8); i += blockDim.x)
+    reinterpret_cast<unsigned long long*>(sh)[i] = reinterpret_cast<const unsigned long long*>(tab)[i];
+  __syncthreads();
+  for (int vb = blockIdx.x; vb < total_blocks; vb += gridDim.x) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {                                 // last entry with block_begin <= vb
+      const int mid = (lo + hi + 1) >> 1;
+      if (sh[mid].block_begin <= vb) lo = mid; else hi = mid - 1;
+    }
+    const ReduceEntry& e = sh[lo];
+    wgrad_reduce_block<T>(vb - e.block_begin, e.partial, e.splits, (size_t)e.count, (size_t)e.count, e.grad,
+                          (const T*)e.delta, e.imp_part, (T*)e.W, opt, do_sgd, delta_is_snapshot, e.master, e.m_state,
+                          e.v_state);
   }
 }
 
@@ -162,17 +230,27 @@ colsum_partial_kernel(const T* __restrict__ dZ, int M, int width, float* __restr
 constexpr int kBiasCols = 32;
 constexpr int kBiasLanes = 32;
 template <typename T>
-__global__ void __launch_bounds__(kBiasCols * kBiasLanes)
-bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
-                   float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
-                   T* __restrict__ b, OptParams opt, int do_sgd, int delta_is_snapshot, float* __restrict__ master,
-                   float* __restrict__ m_state, float* __restrict__ v_state) {
+__device__ __forceinline__ void bias_finish_block(int block, const float* __restrict__ part, int chunks, int width,
+                                                  int count, float* __restrict__ grad, const T* __restrict__ delta,
+                                                  float* __restrict__ imp_part, T* __restrict__ b, const OptParams& opt,
+                                                  int do_sgd, int delta_is_snapshot, float* __restrict__ master,
+                                                  float* __restrict__ m_state, float* __restrict__ v_state) {
   __shared__ float sm[kBiasLanes][kBiasCols + 1];
-  const int j = blockIdx.x * kBiasCols + threadIdx.x;
+  const int j = block * kBiasCols + threadIdx.x;
   float g = 0.0f;
   if (j < count) {
     const int col = j % width;
-    for (int c = threadIdx.y; c < chunks; c += kBiasLanes) g += part[(size_t)c * width + col];
+    // four independent chains of loads: the kernel is latency-bound
+    float g1 = 0.0f, g2 = 0.0f, g3 = 0.0f;
+    int c = threadIdx.y;
+    for (; c + 3 * kBiasLanes < chunks; c += 4 * kBiasLanes) {
+      g += part[(size_t)c * width + col];
+      g1 += part[(size_t)(c + kBiasLanes) * width + col];
+      g2 += part[(size_t)(c + 2 * kBiasLanes) * width + col];
+      g3 += part[(size_t)(c + 3 * kBiasLanes) * width + col];
+    }
+    for (; c < chunks; c += kBiasLanes) g += part[(size_t)c * width + col];
+    g = (g + g1) + (g2 + g3);
   }
   sm[threadIdx.y][threadIdx.x] = g;
   __syncthreads();
@@ -205,8 +283,53 @@ bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int co
     }
     if (delta != nullptr) {                           // one warp: fixed shuffle tree
       dot = warp_sum(dot);
-      if (threadIdx.x == 0) imp_part[blockIdx.x] = dot;
+      if (threadIdx.x == 0) imp_part[block] = dot;
     }
+  }
+}
+template <typename T>
+__global__ void __launch_bounds__(kBiasCols * kBiasLanes)
+bias_finish_kernel(const float* __restrict__ part, int chunks, int width, int count,
+                   float* __restrict__ grad, const T* __restrict__ delta, float* __restrict__ imp_part,
+                   T* __restrict__ b, OptParams opt, int do_sgd, int delta_is_snapshot, float* __restrict__ master,
+                   float* __restrict__ m_state, float* __restrict__ v_state) {
+  bias_finish_block<T>((int)blockIdx.x, part, chunks, width, count, grad, delta, imp_part, b, opt, do_sgd,
+                       delta_is_snapshot, master, m_state, v_state);
+}
+// One launch for every selected bias of a step: a table in device memory names each bias's partial sums,
+// outputs and first block; a block finds its entry by binary search and does exactly what a
+// bias_finish_kernel block of that bias does.
+struct BiasEntry {
+  const float* part;
+  float* grad;
+  const void* delta;
+  float* imp_part;
+  void* b;
+  float* master;
+  float* m_state;
+  float* v_state;
+  int chunks, width, count;
+  int block_begin;
+};
+template <typename T>
+__global__ void __launch_bounds__(kBiasCols * kBiasLanes)
+bias_finish_group_kernel(const BiasEntry* __restrict__ tab, int n, int total_blocks, OptParams opt, int do_sgd,
+                         int delta_is_snapshot) {
+  __shared__ BiasEntry sh[kGroupMax];
+  const int tid = threadIdx.y * blockDim.x + threadIdx.x;
+  for (int i = tid; i < n * (int)(sizeof(BiasEntry) / 8); i += blockDim.x * blockDim.y)
+    reinterpret_cast<unsigned long long*>(sh)[i] = reinterpret_cast<const unsigned long long*>(tab)[i];
+  __syncthreads();
+  for (int vb = blockIdx.x; vb < total_blocks; vb += gridDim.x) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (sh[mid].block_begin <= vb) lo = mid; else hi = mid - 1;
+    }
+    const BiasEntry& e = sh[lo];
+    bias_finish_block<T>(vb - e.block_begin, e.part, e.chunks, e.width, e.count, e.grad, (const T*)e.delta,
+                         e.imp_part, (T*)e.b, opt, do_sgd, delta_is_snapshot, e.master, e.m_state, e.v_state);
+    __syncthreads();                                  // the block's shared partials are reused by the next one
   }
 }
 

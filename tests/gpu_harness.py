@@ -24,11 +24,15 @@ def to_np(t: torch.Tensor) -> np.ndarray:
 class GpuRun:
     """Holds device tensors of a workload bound to an et stack."""
 
-    def __init__(self, w: wl.Workload):
+    def __init__(self, w: wl.Workload, gemm_list=None):
+        """gemm_list: None = the library's default; False = one launch per GEMM (the two-stream path) even where
+        the one-launch backward would apply; True = say so explicitly."""
         self.w = w
         et.et_debug_guard_regions(True)          # every test stack carries guard words round its workspace regions
         self.stack = et.et_stack_create(w.layers, w.M, w.dtype)
         et.et_debug_guard_regions(False)
+        if gemm_list is not None:
+            et.et_stack_set_option(self.stack, et.ET_OPTION_GEMM_LIST, 1 if gemm_list else 0)
         self.W = [to_dev(a, w.dtype) for a in w.W]
         self.b = [to_dev(a, w.dtype) for a in w.b]
         nbytes = et.et_stack_workspace_bytes(self.stack)
@@ -114,13 +118,13 @@ class StepChecker:
     master=True attaches fp32 master copies of bf16 parameters (the update is applied to them and the
     bf16 tensors are rewritten as their roundings)."""
 
-    def __init__(self, w: wl.Workload, tol: float, master: bool = False):
+    def __init__(self, w: wl.Workload, tol: float, master: bool = False, gemm_list=None):
         self.w, self.tol, self.master = w, tol, master
         self.saved = orc.forward(w.layers, w.W, w.b, w.x)
         self.loss, self.dY = orc.mse_loss_grad(self.saved.a[-1], w.target)
         self.params_o = orc.tensors_of(w.W, w.b)
         self._grads = {}
-        run = self.run = GpuRun(w)
+        run = self.run = GpuRun(w, gemm_list=gemm_list)
         self.before = [p.clone() for p in run.params()]
         self.m32 = None
         if master:
@@ -240,12 +244,12 @@ class StepChecker:
 
 
 def check_step(w: wl.Workload, mask, tol: float, delta_seed: int = 77, w_tol: float = 1e-3, stats=None,
-               aligned_delta: bool = False, derived_w_tol: bool = False):
+               aligned_delta: bool = False, derived_w_tol: bool = False, gemm_list=None):
     """Full parity check of one training step: forward, loss, elastic backward with fused
     importance and SGD.  Returns the report.  With aligned_delta the importance is checked
     by its plain relative error.  Updated weights must be within w_tol (1e-3) of the oracle's;
     with derived_w_tol the bound also admits what the arithmetic cannot avoid when weights or
     gradients are large: the bf16 store's half ulp (2^-9 |w|) and lr * tol * ||g||_inf from the
     gradient's own tolerance."""
-    return StepChecker(w, tol).check(mask, delta_seed=delta_seed, w_tol=w_tol, stats=stats,
-                                     aligned_delta=aligned_delta, derived_w_tol=derived_w_tol)
+    return StepChecker(w, tol, gemm_list=gemm_list).check(mask, delta_seed=delta_seed, w_tol=w_tol, stats=stats,
+                                                          aligned_delta=aligned_delta, derived_w_tol=derived_w_tol)

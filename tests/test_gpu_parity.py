@@ -131,13 +131,35 @@ def test_bf16_small_vit_block_ragged_rows():
     h.check_step(w, w.mask, TOL_BF16)
 
 
+@pytest.mark.parametrize("gemm_list", [True, False])
 @pytest.mark.parametrize("seed", [0, 1, 2, 3])
-def test_bf16_random_masks_small_vit(seed):
+def test_bf16_random_masks_small_vit(seed, gemm_list):
+    """Both launch schemes of the backward pass: every GEMM of the call in one cooperative launch
+    (gemm_list) and one launch per GEMM on two streams."""
     h = _h()
     w = wl.vit_b(seed=20 + seed, p_select=0.3, n_blocks=3, tokens=[197, 520, 1000, 333][seed], d=256, ffn=768)
     if not w.mask.any():
         w.mask[-2:] = 1
-    h.check_step(w, w.mask, TOL_BF16)
+    rep = h.check_step(w, w.mask, TOL_BF16, gemm_list=gemm_list)
+    n_gemms = int(rep.dgrad.sum() + rep.wgrad.sum())
+    if gemm_list:
+        assert rep.launches <= 6                     # loss-side kernels, one GEMM launch, two grouped finishers
+    else:
+        assert rep.launches >= n_gemms
+
+
+def test_bf16_one_launch_backward_all_masks_of_a_block():
+    """Every selection of the eight tensors of one transformer block (256 masks) through the one-launch
+    backward: the task list, its dependency counters and the fused weight-gradient epilogues are rebuilt
+    for each mask on the same stack."""
+    h = _h()
+    w = wl.vit_b(seed=41, p_select=0.5, n_blocks=1, tokens=600, d=256, ffn=512)
+    c = h.StepChecker(w, TOL_BF16, gemm_list=True)
+    for bits in range(1, 256, 7):
+        mask = np.array([(bits >> i) & 1 for i in range(8)], dtype=np.uint8)
+        c.check(mask)
+    c.check(np.ones(8, dtype=np.uint8), aligned_delta=True)
+    c.check(np.ones(8, dtype=np.uint8), snapshot=True)
 
 
 def test_bf16_ragged_widths_and_bias_only_selection():
@@ -207,6 +229,10 @@ def test_bf16_vit_b_full_size_config(vit_b_checker):
     stats = {}
     c.check(c.w.mask, stats=stats)
     c.check(c.w.mask, stats=stats, aligned_delta=True)
+    # the same step launched GEMM by GEMM on two streams (the path stacks with other layer kinds take)
+    et.et_stack_set_option(c.run.stack, et.ET_OPTION_GEMM_LIST, 0)
+    c.check(c.w.mask, stats=stats)
+    et.et_stack_set_option(c.run.stack, et.ET_OPTION_GEMM_LIST, 1)
     print("vit_b parity diagnostics", stats)
 
 
