@@ -122,7 +122,7 @@ typedef struct {
                              at most 2048), act = ET_ACT_NONE, fold = 1, residual_src = -1 */
   float eps;              /* ET_LAYER_NORM: added to the variance, > 0 or 0 */
   int32_t heads;          /* ET_LAYER_ATTENTION: in_features = 3 * out_features, out_features = 64 * heads;   */
-  int32_t seq_len;        /*   rows form sequences of seq_len (<= 208) consecutive rows, M a multiple of it;  */
+  int32_t seq_len;        /*   rows form sequences of seq_len (<= 256) consecutive rows, M a multiple of it;  */
                           /*   ET_BF16 only; not the first or last layer; the layer below has no activation;   */
                           /*   act = ET_ACT_NONE, fold = 1, residual_src = -1.  Both fields 0 for other kinds. */
   int32_t height;         /* ET_LAYER_IM2COL: rows are images of height x width pixels, NHWC (M a multiple of  */

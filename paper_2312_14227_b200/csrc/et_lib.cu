@@ -726,27 +726,18 @@ et_status run_bn_backward(et_stack* s, int l, const void* dY, bool want_dx, bool
 
 // ---- attention core --------------------------------------------------------------------------
 // Dynamic shared memory above 48 KB has to be allowed per kernel and device.
-et_status attn_allow_forward(size_t bytes) {
-  static size_t allowed[64] = {};
+et_status attn_allow_smem() {
+  static bool done[64] = {};
   int dev = 0;
   CU_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
   std::lock_guard<std::mutex> cache_lock(g_cache_mutex);
-  if (bytes > allowed[dev]) {
-    CU_TRY(cudaFuncSetAttribute(et::attn::attn_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-    allowed[dev] = bytes;
-  }
-  return ET_OK;
-}
-et_status attn_allow_backward(size_t bytes) {
-  static size_t allowed[64] = {};
-  int dev = 0;
-  CU_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return ET_ERR_UNSUPPORTED;
-  std::lock_guard<std::mutex> cache_lock(g_cache_mutex);
-  if (bytes > allowed[dev]) {
-    CU_TRY(cudaFuncSetAttribute(et::attn::attn_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-    allowed[dev] = bytes;
+  if (!done[dev]) {
+    CU_TRY(cudaFuncSetAttribute(et::attn::attn_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)et::attn::FWD_SMEM));
+    CU_TRY(cudaFuncSetAttribute(et::attn::attn_backward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)et::attn::BWD_SMEM));
+    done[dev] = true;
   }
   return ET_OK;
 }
@@ -754,23 +745,23 @@ et_status attn_allow_backward(size_t bytes) {
 et_status run_attn_forward(et_stack* s, int l, cudaStream_t st) {
   TimedLaunch tl(s, ET_K_ATTENTION, st);
   const LayerRT& L = s->ly[l];
-  const size_t smem = et::attn::forward_smem_bytes(L.seq);
-  ET_TRY(attn_allow_forward(smem));
+  ET_TRY(attn_allow_smem());
   const int grid = (int)(s->M / L.seq) * L.heads;
-  et::attn::attn_forward_kernel<<<grid, et::attn::THREADS, smem, st>>>(
-      act_in<bf16>(s, l), (bf16*)s->at(L.off_a_out), (float*)s->at(L.off_lse), L.seq, L.heads, L.N);
+  et::attn::attn_forward_kernel<<<grid, et::attn::THREADS, et::attn::FWD_SMEM, st>>>(
+      a_map(s, l).b128, (bf16*)s->at(L.off_a_out), (float*)s->at(L.off_lse), L.seq, L.heads, L.N,
+      (uint32_t*)s->at(s->off_status));
   return after_launch();
 }
 // G_l (gradient of [q | k | v]) from G_{l+1}; l >= 1 and the layer below has no activation, so G_l is its dZ.
 et_status run_attn_backward(et_stack* s, int l, const void* dY, cudaStream_t st) {
   TimedLaunch tl(s, ET_K_ATTENTION, st);
   const LayerRT& L = s->ly[l];
-  const size_t smem = et::attn::backward_smem_bytes(L.seq);
-  ET_TRY(attn_allow_backward(smem));
+  ET_TRY(attn_allow_smem());
   const int grid = (int)(s->M / L.seq) * L.heads;
-  et::attn::attn_backward_kernel<<<grid, et::attn::THREADS_BWD, smem, st>>>(
-      act_in<bf16>(s, l), (const bf16*)s->at(L.off_a_out), grad_act<bf16>(s, l + 1, dY), (const float*)s->at(L.off_lse),
-      (bf16*)s->at(s->ly[l - 1].off_G_out), L.seq, L.heads, L.N);
+  et::attn::attn_backward_kernel<<<grid, et::attn::THREADS, et::attn::BWD_SMEM, st>>>(
+      a_map(s, l).b128, g_map(s, l + 1).b128, (const bf16*)s->at(L.off_a_out), grad_act<bf16>(s, l + 1, dY),
+      (const float*)s->at(L.off_lse), (bf16*)s->at(s->ly[l - 1].off_G_out), L.seq, L.heads, L.N,
+      (uint32_t*)s->at(s->off_status));
   return after_launch();
 }
 
@@ -1157,7 +1148,7 @@ et_status backward_list(et_stack* s, const void* dY, const uint8_t* mask, float*
         const int n = (int)std::min(tab.size() - i0, (size_t)et::kGroupMax);
         const int nb = chunk_blocks[i0 / et::kGroupMax];
         TimedLaunch tlch(s, ET_K_WGRAD_REDUCE, st);
-        et::wgrad_reduce_group_kernel<bf16><<<std::min(nb, s->sms * 8), et::kEltThreads, 0, st>>>(
+        et::wgrad_reduce_group_kernel<bf16><<<std::min(nb, s->sms * et::kGroupBlocksPerSm), et::kEltThreads, 0, st>>>(
             (const et::ReduceEntry*)s->at(s->off_rtab) + i0, n, nb, opt, sgd ? 1 : 0, snap);
         ET_TRY(after_launch());
         ++launches;

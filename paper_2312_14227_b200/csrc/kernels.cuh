@@ -155,8 +155,9 @@ struct ReduceEntry {
 // The grid is a few blocks per SM; each walks the concatenated block range with the table held in shared
 // memory, so that finding a block's tensor costs no chain of global loads.
 constexpr int kGroupMax = 128;                          // table entries per launch
+constexpr int kGroupBlocksPerSm = 4;                    // resident blocks the grouped reducer is compiled for
 template <typename T>
-__global__ void __launch_bounds__(kEltThreads)
+__global__ void __launch_bounds__(kEltThreads, kGroupBlocksPerSm)
 wgrad_reduce_group_kernel(const ReduceEntry* __restrict__ tab, int n, int total_blocks, OptParams opt, int do_sgd,
                           int delta_is_snapshot) {
   __shared__ ReduceEntry sh[kGroupMax];

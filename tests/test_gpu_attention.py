@@ -29,9 +29,9 @@ def _mask_all(layers):
     return m
 
 
-@pytest.mark.parametrize("heads,seq,batch", [(4, 50, 3), (2, 197, 2), (1, 208, 1), (2, 16, 5), (3, 1, 40), (2, 65, 3)])
+@pytest.mark.parametrize("heads,seq,batch", [(4, 50, 3), (2, 197, 2), (1, 208, 1), (2, 16, 5), (3, 1, 40), (2, 65, 3), (1, 256, 2), (2, 129, 2), (1, 128, 3)])
 def test_all_trainable_tensors_selected(heads, seq, batch):
-    # sequence lengths below, at and across the 64-row query blocks and the 16-column tiles
+    # sequence lengths below, at and across the 128-row halves of a tile and the 16-column steps
     h = _h()
     layers = _stack(64 * heads, heads, seq)
     w = wl.small_stack(layers, batch * seq, wl.DT_BF16, 81, mask=_mask_all(layers), w_std=0.1, bias_std=0.05)
@@ -68,7 +68,7 @@ def test_unsupported_shapes_and_selections_are_refused():
     with pytest.raises(et.EtError):                                   # rows are not whole sequences
         et.et_stack_create(ok, 90, wl.DT_BF16)
     with pytest.raises(et.EtError):                                   # sequence too long
-        et.et_stack_create(_stack(128, 2, 224), 448, wl.DT_BF16)
+        et.et_stack_create(_stack(128, 2, 272), 544, wl.DT_BF16)
     with pytest.raises(et.EtError):                                   # head width is not 64
         et.et_stack_create([wl.Layer(64, 96), wl.Layer(96, 3 * 96), wl.attention_layer(96, 2, 8), wl.Layer(96, 8)], 16, wl.DT_BF16)
     with pytest.raises(et.EtError):                                   # last layer
