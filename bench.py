@@ -586,8 +586,9 @@ def run_side(args):
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
-    w = {"resnet": wl.resnet_1x1, "prenorm": wl.vit_b_prenorm, "full": wl.vit_b_full, "bottleneck": wl.resnet_bottleneck,
-         "bottleneck_bn": lambda: wl.resnet_bottleneck(bn=True),
+    nb = {} if args.blocks == 12 else {"n_blocks": args.blocks}     # --blocks: a reduced stack of the same shapes (profiling)
+    w = {"resnet": wl.resnet_1x1, "prenorm": lambda: wl.vit_b_prenorm(**nb), "full": lambda: wl.vit_b_full(**nb),
+         "bottleneck": wl.resnet_bottleneck, "bottleneck_bn": lambda: wl.resnet_bottleneck(bn=True),
          "schedule": wl.vit_l, "schedule_full": wl.vit_l_full}[args.workload]()
     tdt = torch.bfloat16
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(tdt).to(dev).contiguous()

@@ -35,6 +35,13 @@ using namespace et::tc;
 constexpr int DH = 64;           // head width
 constexpr int S_MAX = 256;       // longest sequence
 constexpr float SCALE = 0.125f;  // 1 / sqrt(DH)
+constexpr float SCALE_LOG2E = 0.125f * 1.4426950408889634f;   // exp(x / 8) = 2^(x * SCALE_LOG2E)
+constexpr float LOG2E = 1.4426950408889634f;
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 constexpr uint32_t TILE_BYTES = 128 * DH * 2;          // one 128-row x 64-column bf16 tile: 16 KB
 constexpr int THREADS = 320;     // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2-9: row threads
 constexpr uint32_t FWD_SMEM = 6 * TILE_BYTES + 8 * TILE_BYTES + 1024 + 256;   // q, k, v (2 tiles each), P (2 x 4 tiles)
@@ -157,25 +164,36 @@ attn_forward_kernel(const __grid_constant__ CUtensorMap map_qkv, bf16* __restric
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(hh * 256);
         const int nchunk = (SP + 31) / 32;
+        // chunks of 32 keys; only the last one can reach past the sequence and needs the per-key test
+        const int nfull = S / 32;
         float m = -INFINITY;
         for (int c = 0; c < nchunk; ++c) {
           float v[32];
           tmem_ld32(taddr + c * 32, v);
+          if (c < nfull) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) m = fmaxf(m, (c * 32 + i < S) ? v[i] : -INFINITY);
+            for (int i = 0; i < 32; ++i) m = fmaxf(m, v[i]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) m = fmaxf(m, (c * 32 + i < S) ? v[i] : -INFINITY);
+          }
         }
         float sum = 0.0f;
         uint8_t* Pt = gen + 6 * TILE_BYTES + hh * 4 * TILE_BYTES;
         const bool valid = row < S;
+        const float mk = valid ? m * SCALE_LOG2E : INFINITY;     // rows past the sequence: 2^(-inf) = 0 everywhere
         for (int c = 0; c < nchunk; ++c) {
           float v[32];
           tmem_ld32(taddr + c * 32, v);
+          if (c < nfull) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            // rounded to bf16 here so that the row sum matches what the product below actually uses
-            const float e = (valid && c * 32 + i < S) ? __expf((v[i] - m) * SCALE) : 0.0f;
-            v[i] = __bfloat162float(__float2bfloat16_rn(e));
-            sum += v[i];
+            for (int i = 0; i < 32; ++i) { v[i] = ex2(fmaf(v[i], SCALE_LOG2E, -mk)); sum += v[i]; }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              v[i] = (c * 32 + i < S) ? ex2(fmaf(v[i], SCALE_LOG2E, -mk)) : 0.0f;
+              sum += v[i];
+            }
           }
           sts_row32(Pt + (c >> 1) * TILE_BYTES, trow, c & 1, v);
         }
@@ -340,7 +358,9 @@ attn_backward_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_c
       const int kh = i / halves, rh = i - kh * halves;
       const int row = rh * 128 + trow;
       const bool rvalid = row < S;
-      const float D = rh == 0 ? Dr[0] : Dr[1], l = rh == 0 ? lr[0] : lr[1];
+      // P = 2^(s log2e / 8 - lse log2e), all zero in rows past the sequence; dS = P (dP - D) / 8
+      const float DS = (rh == 0 ? Dr[0] : Dr[1]) * SCALE;
+      const float l2 = rvalid ? (rh == 0 ? lr[0] : lr[1]) * LOG2E : INFINITY;
       ok = mbar_wait(bar_sdp, (uint32_t)i & 1u, abort_flag, status, kTimeoutAttn);
       if (!ok) break;
       if (i > 0) {                                                // the previous block's P / dS have been consumed
@@ -361,11 +381,20 @@ attn_backward_kernel(const __grid_constant__ CUtensorMap map_qkv, const __grid_c
           mbar_arrive(bar_sfree);
         }
         const int key0 = kh * 128 + cg * 64 + c * 32;
+        if (key0 + 32 <= S) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float p = (rvalid && key0 + j < S) ? __expf(sv[j] * SCALE - l) : 0.0f;
-          sv[j] = p;
-          pv[j] = p * (pv[j] - D) * SCALE;
+          for (int j = 0; j < 32; ++j) {
+            const float p = ex2(fmaf(sv[j], SCALE_LOG2E, -l2));
+            sv[j] = p;
+            pv[j] = p * fmaf(pv[j], SCALE, -DS);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float p = key0 + j < S ? ex2(fmaf(sv[j], SCALE_LOG2E, -l2)) : 0.0f;
+            sv[j] = p;
+            pv[j] = p * fmaf(pv[j], SCALE, -DS);
+          }
         }
         sts_row32(Pt, trow, c, sv);
         sts_row32(Dt, trow, c, pv);
