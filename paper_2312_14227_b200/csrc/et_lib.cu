@@ -110,6 +110,41 @@ et_status make_map3(CUtensorMap* m, const void* ptr, int inner, long long outer,
   }
   return ET_OK;
 }
+// NHWC bf16 tensor [images x height x width x channels] for TMA's im2col mode: a load fetches `pixels`
+// consecutive base pixels (w fastest, then h, then image) x 64 channels, each pixel read at a tap offset in
+// [0, ksize) from its base; base pixels range over [-pad, extent - pad) (stride 1, zero padding ksize / 2), and
+// whatever falls outside the image reads as zero.
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeIm2colFn lookup_im2col_fn() {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &q) == cudaSuccess &&
+      q == cudaDriverEntryPointSuccess)
+    return (EncodeIm2colFn)p;
+  (void)cudaGetLastError();
+  return nullptr;
+}
+et_status make_im2col_map(CUtensorMap* m, const void* ptr, int channels, int width, int height, long long images, int ksize,
+                          int pixels) {
+  static const EncodeIm2colFn fn = lookup_im2col_fn();
+  if (fn == nullptr) return ET_ERR_CUDA;
+  const int pad = ksize / 2;
+  cuuint64_t dims[4] = {(cuuint64_t)channels, (cuuint64_t)width, (cuuint64_t)height, (cuuint64_t)images};
+  cuuint64_t strides[3] = {(cuuint64_t)channels * 2, (cuuint64_t)channels * 2 * width, (cuuint64_t)channels * 2 * width * height};
+  int lower[2] = {-pad, -pad};
+  int upper[2] = {pad - (ksize - 1), pad - (ksize - 1)};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, lower, upper, 64,
+                  (cuuint32_t)pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_last_cuda = (int)cudaErrorInvalidValue;
+    return ET_ERR_CUDA;
+  }
+  return ET_OK;
+}
 // All the views of one bf16 activation / gradient / weight matrix that the GEMMs use.
 struct TMaps {
   CUtensorMap b64;     // 64 x 64 boxes: MN-major operand fetched chunk by chunk
@@ -176,6 +211,13 @@ struct LayerRT {
   int split_list = 1;       // wgrad contraction splits in the one-launch backward
   size_t off_partial_list = 0;   // this layer's own split partials there (kept until the grouped reducer runs)
   bool list_ok = false;     // shapes the one-launch backward takes (bf16 dense layer, widths multiples of 64)
+  // Patch gather whose gathered matrix is never formed: the three GEMMs of the dense layer above fetch the
+  // patches themselves (TMA im2col mode).  Set on the gather layer.
+  bool implicit = false;
+  CUtensorMap im_fwd, im_wg, im_dg;          // im2col views: input (128 / 64 pixels per load), dZ of the layer above
+  const void* im_in_ptr = nullptr;           // what im_fwd / im_wg were made for
+  const void* im_dg_ptr = nullptr;           // what im_dg was made for
+  CUtensorMap map_Wd_conv;                   // on the dense layer above: W as K-major B in 128-row boxes
   int split_now = 1;        // per task list: splits of this layer's weight-gradient task
 };
 
@@ -422,26 +464,54 @@ et::tc::Params tc_params(const et_stack* s, int rows, int cols, int contraction,
   p.kb_per_split = ceil_div(p.kb_total, split);
   p.b_k_seg_stride = 0; p.b_mn_seg_stride = 0; p.b_mn_wrap = 0;
   p.a_3d = 0; p.b_3d = 0;
+  p.a_im2col = 0; p.img_w = 0; p.img_h = 0; p.ksize = 0; p.chan = 0; p.a_tap_flip = 0;
   p.status = (uint32_t*)s->at(s->off_status);
   return p;
 }
 
 // Z_l = a_l W_l + b_l, activation, fold, residual -> a_{l+1}
+// The im2col views of gather layer g's input (made again when the input pointer has changed: layer 0 reads
+// the caller's x).
+et_status conv_input_maps(et_stack* s, int g) {
+  LayerRT& G = s->ly[g];
+  const void* in = g == 0 ? s->x : (const void*)s->at(s->ly[g - 1].off_a_out);
+  if (G.im_in_ptr == in) return ET_OK;
+  const long long images = s->M / ((long long)G.img_h * G.img_w);
+  ET_TRY(make_im2col_map(&G.im_fwd, in, G.K, G.img_w, G.img_h, images, G.ksize, 128));
+  ET_TRY(make_im2col_map(&G.im_wg, in, G.K, G.img_w, G.img_h, images, G.ksize, 64));
+  G.im_in_ptr = in;
+  return ET_OK;
+}
+void conv_params(et::tc::Params* p, const LayerRT& G, int mode) {
+  p->a_im2col = mode; p->img_w = G.img_w; p->img_h = G.img_h; p->ksize = G.ksize; p->chan = G.K;
+}
+
 template <typename T>
 et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
   TimedLaunch tl(s, ET_K_FORWARD, st);
   const LayerRT& L = s->ly[l];
   if constexpr (is_bf16<T>::value) {
-    et::tc::Params p = tc_params(s, (int)s->M, L.Nw, L.K, L.fold, 1);
+    const bool conv = l >= 1 && s->ly[l - 1].implicit;      // A = patches of the gather layer's input, one tap per segment
+    et::tc::Params p = conv ? tc_params(s, (int)s->M, L.Nw, s->ly[l - 1].K, s->ly[l - 1].ksize * s->ly[l - 1].ksize, 1)
+                            : tc_params(s, (int)s->M, L.Nw, L.K, L.fold, 1);
     p.b_mn_seg_stride = L.Nw;
+    if (conv) {
+      ET_TRY(conv_input_maps(s, l - 1));
+      conv_params(&p, s->ly[l - 1], 1);
+      p.b_mn_seg_stride = 0;
+      p.b_k_seg_stride = s->ly[l - 1].K;                   // W's rows are (tap, channel)
+    }
     et::tc::EpiMaps em;
     const CUtensorMap& out = (l == s->L - 1 ? s->map_y : L.map_aout).b128;
     em.in[0] = L.residual_src >= 0 ? a_map(s, L.residual_src).b128 : out;
     em.out[0] = out;
     em.in[1] = out;
     em.out[1] = L.act != ET_ACT_NONE ? L.map_Z.b128 : out;
-    const int bnh = L.pair_fwd ? L.bn_fwd / 2 : L.bn_fwd;
+    const int bn_f = conv ? 128 : L.bn_fwd;
+    const bool pair_f = conv ? false : L.pair_fwd;
+    const int bnh = pair_f ? bn_f / 2 : bn_f;
     const CUtensorMap& wmap = mn_map(L.map_W, bnh / 64, &p.b_3d);
+    const CUtensorMap& amap = conv ? s->ly[l - 1].im_fwd : a_map(s, l).b128;
     auto fill = [&](auto& epi) {
       epi.has_in[0] = L.residual_src >= 0; epi.has_in[1] = false;
       epi.has_out[0] = true; epi.has_out[1] = L.act != ET_ACT_NONE;
@@ -449,10 +519,10 @@ et_status run_forward_layer(et_stack* s, int l, void* y, cudaStream_t st) {
     };
     if (L.act != ET_ACT_NONE) {
       et::FwdEpiS<2> epi; fill(epi);
-      return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch);
+      return launch_tc<false, true>(bn_f, pair_f, amap, wmap, em, p, epi, s->sms, st, false, s->overlap_launch);
     }
     et::FwdEpiS<1> epi; fill(epi);
-    return launch_tc<false, true>(L.bn_fwd, L.pair_fwd, a_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch);
+    return launch_tc<false, true>(bn_f, pair_f, amap, wmap, em, p, epi, s->sms, st, false, s->overlap_launch);
   } else {
     et::FwdEpi<T> epi;
     epi.bias = (const T*)L.b;
@@ -484,13 +554,32 @@ template <typename T>
 et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, bool want_colsum = false) {
   TimedLaunch tl(s, ET_K_DGRAD, st);
   const LayerRT& L = s->ly[l];
-  const LayerRT& P = s->ly[l - 1];
-  const bool need_skip = L.consumer >= 0;
+  // Above a patch gather that is never materialised this GEMM is the convolution's error gradient: it goes
+  // straight to the gather's input (layer l - 1's), reading dZ_l's patches with the kernel turned by 180 degrees.
+  const bool conv = is_bf16<T>::value && s->ly[l - 1].implicit;
+  const int lo = conv ? l - 1 : l;                          // G_lo is what this GEMM produces
+  const LayerRT& Lc = s->ly[lo];
+  const LayerRT& P = s->ly[lo - 1];
+  const bool need_skip = Lc.consumer >= 0;
   const bool need_act = P.act != ET_ACT_NONE;
-  const bool need_G = !need_act || P.residual_src >= 0;     // G_l itself is read later
+  const bool need_G = !need_act || P.residual_src >= 0;     // G_lo itself is read later
   if constexpr (is_bf16<T>::value) {
-    et::tc::Params p = tc_params(s, (int)s->M, L.K, L.Nw, L.fold, 1);
+    et::tc::Params p = conv ? tc_params(s, (int)s->M, Lc.K, L.Nw, Lc.ksize * Lc.ksize, 1)
+                            : tc_params(s, (int)s->M, L.K, L.Nw, L.fold, 1);
     p.b_k_seg_stride = L.Nw;
+    if (conv) {
+      LayerRT& G = s->ly[lo];
+      const void* dz = dz_src<T>(s, l, dY);
+      if (G.im_dg_ptr != dz) {
+        ET_TRY(make_im2col_map(&G.im_dg, dz, L.Nw, G.img_w, G.img_h, s->M / ((long long)G.img_h * G.img_w), G.ksize, 128));
+        G.im_dg_ptr = dz;
+      }
+      conv_params(&p, G, 1);
+      p.a_tap_flip = 1;
+      p.b_k_seg_stride = 0;
+      p.b_mn_seg_stride = G.K;                              // W's rows are (tap, channel): one tap per segment
+      want_colsum = false;                                  // the bias below a gather takes the column-sum kernel
+    }
     et::tc::EpiMaps em;
     const CUtensorMap& gout = P.map_Gout.b128;                // G_l lives in layer l-1's buffer
     // Two tile plans: alone on the GPU whole waves count (768-wide outputs on 12608 rows: 192-wide pair
@@ -498,34 +587,36 @@ et_status run_dgrad_layer(et_stack* s, int l, const void* dY, cudaStream_t st, b
     // not lost, and the wider tile with less operand traffic per flop wins (256-wide: 150 units; measured on
     // the ViT-B step 2.45 -> 2.33 ms).
     const bool sh = s->shared_plan;
-    const int bn_d = sh ? L.bn_dgrad_sh : L.bn_dgrad;
-    const bool pair_d = sh ? L.pair_dgrad_sh : L.pair_dgrad;
-    const CUtensorMap& wmap = sh ? L.map_Wd_sh : L.map_Wd;
-    const CUtensorMap& skip = need_skip ? g_map(s, L.consumer + 1).b128 : gout;
+    const int bn_d = conv ? 128 : sh ? L.bn_dgrad_sh : L.bn_dgrad;
+    const bool pair_d = conv ? false : sh ? L.pair_dgrad_sh : L.pair_dgrad;
+    const CUtensorMap& wmap = conv ? L.map_Wd_conv : sh ? L.map_Wd_sh : L.map_Wd;
+    const CUtensorMap& amap = conv ? s->ly[lo].im_dg : dz_map(s, l).b128;
+    const int ld_out = Lc.K;
+    const CUtensorMap& skip = need_skip ? g_map(s, Lc.consumer + 1).b128 : gout;
     const CUtensorMap& zmap = P.map_Z.b128;
     const CUtensorMap& dzout = P.map_dZ.b128;
     if (!need_act) {                                          // G_l = acc (+ skip)
       et::DgradEpiS<1> epi;
       epi.has_in[0] = need_skip; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = false; epi.act_prev = P.act;
-      epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
+      epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = ld_out;
       em.in[0] = skip; em.out[0] = gout; em.in[1] = gout; em.out[1] = gout;
-      return launch_tc<false, false>(bn_d, pair_d, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
+      return launch_tc<false, false>(bn_d, pair_d, amap, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
     }
     if (!need_skip && !need_G) {                              // dZ_{l-1} = acc * act'(Z_{l-1})
       et::DgradEpiS<1> epi;
       epi.has_in[0] = true; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
       epi.mul_act = true; epi.act_prev = P.act;
-      epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
+      epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = ld_out;
       em.in[0] = zmap; em.out[0] = dzout; em.in[1] = zmap; em.out[1] = dzout;
-      return launch_tc<false, false>(bn_d, pair_d, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
+      return launch_tc<false, false>(bn_d, pair_d, amap, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
     }
     et::DgradEpiS<2> epi;                                     // both G_l and dZ_{l-1}
     epi.has_in[0] = need_skip; epi.has_in[1] = true; epi.has_out[0] = need_G; epi.has_out[1] = true;
     epi.mul_act = false; epi.act_prev = P.act;
-    epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = L.K;
+    epi.colsum = want_colsum ? (float*)s->at(P.off_biaspart) : nullptr; epi.ld = ld_out;
     em.in[0] = skip; em.out[0] = gout; em.in[1] = zmap; em.out[1] = dzout;
-    return launch_tc<false, false>(bn_d, pair_d, dz_map(s, l).b128, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
+    return launch_tc<false, false>(bn_d, pair_d, amap, wmap, em, p, epi, s->sms, st, false, s->overlap_launch && !s->chain_shares_gpu);
   } else {
     et::DgradEpi<T> epi;
     epi.skip = need_skip ? grad_act<T>(s, L.consumer + 1, dY) : nullptr;
@@ -810,10 +901,18 @@ et_status run_wgrad_layer(et_stack* s, int l, const void* dY, float* grad, const
       p.b_mn_wrap = L.fold > 1 ? L.Nw : 0;
       et::tc::EpiMaps em;
       em.in[0] = em.in[1] = em.out[0] = em.out[1] = L.map_W.b64;      // unused by the direct epilogue
+      if (l >= 1 && s->ly[l - 1].implicit) {
+        // kernel gradient of a convolution: the rows of A^T are (tap, channel), gathered 64 pixels at a time
+        ET_TRY(conv_input_maps(s, l - 1));
+        conv_params(&p, s->ly[l - 1], 2);
+        const CUtensorMap& bmap = mn_map(dz_map(s, l), 2, &p.b_3d);
+        ET_TRY((launch_tc<true, true>(128, false, s->ly[l - 1].im_wg, bmap, em, p, epi, s->sms, st, s->wgrad_one_unit)));
+      } else {
       const int bnh = L.pair_wgrad ? L.bn_wgrad / 2 : L.bn_wgrad;
       const CUtensorMap& amap = mn_map(a_map(s, l), 2, &p.a_3d);
       const CUtensorMap& bmap = mn_map(dz_map(s, l), bnh / 64, &p.b_3d);
       ET_TRY((launch_tc<true, true>(L.bn_wgrad, L.pair_wgrad, amap, bmap, em, p, epi, s->sms, st, s->wgrad_one_unit)));
+      }
     } else {
       et::simt::Params p;
       p.rows = L.K; p.cols = L.N; p.kc = (int)s->M; p.segs = 1;
@@ -1294,6 +1393,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
       }
       if (!Y.trainable()) {
         // a non-trainable layer: only passes the error gradient on, above the deepest selected layer
+        if (Y.implicit) continue;                            // done by the error-gradient GEMM of the layer above
         if (l > d) {
           if (Y.kind == ET_LAYER_ATTENTION) ET_TRY(run_attn_backward(s, l, dY, cs));
           else ET_TRY(run_im2col_backward<T>(s, l, dY, cs));
@@ -1320,6 +1420,7 @@ et_status backward_impl(et_stack* s, const void* dY, const uint8_t* mask, float*
       if (l > d) {
         ET_TRY(run_dgrad_layer<T>(s, l, dY, cs, mask[2 * (l - 1) + 1] != 0));
         if (two) CU_TRY(cudaEventRecord(s->chain_ev[l], cs));   // dZ_{l-1} ready, W_l no longer needed
+        if (two && s->ly[l - 1].implicit) CU_TRY(cudaEventRecord(s->chain_ev[l - 1], cs));   // and the gather's backward with it
         ++launches;
         flops += gemm;
       }
@@ -1381,7 +1482,7 @@ et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
     if (s->ly[l].kind == ET_LAYER_NORM) ET_TRY(run_norm_forward<T>(s, l, y, st));
     else if (s->ly[l].kind == ET_LAYER_BATCHNORM) ET_TRY(run_bn_forward<T>(s, l, y, st));
     else if (s->ly[l].kind == ET_LAYER_ATTENTION) ET_TRY(run_attn_forward(s, l, st));
-    else if (s->ly[l].kind == ET_LAYER_IM2COL) ET_TRY(run_im2col_forward<T>(s, l, st));
+    else if (s->ly[l].kind == ET_LAYER_IM2COL) { if (!s->ly[l].implicit) ET_TRY(run_im2col_forward<T>(s, l, st)); }
     else ET_TRY(run_forward_layer<T>(s, l, y, st));
   }
   s->forwarded = true;
@@ -1476,6 +1577,15 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
   }
   for (int l = 0; l < L && err == ET_OK; ++l)
     if (s->ly[l].kind == ET_LAYER_ATTENTION && s->ly[l].consumer >= 0) err = ET_ERR_UNSUPPORTED;   // [q|k|v] feeds nothing else
+  // A patch gather followed directly by a dense layer is folded into that layer's GEMMs (the gathered matrix is
+  // never formed) when the shapes allow TMA's im2col loads: bf16, channels a multiple of 128 (a 128-row tile of
+  // the kernel gradient then lies within one tap), not the first layer (its input would need no gradient).
+  for (int l = 1; l + 1 < L && err == ET_OK; ++l) {
+    LayerRT& y = s->ly[l];
+    const LayerRT& up = s->ly[l + 1];
+    y.implicit = dtype == ET_BF16 && y.kind == ET_LAYER_IM2COL && y.K % 128 == 0 && up.kind == ET_LAYER_DENSE &&
+                 up.fold == 1 && up.N % 64 == 0;
+  }
   if (err != ET_OK) { delete s; return err; }
 
   // ---- workspace layout
@@ -1495,7 +1605,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
   for (int l = 0; l < L; ++l) {
     LayerRT& y = s->ly[l];
     const size_t act_bytes = (size_t)M * y.Nw * s->elt;
-    if (l < L - 1) { y.off_a_out = take(act_bytes); y.off_G_out = take(act_bytes); }
+    if (l < L - 1 && !y.implicit) { y.off_a_out = take(act_bytes); y.off_G_out = take(act_bytes); }
     if (y.act != ET_ACT_NONE) { y.off_Z = take(act_bytes); y.off_dZ = take(act_bytes); }
     if (y.kind == ET_LAYER_ATTENTION) {
       y.off_lse = take((size_t)M * y.heads * sizeof(float));
@@ -1664,10 +1774,12 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
         ET_TRY(make_map(&y.map_Wd_sh, y.W, y.N, y.K, y.pair_dgrad_sh ? y.bn_dgrad_sh / 2 : y.bn_dgrad_sh));
         if (y.list_ok) ET_TRY(make_map(&y.map_Wd_list, y.W, y.N, y.K, et::tl::LBNH));
       }
-      if (l < s->L - 1) {
+      if (l < s->L - 1 && !y.implicit) {
         ET_TRY(make_tmaps(&y.map_aout, s->at(y.off_a_out), y.Nw, s->M));
         ET_TRY(make_tmaps(&y.map_Gout, s->at(y.off_G_out), y.Nw, s->M));
       }
+      y.im_in_ptr = nullptr; y.im_dg_ptr = nullptr;
+      if (y.kind == ET_LAYER_DENSE && l >= 1 && s->ly[l - 1].implicit) ET_TRY(make_map(&y.map_Wd_conv, y.W, y.N, y.K, 128));
       if (y.act != ET_ACT_NONE) {
         ET_TRY(make_tmaps(&y.map_Z, s->at(y.off_Z), y.Nw, s->M));
         ET_TRY(make_tmaps(&y.map_dZ, s->at(y.off_dZ), y.Nw, s->M));
@@ -1959,6 +2071,7 @@ et_status et_profile_costs(et_stack* s, const void* x, void* y, const void* dY, 
         double t_attn = 0.0;
         if (l >= 1) {
           if (s->ly[l].kind == ET_LAYER_ATTENTION) ET_TRY(timed([&]() { return run_attn_backward(s, l, dY, st); }, &t_attn));
+          else if (s->ly[l].implicit) t_attn = 0.0;       // part of the error-gradient GEMM of the layer above
           else if (s->dtype == ET_BF16) ET_TRY(timed([&]() { return run_im2col_backward<bf16>(s, l, dY, st); }, &t_attn));
           else ET_TRY(timed([&]() { return run_im2col_backward<float>(s, l, dY, st); }, &t_attn));
         }

@@ -88,6 +88,14 @@ struct Params {
   int b_mn_wrap;             // B's mn coordinate taken modulo this, 0 = off (wgrad through a fold)
   int a_3d, b_3d;            // MN-major operand fetched by one 3-D copy (all 64-wide chunks at once)
                              // instead of one 2-D copy per chunk; needs its width to be a multiple of 64
+  // Convolution without a gathered matrix (single-CTA tiles only): A's tiles are fetched by TMA in im2col
+  // mode from the NHWC tensor.  1: rows of A are pixels (forward, dgrad: K-major, one tap per fold segment,
+  // map with 128 pixels per column); 2: the contraction runs over pixels (wgrad: MN-major, rows of A are
+  // (tap, channel), map with 64 pixels per column).
+  int a_im2col;
+  int img_w, img_h, ksize;   // image extent in pixels, taps per side (zero padding ksize / 2, stride 1)
+  int chan;                  // wgrad: channels per tap (a multiple of 128)
+  int a_tap_flip;            // dgrad: segment s reads tap ksize^2 - 1 - s (the kernel turned by 180 degrees)
   uint32_t* status;          // device word, 0 = ok; first failure wins
 };
 
@@ -158,6 +166,16 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar & kPeerBitMask), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// im2col mode: `pixels per column` consecutive base pixels of the tensor map's bounding box, walked w first,
+// then h, then image, starting at base pixel (w, h, n); each read at offset (ow, oh) from its base pixel,
+// channels [c, c + 64); zeros outside the image.
+__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w, int h, int n,
+                                                int ow, int oh) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"((uint16_t)ow), "h"((uint16_t)oh)
       : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -446,7 +464,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           // Few, large copies: issuing a TMA copy costs the producer thread far more than
           // the copy's size does.  K-major operands come as one box of 64 k x (tile rows);
           // MN-major operands as one 3-D box (64 mn, 64 k, chunks) when their width allows.
-          if constexpr (!A_MN) {
+          if (!PAIR && p.a_im2col != 0) {
+            const int pad = p.ksize >> 1, hw = p.img_h * p.img_w;
+            if constexpr (!A_MN) {
+              // 128 pixels from m0 on; this segment's tap
+              const int tap = p.a_tap_flip ? p.ksize * p.ksize - 1 - seg : seg;
+              const int n_img = m0 / hw, r = m0 - n_img * hw, ph = r / p.img_w, pw = r - ph * p.img_w;
+              tma_load_im2col(sa, &map_a, bar, kk, pw - pad, ph - pad, n_img, tap % p.ksize, tap / p.ksize);
+            } else {
+              // rows m0.. of A are (tap, channel); this k-block is 64 pixels from pixel kk on
+              const int tap = m0 / p.chan, c0 = m0 - tap * p.chan;
+              const int n_img = kk / hw, r = kk - n_img * hw, ph = r / p.img_w, pw = r - ph * p.img_w;
+#pragma unroll
+              for (int c = 0; c < BM / 64; ++c)
+                tma_load_im2col(sa + c * CHUNK_BYTES, &map_a, bar, c0 + c * 64, pw - pad, ph - pad, n_img, tap % p.ksize,
+                                tap / p.ksize);
+            }
+          } else if constexpr (!A_MN) {
             load(sa, &map_a, bar, kk, m0);
           } else if (p.a_3d) {
             load3(sa, &map_a, bar, 0, kk, m0 >> 6);
