@@ -664,9 +664,10 @@ def run_side(args):
             g = [ly for ly in w.layers if ly.kind == wl.KIND_IM2COL]
             nbytes = sum(2.0 * (w.M * ly.in_features + w.M * ly.out_features) * 2 for ly in g)   # fwd + bwd, bf16
             gather_ms = t["attention"][0] / 5
+            # no gather kernel runs where the GEMMs fetch the patches themselves (bf16, channels a multiple of 128)
             extra = {"gather_ms_per_forward_plus_backward": gather_ms, "gather_launches": t["attention"][1] / 5,
-                     "gather_gbs": nbytes / gather_ms / 1e6,
-                     "gather_frac_of_hbm_peak": nbytes / gather_ms / 1e6 / _peaks()["hbm_gbs"],
+                     "gather_gbs": nbytes / gather_ms / 1e6 if gather_ms > 0 else None,
+                     "gather_frac_of_hbm_peak": nbytes / gather_ms / 1e6 / _peaks()["hbm_gbs"] if gather_ms > 0 else None,
                      "dgrad_ms": t["dgrad"][0] / 5, "wgrad_ms": t["wgrad"][0] / 5, "forward_gemm_ms": t["forward"][0] / 5,
                      "norm_ms_per_forward_plus_backward": t["norm"][0] / 5, "norm_timed_regions": t["norm"][1] / 5}
         if args.workload == "full":
