@@ -40,7 +40,10 @@
  *   padding k / 2) from NHWC rows:  a_{l+1}[(n,h,w), (kh*k + kw)*C + c] = a_l[(n, h+kh-k/2, w+kw-k/2), c].
  *   Followed by a dense layer with in_features = k*k*C it is the convolutional layer of Section 5.1
  *   (that layer's kernel is the convolution kernel in (kh, kw, c_in) x c_out layout).  Like the
- *   attention core it has no tensors: NULL pointers, mask bits 0.
+ *   attention core it has no tensors: NULL pointers, mask bits 0.  On ET_BF16 stacks, when C is a
+ *   multiple of 128, the layer is not the first one and the dense layer follows it directly (fold = 1,
+ *   out_features a multiple of 64), the gathered matrix a_{l+1} is never formed: the dense layer's three
+ *   GEMMs fetch the patches themselves, and the gather's forward and backward launch nothing.
  *
  *   A layer of kind ET_LAYER_NORM is a layer normalisation over the features of each row
  *   (Section 5.2 treats normalisation layers as two trainable tensors, Gamma and Beta;
@@ -258,10 +261,12 @@ et_status et_loss_mse_grad(et_stack* s, const void* y, const void* target, void*
  * Nothing is launched for layers below the deepest selected one; with an empty mask
  * nothing is launched at all except zeroing importance_dev.  Needs a preceding
  * et_forward_stack on the same stack.
- * The error-gradient chain runs on an internal high-priority stream that forks from and joins
- * back into `stream` inside the call (weight gradients fill the SMs the chain leaves idle); to
- * the caller everything is ordered on `stream`.  ET_SINGLE_STREAM=1 in the environment keeps
- * all kernels on `stream`. */
+ * How it is launched (see et_stack_set_option): stacks whose layers from the deepest selected one upwards
+ * are all dense (bf16, widths multiples of 64) run every GEMM of the call as one cooperative launch,
+ * followed by one grouped reducer and one grouped bias finisher, all on `stream`.  Other stacks launch
+ * layer by layer: the error-gradient chain on an internal high-priority stream that forks from and joins
+ * back into `stream` inside the call (weight gradients fill the SMs the chain leaves idle).  Either way,
+ * to the caller everything is ordered on `stream`. */
 et_status et_backward_elastic(et_stack* s, const void* dY, const uint8_t* mask, int32_t n_tensors,
                               float* const* grads, const void* const* delta,
                               float* importance_dev, uint32_t flags, float lr,
