@@ -164,7 +164,10 @@ et_status et_stack_destroy(et_stack* s);
  *                            streams when they run, for a GPU to itself otherwise; ET_TILE_PLAN_ALONE /
  *                            ET_TILE_PLAN_SHARED force one (per-kernel timing keeps kernels on one stream and
  *                            can still time the shapes the two-stream step launches).
- *   ET_OPTION_GEMM_LIST      1 (default): where every layer from the deepest selected one upwards is a dense layer
+ *   ET_OPTION_GEMM_LIST      1 (default): where every layer is a dense layer with widths that are multiples of 64 (bf16
+ *                            stacks; no layer with both an activation and a residual), et_forward_stack runs all layers
+ *                            as ONE cooperative launch whose work units wait on one another row tile by row tile; and
+ *                            where every layer from the deepest selected one upwards is a dense layer
  *                            with widths that are multiples of 64 (bf16 stacks), et_backward_elastic runs all
  *                            error-gradient and weight-gradient GEMMs of the call as ONE cooperative launch whose
  *                            work units wait on one another row tile by row tile, followed by one grouped launch

@@ -261,6 +261,10 @@ struct et_stack {
   std::vector<et::tl::Task> tasks_host;
   std::vector<uint8_t> tasks_key;      // mask and pointers the device task list was built for
   int tasks_units = 0, tasks_counters = 0;
+  size_t off_ftasks = 0;               // the forward pass's task list
+  std::vector<et::tl::Task> ftasks_host;
+  std::vector<uint8_t> ftasks_key;
+  int ftasks_units = 0, ftasks_counters = 0;
   std::vector<et::ReduceEntry> rtab_host;
   std::vector<et::BiasEntry> btab_host;
   int list_state = 0;                  // 0 = untried, 1 = works, -1 = the cooperative launch was refused: per-layer path
@@ -1053,6 +1057,8 @@ bool list_eligible(const et_stack* s, int d) {
   return list_max_clusters(s->sms) > 0;
 }
 
+et_status launch_list(et_stack* s, const et::tl::Task* tasks_dev, int units, int counters, cudaStream_t st, bool* refused);
+
 // Every GEMM of the pass as one task list and one cooperative launch of gemm_list_kernel, then one grouped
 // launch each for the split reductions and the bias finishers.  *refused: the device would not take the
 // cooperative launch; nothing of the pass has been changed, the caller runs the per-layer path instead.
@@ -1186,30 +1192,8 @@ et_status backward_list(et_stack* s, const void* dY, const uint8_t* mask, float*
   const et::OptParams opt = opt_params(s, lr);
   const int snap = s->delta_is_snapshot ? 1 : 0;
   if (s->tasks_units > 0) {
-    if (s->tasks_counters > 0)
-      CU_TRY(cudaMemsetAsync(s->at(s->off_counters), 0, sizeof(unsigned) * (size_t)s->tasks_counters, st));
-    TimedLaunch tlch(s, ET_K_LIST, st);
-    const int workers = std::min(s->tasks_units, list_max_clusters(s->sms));
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[2];
-    cfg.gridDim = dim3(2 * workers); cfg.blockDim = dim3(et::tc::THREADS); cfg.dynamicSmemBytes = tl::LSMEM_BYTES;
-    cfg.stream = st;
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeCooperative;           // every CTA resident: units may wait on one another
-    attr[1].val.cooperative = 1;
-    cfg.attrs = attr; cfg.numAttrs = s->opt_list_cooperative ? 2 : 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, tl::gemm_list_kernel, (const tl::Task*)s->at(s->off_tasks),
-                                             s->tasks_units, (unsigned*)s->at(s->off_counters),
-                                             (uint32_t*)s->at(s->off_status));
-    if (e != cudaSuccess) {
-      (void)cudaGetLastError();
-      if (s->list_state == 0) { s->list_state = -1; *refused = true; return ET_OK; }
-      g_last_cuda = (int)e;
-      return ET_ERR_CUDA;
-    }
-    s->list_state = 1;
-    ET_TRY(after_launch());
+    ET_TRY(launch_list(s, (const tl::Task*)s->at(s->off_tasks), s->tasks_units, s->tasks_counters, st, refused));
+    if (*refused) return ET_OK;
     ++launches;
   }
 
@@ -1468,6 +1452,100 @@ et_status validate_backward_args(const et_stack* s, const void* dY, const uint8_
   return ET_OK;
 }
 
+// The forward pass of a stack of plain dense layers as one task list (the same kernel as the one-launch
+// backward): layer l + 1's row tile r waits for layer l's row tile r.  *refused as in backward_list.
+et_status launch_list(et_stack* s, const et::tl::Task* tasks_dev, int units, int counters, cudaStream_t st, bool* refused) {
+  namespace tl = et::tl;
+  *refused = false;
+  if (counters > 0) CU_TRY(cudaMemsetAsync(s->at(s->off_counters), 0, sizeof(unsigned) * (size_t)counters, st));
+  TimedLaunch tlch(s, ET_K_LIST, st);
+  const int workers = std::min(units, list_max_clusters(s->sms));
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[2];
+  cfg.gridDim = dim3(2 * workers); cfg.blockDim = dim3(et::tc::THREADS); cfg.dynamicSmemBytes = tl::LSMEM_BYTES;
+  cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeCooperative;           // every CTA resident: units may wait on one another
+  attr[1].val.cooperative = 1;
+  cfg.attrs = attr; cfg.numAttrs = s->opt_list_cooperative ? 2 : 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, tl::gemm_list_kernel, tasks_dev, units, (unsigned*)s->at(s->off_counters),
+                                           (uint32_t*)s->at(s->off_status));
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    if (s->list_state == 0) { s->list_state = -1; *refused = true; return ET_OK; }
+    g_last_cuda = (int)e;
+    return ET_ERR_CUDA;
+  }
+  s->list_state = 1;
+  return after_launch();
+}
+
+bool forward_list_eligible(const et_stack* s) {
+  if (s->dtype != ET_BF16 || !s->opt_gemm_list || s->list_state < 0) return false;
+  for (int l = 0; l < s->L; ++l) {
+    const LayerRT& y = s->ly[l];
+    if (!y.list_ok) return false;
+    if (y.act != ET_ACT_NONE && y.residual_src >= 0) return false;   // Z, the output and a residual: three chunks
+  }
+  return list_max_clusters(s->sms) > 0;
+}
+
+et_status forward_list(et_stack* s, const void* x, void* y, cudaStream_t st, bool* refused) {
+  namespace tl = et::tl;
+  const int L = s->L;
+  const long long M = s->M;
+  const int tiles_m = ceil_div(M, 2 * et::tc::BM);
+  std::vector<uint8_t> key;
+  {
+    const void* q[2] = {x, y};
+    const unsigned serial = s->bind_serial;
+    key.insert(key.end(), (const uint8_t*)q, (const uint8_t*)q + sizeof(q));
+    key.insert(key.end(), (const uint8_t*)&serial, (const uint8_t*)&serial + sizeof(serial));
+  }
+  if (key != s->ftasks_key) {
+    std::vector<tl::Task>& tk = s->ftasks_host;
+    tk.clear();
+    std::vector<int> sig_base(L, -1), tiles_n_of(L, 0);
+    int counters = 0, units = 0;
+    for (int l = 0; l < L; ++l) {
+      const LayerRT& Y = s->ly[l];
+      tl::Task t;
+      std::memset(&t, 0, sizeof(t));
+      t.kind = tl::kFwd;
+      t.rows = (int)M; t.cols = Y.Nw;
+      t.tiles_m = tiles_m; t.tiles_n = ceil_div(Y.Nw, tl::LBN); t.split = 1;
+      t.kb_per_seg = ceil_div(Y.K, et::tc::BK); t.kb_total = t.kb_per_seg * Y.fold; t.kb_per_split = t.kb_total;
+      t.b_k_seg_stride = 0; t.b_mn_wrap = 0; t.b_mn_seg_stride = Y.Nw;
+      t.map_a = a_map(s, l).b128;
+      t.map_b = Y.map_W.c3[0];
+      const CUtensorMap& out = (l == L - 1 ? s->map_y : Y.map_aout).b128;
+      t.map_in = Y.residual_src >= 0 ? a_map(s, Y.residual_src).b128 : out;
+      t.map_out = out;
+      t.map_out2 = Y.act != ET_ACT_NONE ? Y.map_Z.b128 : out;
+      t.has_in = Y.residual_src >= 0 ? 1 : 0;
+      t.entries = Y.act != ET_ACT_NONE ? 2 : 1;
+      t.act = Y.act; t.fold = Y.fold; t.ld = Y.Nw; t.bias = (const bf16*)Y.b;
+      t.unit_begin = units; t.units = t.tiles_m * t.tiles_n; units += t.units;
+      t.wait_base = l >= 1 ? sig_base[l - 1] : -1; t.wait_per_row = 1;
+      t.wait_target = l >= 1 ? 4u * (unsigned)tiles_n_of[l - 1] : 0u;
+      t.wait2_base = -1; t.wait2_target = 0;
+      if (Y.residual_src >= 1) {                              // a_j is the output of layer j - 1
+        t.wait2_base = sig_base[Y.residual_src - 1];
+        t.wait2_target = 4u * (unsigned)tiles_n_of[Y.residual_src - 1];
+      }
+      t.signal_base = counters; sig_base[l] = counters; tiles_n_of[l] = t.tiles_n;
+      counters += t.tiles_m + 1;
+      tk.push_back(t);
+    }
+    if (counters > s->max_counters) return ET_ERR_WORKSPACE;
+    s->ftasks_units = units; s->ftasks_counters = counters;
+    CU_TRY(cudaMemcpyAsync(s->at(s->off_ftasks), tk.data(), tk.size() * sizeof(tl::Task), cudaMemcpyHostToDevice, st));
+    s->ftasks_key = key;
+  }
+  return launch_list(s, (const tl::Task*)s->at(s->off_ftasks), s->ftasks_units, s->ftasks_counters, st, refused);
+}
+
 template <typename T>
 et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
   if constexpr (is_bf16<T>::value) {
@@ -1478,6 +1556,13 @@ et_status forward_impl(et_stack* s, const void* x, void* y, cudaStream_t st) {
     }
   }
   s->x = x;
+  if constexpr (is_bf16<T>::value) {
+    if (forward_list_eligible(s)) {
+      bool refused = false;
+      ET_TRY(forward_list(s, x, y, st, &refused));
+      if (!refused) { s->forwarded = true; return ET_OK; }
+    }
+  }
   for (int l = 0; l < s->L; ++l) {
     if (s->ly[l].kind == ET_LAYER_NORM) ET_TRY(run_norm_forward<T>(s, l, y, st));
     else if (s->ly[l].kind == ET_LAYER_BATCHNORM) ET_TRY(run_bn_forward<T>(s, l, y, st));
@@ -1699,6 +1784,7 @@ et_status et_stack_create(const et_layer_desc* layers, int32_t L, int64_t M, et_
   s->off_imp_stage = take((size_t)2 * L * sizeof(float));
   if (dtype == ET_BF16) {
     s->off_tasks = take((size_t)2 * L * sizeof(et::tl::Task));
+    s->off_ftasks = take((size_t)L * sizeof(et::tl::Task));
     s->max_counters = L * (ceil_div(M, 2 * et::tc::BM) + 1);
     s->off_counters = take((size_t)s->max_counters * sizeof(unsigned));
     s->off_rtab = take((size_t)L * sizeof(et::ReduceEntry));
@@ -1793,6 +1879,7 @@ et_status et_stack_bind(et_stack* s, void* const* W, void* const* b, void* works
   CU_TRY(cudaStreamSynchronize(st));     // the host vectors may be freed / changed afterwards
   ++s->bind_serial;                      // device tables of the one-launch backward are rebuilt on next use
   s->tasks_key.clear();
+  s->ftasks_key.clear();
   s->rtab_host.clear();
   s->btab_host.clear();
   s->bound = true;

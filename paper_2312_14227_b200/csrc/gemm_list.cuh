@@ -17,6 +17,9 @@
 //   kDgrad  A = dZ_l K-major, B = W_l K-major, staged epilogue DgradEpiS<1> (skip gradient or
 //           act'(Z) of the layer below, optional fused bias column sums)
 //   kWgrad  A = a_l MN-major, B = dZ_l MN-major, fp32 partial sums of one contraction split
+//   kFwd    the forward pass as the same kind of list (rows [r, r + 256) of a_{l+1} need rows [r, r + 256) of
+//           a_l): A = a_l K-major, B = W_l MN-major, staged epilogue FwdEpiS (bias, activation, residual);
+//           a layer with an activation stores two chunks per 64 columns, Z_l and a_{l+1}
 #pragma once
 
 #include "gemm_tc.cuh"
@@ -37,17 +40,18 @@ static_assert(LSMEM_BYTES <= SMEM_LIMIT, "shared memory");
 constexpr int LNCHUNK = LBN / 64;
 constexpr uint32_t DEP_POLL_LIMIT = 1u << 24;           // polls of a dependency counter before giving up
 
-enum TaskKind : int { kDgrad = 0, kWgrad = 1 };
+enum TaskKind : int { kDgrad = 0, kWgrad = 1, kFwd = 2 };
 enum ListStatus : uint32_t { kTimeoutDependency = 6 };
 
 struct alignas(128) Task {
   CUtensorMap map_a, map_b;      // operands
-  CUtensorMap map_in, map_out;   // staged epilogue: input chunk (skip gradient or Z), output chunk
+  CUtensorMap map_in, map_out;   // staged epilogue: input chunk (skip gradient, Z, or residual), output chunk
+  CUtensorMap map_out2;          // kFwd with an activation: Z_l (stored before a_{l+1})
   int kind;
   int rows, cols;                // extent of the output
   int tiles_m, tiles_n, split;
   int kb_total, kb_per_seg, kb_per_split;
-  int b_k_seg_stride, b_mn_wrap;
+  int b_k_seg_stride, b_mn_wrap, b_mn_seg_stride;
   int unit_begin, units;         // this task's slice of the list
   // dependency: counters[wait_base + (wait_per_row ? row tile : 0)] >= wait_target before the A operand
   // (and the epilogue input) of a unit may be fetched; wait2_* likewise for the epilogue input alone
@@ -61,6 +65,10 @@ struct alignas(128) Task {
   // kDgrad epilogue
   int has_in, mul_act, act_prev, ld;
   float* colsum;
+  // kFwd epilogue (has_in = a residual is added; ld = out_features / fold)
+  int entries;                   // chunks stored per 64 columns: 2 with an activation (Z, then the output), else 1
+  int act, fold;
+  const bf16* bias;
   // kWgrad epilogue
   float* partial;
   unsigned long long split_stride;
@@ -172,7 +180,8 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
         const int kb0 = q.sp * T->kb_per_split;
         const int kb1 = min(T->kb_total, kb0 + T->kb_per_split);
         const int kb_per_seg = T->kb_per_seg, b_k_seg_stride = T->b_k_seg_stride;
-        const bool mn = T->kind == kWgrad;
+        const bool a_mn = T->kind == kWgrad, b_mn = T->kind != kDgrad;
+        const int b_mn_seg_stride = T->b_mn_seg_stride;
         int seg = kb0 / kb_per_seg, kk = (kb0 - seg * kb_per_seg) * BK;
         int bn = T->b_mn_wrap > 0 ? n0 % T->b_mn_wrap : n0;
         bn += (int)rank * LBNH;
@@ -187,13 +196,11 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
           const uint32_t bar = full_bar(stage);
           if (leader_cta) mbar_expect_tx(bar, 2u * LSTAGE_BYTES);
           const int bk = kk + seg * b_k_seg_stride;
-          if (!mn) {
-            tma_load_2d_pair(sa, &T->map_a, bar, kk, m0);
-            tma_load_2d_pair(sb, &T->map_b, bar, bk, bn);
-          } else {
-            tma_load_3d_pair(sa, &T->map_a, bar, 0, kk, m0 >> 6);
-            tma_load_3d_pair(sb, &T->map_b, bar, 0, bk, bn >> 6);
-          }
+          const int bnk = bn + seg * b_mn_seg_stride;
+          if (!a_mn) tma_load_2d_pair(sa, &T->map_a, bar, kk, m0);
+          else tma_load_3d_pair(sa, &T->map_a, bar, 0, kk, m0 >> 6);
+          if (!b_mn) tma_load_2d_pair(sb, &T->map_b, bar, bk, bnk);
+          else tma_load_3d_pair(sb, &T->map_b, bar, 0, bk, bnk >> 6);
           ++fills[stage];
           if (++stage == LSTAGES) { stage = 0; phase ^= 1u; }
           kk += BK;
@@ -228,12 +235,12 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
         const UnitPos q = unit_pos(T, u);
         const int kb0 = q.sp * T->kb_per_split;
         const int kb1 = min(T->kb_total, kb0 + T->kb_per_split);
-        const bool mn = T->kind == kWgrad;
-        const uint32_t idesc = make_idesc<TILE_M, LBN, false, false>() | (mn ? (3u << 15) : 0u);
-        const uint64_t desc_a0 = mn ? make_desc(base, CHUNK_BYTES, 1024) : make_desc(base, 16, 1024);
-        const uint64_t desc_b0 = mn ? make_desc(base + A_STAGE_BYTES, CHUNK_BYTES, 1024)
-                                    : make_desc(base + A_STAGE_BYTES, 16, 1024);
-        const uint32_t step = (mn ? 2048u : 32u) >> 4;
+        const bool a_mn = T->kind == kWgrad, b_mn = T->kind != kDgrad;
+        const uint32_t idesc = make_idesc<TILE_M, LBN, false, false>() | (a_mn ? (1u << 15) : 0u) | (b_mn ? (1u << 16) : 0u);
+        const uint64_t desc_a0 = a_mn ? make_desc(base, CHUNK_BYTES, 1024) : make_desc(base, 16, 1024);
+        const uint64_t desc_b0 = b_mn ? make_desc(base + A_STAGE_BYTES, CHUNK_BYTES, 1024)
+                                      : make_desc(base + A_STAGE_BYTES, 16, 1024);
+        const uint32_t step_a = (a_mn ? 2048u : 32u) >> 4, step_b = (b_mn ? 2048u : 32u) >> 4;
         ok = mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, status, kTimeoutMma);
         if (!ok) break;
         tc_fence_after();
@@ -246,7 +253,7 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
           const uint64_t db = desc_b0 + (uint64_t)((uint32_t)stage * (LSTAGE_BYTES >> 4));
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k)
-            tc_mma_pair(d_tmem, da + k * step, db + k * step, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+            tc_mma_pair(d_tmem, da + k * step_a, db + k * step_b, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           tc_commit_pair(empty_bar(stage));
           if (++stage == LSTAGES) { stage = 0; phase ^= 1u; }
         }
@@ -259,32 +266,35 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
     // ------------------------------------------------------------------ epilogue TMA thread of group g
     const int g = warp - (2 + 4 * EPI_GROUPS);
     if (lane == 0 && g < EPI_GROUPS) {
-      // Walks the kDgrad units of this CTA in list order, twice: once ahead, requesting the input chunks,
-      // once behind, storing finished chunks and signalling finished units.  Neither walk ever blocks the
-      // other: a request whose dependency is not met yet is simply retried on the next round.
+      // Walks the units with a staged epilogue (kDgrad, kFwd) of this CTA in list order, twice: once ahead,
+      // requesting the input chunks, once behind, storing finished chunks and signalling finished units.  Neither
+      // walk ever blocks the other: a request whose dependency is not met yet is simply retried on the next
+      // round.  What moves through a buffer set is an "entry": one per 64-column chunk, or two (Z, then the
+      // output) for a forward layer with an activation.
       struct Walk {
         int u, ti;
         bool valid;
         const Task* T;
-        int tm, m0, n0, nch, k;      // row tile, first row / column, chunks of this group in the unit, chunks done
+        int tm, m0, n0, nch, k, ent;  // row tile, first row / column, entries of this group in the unit, entries done, entries per chunk
       };
-      auto enter = [&](Walk& w) {      // position w on the kDgrad unit at or after w.u
+      auto enter = [&](Walk& w) {      // position w on the staged-epilogue unit at or after w.u
         w.valid = false;
         while (w.u < total_units) {
           const Task* T = find_task(tasks, w.ti, w.u);
-          if (T->kind == kDgrad) {
+          if (T->kind != kWgrad) {
             const UnitPos q = unit_pos(T, w.u);
             w.T = T; w.tm = q.tm;
             w.m0 = q.tm * TILE_M + (int)rank * BM; w.n0 = q.tn * LBN;
+            w.ent = T->kind == kFwd ? T->entries : 1;
             w.nch = 0;
-            for (int c = g; c < LNCHUNK; c += EPI_GROUPS) w.nch += (w.n0 + c * 64 < T->cols) ? 1 : 0;
+            for (int c = g; c < LNCHUNK; c += EPI_GROUPS) w.nch += (w.n0 + c * 64 < T->cols) ? w.ent : 0;
             w.k = 0; w.valid = true;
             return;
           }
           w.u += unit_step;
         }
       };
-      Walk fw{unit0, 0, false, nullptr, 0, 0, 0, 0, 0}, sw = fw;
+      Walk fw{unit0, 0, false, nullptr, 0, 0, 0, 0, 0, 1}, sw = fw;
       enter(fw);
       enter(sw);
       int fetched = 0, stored = 0;
@@ -318,7 +328,7 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
             fence_proxy_async_all();
             mbar_expect_tx(bar, EPI_CHUNK_BYTES);
             const uint32_t dst = epi_base + (uint32_t)((g * EPI_SETS + b) * EPI_CHUNK_BYTES);
-            tma_load_2d(dst, &T->map_in, bar, fw.n0 + (g + EPI_GROUPS * fw.k) * 64, fw.m0);
+            tma_load_2d(dst, &T->map_in, bar, fw.n0 + (g + EPI_GROUPS * (fw.k / fw.ent)) * 64, fw.m0);
           } else {
             mbar_arrive(bar);
           }
@@ -328,7 +338,8 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
         if (mbar_try_wait(out_ready_bar(g, stored & 1), (uint32_t)(stored >> 1) & 1u)) {
           if (sw.m0 < sw.T->rows) {
             const uint32_t src = epi_base + (uint32_t)((g * EPI_SETS + (stored & 1)) * EPI_CHUNK_BYTES);
-            tma_store_2d(&sw.T->map_out, src, sw.n0 + (g + EPI_GROUPS * sw.k) * 64, sw.m0);
+            const CUtensorMap* om = (sw.ent == 2 && (sw.k & 1) == 0) ? &sw.T->map_out2 : &sw.T->map_out;
+            tma_store_2d(om, src, sw.n0 + (g + EPI_GROUPS * (sw.k / sw.ent)) * 64, sw.m0);
           }
           tma_store_commit();
           tma_store_wait_read<0>();
@@ -392,6 +403,49 @@ gemm_list_kernel(const Task* __restrict__ tasks, const int total_units, unsigned
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_remote(acc_empty_bar(acc), 0u);
+      } else if (T->kind == kFwd) {
+        // Z = acc + bias; with an activation two entries per chunk: Z into buffer set j, a_{l+1} into set j + 1
+        FwdEpiS<2> epi;
+        epi.has_in[0] = T->has_in != 0; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = T->entries == 2;
+        epi.bias = T->bias; epi.fold = T->fold; epi.ld = T->ld; epi.act = T->act;
+        const int ent = T->entries;
+        int nch = 0;
+#pragma unroll
+        for (int c = 0; c < LNCHUNK; ++c) nch += ((c & 1) == g && n0 + c * 64 < cols) ? 1 : 0;
+        if (nch == 0) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(acc_empty_bar(acc), 0u);
+        }
+#pragma unroll 1
+        for (int i = 0; i < nch; ++i, j += ent) {
+          const int c = g + 2 * i;
+          const int col0 = n0 + c * 64;
+          const int bz = j & 1, bo = (j + ent - 1) & 1;          // buffer sets of Z (if stored) and of the output
+          ok = mbar_wait(in_full_bar(g, bz), (uint32_t)(j >> 1) & 1u, abort_flag, status, kTimeoutEpilogue);
+          if (ok && ent == 2)
+            ok = mbar_wait(in_full_bar(g, bo), (uint32_t)((j + 1) >> 1) & 1u, abort_flag, status, kTimeoutEpilogue);
+          if (!ok) break;
+          uint8_t* bufz = gen_base + LSTAGES * LSTAGE_BYTES + (g * EPI_SETS + bz) * EPI_CHUNK_BYTES;
+          uint8_t* bufo = gen_base + LSTAGES * LSTAGE_BYTES + (g * EPI_SETS + bo) * EPI_CHUNK_BYTES;
+#pragma unroll 1
+          for (int h = 0; h < 2; ++h) {                          // 32 columns at a time keeps the register count down
+            float v[32], s0[32], s1[32];
+            tmem_ld32(taddr + c * 64 + h * 32, v);
+            if (i == nch - 1 && h == 1) {                        // last read of this accumulator by this warp
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive_remote(acc_empty_bar(acc), 0u);
+            }
+            if (epi.has_in[0]) lds_row32(bufo, trow, h, s0);
+            epi.combine(col0 + h * 32, cols - (col0 + h * 32), v, s0, s1);
+            if (ent == 2) sts_row32(bufz, trow, h, s1);
+            sts_row32(bufo, trow, h, s0);
+          }
+          fence_async_smem();
+          mbar_arrive(out_ready_bar(g, bz));
+          if (ent == 2) mbar_arrive(out_ready_bar(g, bo));
+        }
       } else {
         DgradEpiS<1> epi;
         epi.has_in[0] = T->has_in != 0; epi.has_in[1] = false; epi.has_out[0] = true; epi.has_out[1] = false;
